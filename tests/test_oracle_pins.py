@@ -1,0 +1,438 @@
+"""Pins for the CPU oracle: every check here is against something other than the oracle
+itself -- a library routine on a special case, a closed form, an invariant, an identity,
+brute force on tiny vocabularies, or a figure printed in the paper."""
+import os
+
+import numpy as np
+import pytest
+from scipy.special import softmax as sp_softmax
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rng(seed):
+    return np.random.default_rng(seed)
+
+
+def _order(l):
+    """(logit desc, index asc) by a library sort."""
+    return np.lexsort((np.arange(l.size), -l.astype(np.float64)))
+
+
+# ---------------------------------------------------------------------------------------
+# compress: Eq. (4) top-k, plus top-p / renormalisation
+# ---------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("V,k,T", [(50, 5, 0.7), (333, 32, 1.0), (17, 17, 1.3), (9, 20, 0.5)])
+def test_topk_equals_library_topk_then_softmax(V, k, T):
+    # closed form: with pure top-k the full normaliser cancels, so the renormalised sparse
+    # row is the softmax over the k selected logits alone
+    rng = _rng(V * 1000 + k)
+    l = rng.normal(0, 3, size=(2, 3, V)).astype(np.float32)
+    Ts = np.array([T, T * 1.5], np.float32)
+    qi, qp, qc, _ = oracle.compress(l, Ts, top_k=k, top_p=1.0, k_max=k)
+    n = min(k, V)
+    for b in range(2):
+        for i in range(3):
+            sel = _order(l[b, i])[:n]
+            ref = sp_softmax(l[b, i, sel].astype(np.float64) / np.float64(Ts[b]))
+            assert qc[b, i] == n
+            assert np.array_equal(qi[b, i, :n], sel)
+            assert np.all(qi[b, i, n:] == -1) and np.all(qp[b, i, n:] == 0)
+            np.testing.assert_allclose(qp[b, i, :n], ref, rtol=2e-7, atol=0)
+
+
+def test_topk_ties_take_lower_index_first():
+    # integer logits force ties at the k-th value
+    rng = _rng(7)
+    l = rng.integers(-3, 4, size=(1, 4, 64)).astype(np.float32)
+    qi, qp, qc, _ = oracle.compress(l, np.ones(1, np.float32), top_k=10, top_p=1.0, k_max=10)
+    for i in range(4):
+        assert np.array_equal(qi[0, i], _order(l[0, i])[:10])
+    # all-equal logits: uniform over the first k indices
+    l = np.full((1, 1, 40), 2.5, np.float32)
+    qi, qp, qc, _ = oracle.compress(l, np.ones(1, np.float32), top_k=8, top_p=1.0, k_max=8)
+    assert np.array_equal(qi[0, 0], np.arange(8))
+    np.testing.assert_allclose(qp[0, 0], 1.0 / 8, rtol=1e-7)
+
+
+@pytest.mark.parametrize("top_p,k_max,top_k", [(0.9, 64, 0), (0.5, 64, 0), (0.95, 8, 0), (0.9, 64, 4),
+                                               (0.999, 200, 0)])
+def test_top_p_invariants(top_p, k_max, top_k):
+    rng = _rng(int(top_p * 1000) + k_max)
+    V = 200
+    ranks = rng.permuted(np.tile(np.arange(1, V + 1), (6, 1)), axis=1)
+    l = (-1.2 * np.log(ranks) + rng.normal(0, 1.0, size=(6, V))).astype(np.float32).reshape(2, 3, V)
+    T = np.array([0.8, 1.1], np.float32)
+    tp = np.float32(top_p)
+    qi, qp, qc, _ = oracle.compress(l, T, top_k=top_k, top_p=float(tp), k_max=k_max)
+    for b in range(2):
+        for i in range(3):
+            q = sp_softmax(l[b, i].astype(np.float64) / np.float64(T[b]))
+            order = _order(l[b, i])
+            cum = np.cumsum(q[order])
+            k_eff = min(top_k if top_k > 0 else k_max, k_max, V)
+            n = qc[b, i]
+            assert 1 <= n <= k_eff
+            # support is exactly the first n of the sorted order
+            assert np.array_equal(qi[b, i, :n], order[:n])
+            assert np.all(qi[b, i, n:] == -1) and np.all(qp[b, i, n:] == 0)
+            # nucleus rule: smallest prefix reaching top_p, capped at k_eff
+            if n < k_eff:
+                assert cum[n - 1] >= np.float64(tp)
+            if n > 1:
+                assert cum[n - 2] < np.float64(tp)
+            # renormalised: sums to one, proportional to q on the support
+            assert abs(qp[b, i, :n].astype(np.float64).sum() - 1.0) < 1e-6
+            np.testing.assert_allclose(qp[b, i, :n], q[order[:n]] / cum[n - 1], rtol=3e-7)
+
+
+def test_dense_limit_k_ge_V_gives_full_softmax():
+    rng = _rng(3)
+    V = 31
+    l = rng.normal(0, 2, size=(1, 2, V)).astype(np.float32)
+    T = np.array([0.9], np.float32)
+    qi, qp, qc, _ = oracle.compress(l, T, top_k=0, top_p=1.0, k_max=V + 5)
+    for i in range(2):
+        assert qc[0, i] == V
+        dense = np.zeros(V)
+        dense[qi[0, i, :V]] = qp[0, i, :V]
+        np.testing.assert_allclose(dense, sp_softmax(l[0, i].astype(np.float64) / np.float64(T[0])),
+                                   rtol=2e-7)
+
+
+def test_draft_token_draw_is_inverse_cdf_of_sparse_row():
+    rng = _rng(11)
+    V, k = 40, 6
+    l = rng.normal(0, 2, size=(1, 1, V)).astype(np.float32)
+    N = 4000
+    ls = np.repeat(l, N, axis=0)
+    u = ((np.arange(N) + 0.5) / N).astype(np.float32).reshape(N, 1)
+    qi, qp, qc, tok = oracle.compress(ls, np.ones(N, np.float32), top_k=k, top_p=1.0, k_max=k, u_draft=u)
+    # library inverse CDF
+    cum = np.cumsum(qp[0, 0].astype(np.float64))
+    ref = qi[0, 0][np.minimum(np.searchsorted(cum, u[:, 0].astype(np.float64) * cum[-1], side="right"), k - 1)]
+    assert np.array_equal(tok[:, 0], ref)
+    # empirical law of the draw equals the sparse row
+    for j in range(k):
+        assert abs(np.mean(tok[:, 0] == qi[0, 0, j]) - qp[0, 0, j]) < 2.0 / N + 1e-6
+
+
+# ---------------------------------------------------------------------------------------
+# verify: accept test, scan, residual mass
+# ---------------------------------------------------------------------------------------
+
+def test_q_equal_p_accepts_everything_and_residual_vanishes():
+    rng = _rng(5)
+    B, G, V = 6, 3, 23
+    lt = rng.normal(0, 2, size=(B, G + 1, V)).astype(np.float32)
+    T = rng.uniform(0.5, 1.5, size=B).astype(np.float32)
+    qi, qp, qc, _ = oracle.compress(lt[:, :G], T, top_k=0, top_p=1.0, k_max=V)
+    tok = rng.integers(0, V, size=(B, G)).astype(np.int32)
+    for u_val in (0.0, 0.3, 0.999):
+        u = np.full((B, G), u_val, np.float32)
+        r = oracle.verify(lt, T, tok, qi, qp, qc, u, u_resample=np.full((B, 2), 0.5, np.float32))
+        assert np.all(r["accept_len"] == G)
+        assert np.all(np.abs(r["resid_mass"]) < 1e-6)
+
+
+def test_scalar_q_reduces_to_textbook_speculative_test():
+    # K = 1: the sparse row holds only the drafted token and the probability the drafter gave it
+    # (the paper's uplink form); the decision is u < min(1, p(x)/q(x))
+    rng = _rng(9)
+    B, G, V = 400, 3, 12
+    lt = rng.normal(0, 1.5, size=(B, G + 1, V)).astype(np.float32)
+    T = np.full(B, 0.9, np.float32)
+    tok = rng.integers(0, V, size=(B, G)).astype(np.int32)
+    q = rng.uniform(0.02, 0.6, size=(B, G, 1)).astype(np.float32)
+    qi = tok.reshape(B, G, 1).copy()
+    qc = np.ones((B, G), np.int32)
+    u = rng.uniform(0, 1, size=(B, G)).astype(np.float32)
+    r = oracle.verify(lt, T, tok, qi, q, qc, u)
+    p = sp_softmax(lt.astype(np.float64) / np.float64(T[0]), axis=-1)
+    px = np.take_along_axis(p[:, :G], tok[..., None].astype(np.int64), axis=-1)[..., 0]
+    acc = u.astype(np.float64) < np.minimum(1.0, px / q[..., 0].astype(np.float64))
+    lead = np.where(acc.all(1), G, np.argmin(acc, axis=1))
+    assert np.array_equal(r["accept_len"], lead)
+    np.testing.assert_allclose(r["p_draft"], px, rtol=1e-12)
+    # residual with a single-entry q: 1 - min(p(x), q(x))
+    np.testing.assert_allclose(r["resid_mass"], 1.0 - np.minimum(px, q[..., 0]), rtol=1e-9)
+
+
+def test_token_outside_support_is_accepted():
+    rng = _rng(13)
+    B, G, V = 3, 2, 30
+    ld = rng.normal(0, 2, size=(B, G, V)).astype(np.float32)
+    lt = rng.normal(0, 2, size=(B, G + 1, V)).astype(np.float32)
+    T = np.ones(B, np.float32)
+    qi, qp, qc, _ = oracle.compress(ld, T, top_k=4, top_p=1.0, k_max=4)
+    tok = np.empty((B, G), np.int32)
+    for b in range(B):
+        for i in range(G):
+            tok[b, i] = [v for v in range(V) if v not in qi[b, i]][0]
+    r = oracle.verify(lt, T, tok, qi, qp, qc, np.full((B, G), 0.999, np.float32))
+    assert np.all(r["accept_len"] == G)
+
+
+def test_residual_mass_identity_and_accept_rate():
+    # R = 1 - sum_{v in S} min(p_v, q~_v); the mean accept indicator over u tends to 1 - R when
+    # the draft token is drawn from q~
+    rng = _rng(17)
+    G, V, k = 1, 64, 8
+    ld = rng.normal(0, 2, size=(1, G, V)).astype(np.float32)
+    lt = (0.6 * ld[0, 0] + rng.normal(0, 1.0, size=V)).astype(np.float32)
+    lt = np.stack([lt, rng.normal(0, 1, size=V).astype(np.float32)])[None]
+    T = np.array([0.8], np.float32)
+    N = 200000
+    u_d = rng.uniform(0, 1, size=(N, G)).astype(np.float32)
+    qi, qp, qc, tok = oracle.compress(np.repeat(ld, N, 0), np.repeat(T, N), top_k=k, top_p=1.0,
+                                      k_max=k, u_draft=u_d)
+    u = rng.uniform(0, 1, size=(N, G)).astype(np.float32)
+    r = oracle.verify(np.repeat(lt, N, 0), np.repeat(T, N), tok, qi, qp, qc, u, nthreads=4)
+    p = sp_softmax(lt[0, 0].astype(np.float64) / np.float64(T[0]))
+    R_id = 1.0 - np.minimum(p[qi[0, 0]], qp[0, 0].astype(np.float64)).sum()
+    np.testing.assert_allclose(r["resid_mass"][:, 0], R_id, rtol=1e-10)
+    rate = np.mean(r["accept_len"] == 1)
+    assert abs(rate - (1.0 - R_id)) < 4 * np.sqrt(0.25 / N)
+
+
+def test_borderline_count_only_counts_deciding_positions():
+    # build ratios by hand: p(x)/q(x) known from a two-token vocabulary
+    V, G = 2, 3
+    lt = np.zeros((1, G + 1, V), np.float32)            # p = (0.5, 0.5) everywhere
+    T = np.ones(1, np.float32)
+    tok = np.zeros((1, G), np.int32)
+    qi = np.zeros((1, G, 1), np.int32)
+    qp = np.full((1, G, 1), 0.8, np.float32)            # ratio = 0.5 / 0.8 (fp32 0.8 widened)
+    qc = np.ones((1, G), np.int32)
+    ratio = 0.5 / np.float64(np.float32(0.8))
+    near = np.float32(ratio)                            # within 6e-8 relative of the ratio
+    far = np.float32(ratio * (1 - 1e-3))
+    # position 0: far below -> accept, not borderline; position 1: near -> borderline, decides
+    # either way; position 2: near, but only counted if position 1 accepted
+    u = np.array([[far, near, near]], np.float32)
+    r = oracle.verify(lt, T, tok, qi, qp, qc, u)
+    acc1 = np.float64(near) < ratio
+    assert r["accept_len"][0] == (3 if acc1 else 1)
+    assert r["borderline_count"] == (2 if acc1 else 1)
+    # a rejection far from the threshold stops the count
+    u = np.array([[np.float32(0.9), near, near]], np.float32)
+    r = oracle.verify(lt, T, tok, qi, qp, qc, u)
+    assert r["accept_len"][0] == 0 and r["borderline_count"] == 0
+
+
+# ---------------------------------------------------------------------------------------
+# sampler: two-level inverse CDF and the residual distribution
+# ---------------------------------------------------------------------------------------
+
+def test_single_chunk_sampler_is_library_inverse_cdf():
+    rng = _rng(19)
+    V, N = 37, 3000
+    lt = rng.normal(0, 2, size=(1, 1, V)).astype(np.float32)
+    T = np.ones(N, np.float32)
+    u = rng.uniform(0, 1, size=(N, 2)).astype(np.float32)
+    tokens, mass = oracle.residual_sample(np.repeat(lt, N, 0), T, np.zeros(N, np.int32),
+                                          np.zeros((N, 0, 1), np.int32), np.zeros((N, 0, 1), np.float32),
+                                          np.zeros((N, 0), np.int32), u)
+    p = sp_softmax(lt[0, 0].astype(np.float64))
+    cum = np.cumsum(p)
+    ref = np.searchsorted(cum, u[:, 1].astype(np.float64) * cum[-1], side="right")
+    assert np.array_equal(tokens, np.minimum(ref, V - 1))
+    np.testing.assert_allclose(mass, 1.0, rtol=1e-12)
+
+
+@pytest.mark.parametrize("V,chunk,k", [(16, 4, 3), (13, 4, 5), (10, 3, 2)])
+def test_two_level_sampler_law_on_grid(V, chunk, k):
+    # brute force over a fine (u1, u2) grid: the area mapped to each token is r_v / R with
+    # r = max(0, p - q~) written straight from the paper's definition
+    rng = _rng(V * 7 + chunk)
+    ld = rng.normal(0, 1.5, size=(1, 1, V)).astype(np.float32)
+    lt = np.stack([(0.5 * ld[0, 0] + rng.normal(0, 1.2, size=V)).astype(np.float32),
+                   rng.normal(0, 1, size=V).astype(np.float32)])[None]
+    T = np.array([0.9], np.float32)
+    qi, qp, qc, _ = oracle.compress(ld, T, top_k=k, top_p=1.0, k_max=k)
+    n = 400
+    g = (np.arange(n) + 0.5) / n
+    u = np.stack(np.meshgrid(g, g, indexing="ij"), -1).reshape(-1, 2).astype(np.float32)
+    N = u.shape[0]
+    p = sp_softmax(lt[0].astype(np.float64) / np.float64(T[0]), axis=-1)
+    for pos in (0, 1):
+        tokens, mass = oracle.residual_sample(np.repeat(lt, N, 0), np.repeat(T, N),
+                                              np.full(N, pos, np.int32), np.repeat(qi, N, 0),
+                                              np.repeat(qp, N, 0), np.repeat(qc, N, 0), u,
+                                              chunk=chunk, nthreads=4)
+        if pos == 0:
+            qd = np.zeros(V)
+            qd[qi[0, 0, :k]] = qp[0, 0, :k]
+            r = np.maximum(0.0, p[0] - qd)
+        else:
+            r = p[1]
+        law = np.bincount(tokens, minlength=V) / N
+        np.testing.assert_allclose(law, r / r.sum(), atol=3.0 / n)
+        np.testing.assert_allclose(mass, r.sum(), rtol=1e-12)
+        # zero residual weight is never drawn
+        assert np.all(law[r == 0] == 0)
+
+
+def test_zero_residual_falls_back_to_p():
+    rng = _rng(23)
+    V = 20
+    lt = rng.normal(0, 2, size=(1, 2, V)).astype(np.float32)
+    T = np.ones(1, np.float32)
+    qi, qp, qc, _ = oracle.compress(lt[:, :1], T, top_k=0, top_p=1.0, k_max=V)
+    # make q~ >= p everywhere: scale the stored probabilities up slightly
+    qp = (qp * np.float32(1.001)).astype(np.float32)
+    u = np.array([[0.3, 0.7]], np.float32)
+    t_res, _ = oracle.residual_sample(lt, T, np.zeros(1, np.int32), qi, qp, qc, u)
+    empty = (np.zeros((1, 1, 1), np.int32), np.zeros((1, 1, 1), np.float32), np.zeros((1, 1), np.int32))
+    t_p, _ = oracle.residual_sample(lt, T, np.zeros(1, np.int32), *empty, u)
+    assert t_res[0] == t_p[0]
+
+
+# ---------------------------------------------------------------------------------------
+# whole method: output law equals the target distribution (Sec. 2.1 / Sec. 3.3 claim)
+# ---------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("V,k,top_p,chunk", [(16, 5, 1.0, 4), (12, 12, 0.8, 5), (8, 3, 1.0, 1024)])
+def test_output_law_equals_target_per_position(V, k, top_p, chunk):
+    # Monte Carlo over all uniforms with the draft token drawn from q~: conditional on reaching
+    # position i, the emitted token at i follows p_i
+    rng = _rng(V + k)
+    G, N = 3, 400000
+    ld = rng.normal(0, 1.5, size=(1, G, V)).astype(np.float32)
+    lt = np.concatenate([(0.7 * ld[0] + rng.normal(0, 0.9, size=(G, V))).astype(np.float32),
+                         rng.normal(0, 1, size=(1, V)).astype(np.float32)])[None]
+    T = np.array([0.85], np.float32)
+    Ts = np.repeat(T, N)
+    qi, qp, qc, tok = oracle.compress(np.repeat(ld, N, 0), Ts, top_k=k, top_p=top_p, k_max=k,
+                                      u_draft=rng.uniform(0, 1, size=(N, G)).astype(np.float32),
+                                      nthreads=4)
+    r = oracle.verify(np.repeat(lt, N, 0), Ts, tok, qi, qp, qc,
+                      rng.uniform(0, 1, size=(N, G)).astype(np.float32),
+                      u_resample=rng.uniform(0, 1, size=(N, 2)).astype(np.float32),
+                      chunk=chunk, nthreads=4)
+    p = sp_softmax(lt[0].astype(np.float64) / np.float64(T[0]), axis=-1)
+    a = r["accept_len"]
+    for i in range(G + 1):
+        reach = a >= i
+        emitted = np.where(a[reach] > i, tok[reach, min(i, G - 1)], r["token"][reach])
+        n_i = reach.sum()
+        assert n_i > 5000
+        law = np.bincount(emitted, minlength=V) / n_i
+        sigma = np.sqrt(p[i] * (1 - p[i]) / n_i)
+        assert np.all(np.abs(law - p[i]) < 4.5 * sigma + 1e-9), (i, np.abs(law - p[i]).max())
+
+
+def test_exact_law_by_enumeration_tiny():
+    # V = 4, gamma = 1: enumerate the draft token over the support and integrate the uniforms
+    # on a grid fine enough that the discretisation error is below the tolerance
+    rng = _rng(29)
+    V, k = 4, 2
+    ld = rng.normal(0, 1, size=(1, 1, V)).astype(np.float32)
+    lt = rng.normal(0, 1, size=(1, 2, V)).astype(np.float32)
+    T = np.ones(1, np.float32)
+    qi, qp, qc, _ = oracle.compress(ld, T, top_k=k, top_p=1.0, k_max=k)
+    p = sp_softmax(lt[0, 0].astype(np.float64))
+    n = 160
+    g = ((np.arange(n) + 0.5) / n).astype(np.float32)
+    ua, u1, u2 = [x.reshape(-1) for x in np.meshgrid(g, g, g, indexing="ij")]
+    N = ua.size
+    law = np.zeros(V)
+    for j in range(k):
+        tok = np.full((N, 1), qi[0, 0, j], np.int32)
+        r = oracle.verify(np.repeat(lt, N, 0), np.ones(N, np.float32), tok, np.repeat(qi, N, 0),
+                          np.repeat(qp, N, 0), np.repeat(qc, N, 0), ua.reshape(N, 1),
+                          u_resample=np.stack([u1, u2], -1), chunk=2, nthreads=4)
+        out = np.where(r["accept_len"] == 1, tok[:, 0], r["token"])
+        law += float(qp[0, 0, j]) * np.bincount(out, minlength=V) / N
+    np.testing.assert_allclose(law, p, atol=2.5 / n)
+
+
+def test_expected_length_matches_eq5():
+    rows = [ln.split() for ln in open(os.path.join(GOLDEN, "expected_length.txt")) if ln[0] not in "#\n"]
+    rng = _rng(31)
+    V = 2
+    for alpha_s, gamma_s, el_s in rows:
+        alpha, G, EL = float(alpha_s), int(gamma_s), float(el_s)
+        # two-token vocabulary, q~ = (1, 0) on token 0, p = (alpha, 1 - alpha): the accept
+        # probability of the (always drafted) token 0 is exactly alpha at every position
+        N = 200000 if alpha > 0 else 1000
+        if alpha > 0:
+            lt = np.log(np.array([alpha, 1 - alpha])).astype(np.float32)
+        else:
+            lt = np.array([-np.inf, 0.0], np.float32)
+        lt = np.tile(lt, (N, G + 1, 1))
+        tok = np.zeros((N, G), np.int32)
+        qi = np.zeros((N, G, 1), np.int32)
+        qp = np.ones((N, G, 1), np.float32)
+        qc = np.ones((N, G), np.int32)
+        u = rng.uniform(0, 1, size=(N, G)).astype(np.float32)
+        r = oracle.verify(lt, np.ones(N, np.float32), tok, qi, qp, qc, u, nthreads=4)
+        gen_len = np.minimum(r["accept_len"] + 1, G)       # Eq. (5) caps the cycle at gamma
+        assert abs(gen_len.mean() - EL) < 0.01, (alpha, gen_len.mean(), EL)
+        # with the bonus row the per-call yield is (1 - alpha^(gamma+1)) / (1 - alpha)
+        full = (1 - alpha ** (G + 1)) / (1 - alpha)
+        assert abs((r["accept_len"] + 1).mean() - full) < 0.012
+
+
+# ---------------------------------------------------------------------------------------
+# printed figures and degenerate inputs
+# ---------------------------------------------------------------------------------------
+
+def test_sparse_layout_matches_printed_payload_sizes():
+    vals = {}
+    for ln in open(os.path.join(GOLDEN, "payload_sizes.txt")):
+        ln = ln.split("#")[0].split()
+        if ln:
+            vals[ln[0]] = ln[1:]
+    V = int(vals["vocab_llama31"][0])
+    K = int(vals["topk_example_k"][0])
+    l = np.zeros((1, 1, V), np.float32)
+    qi, qp, qc, _ = oracle.compress(l, np.ones(1, np.float32), top_k=K, top_p=1.0, k_max=K)
+    entry = qi.dtype.itemsize + qp.dtype.itemsize
+    assert entry == 8
+    assert qi[0, 0].nbytes + qp[0, 0].nbytes == int(vals["topk_row_bytes"][0]) < int(vals["topk_row_bytes"][2])
+    full = V * qp.dtype.itemsize
+    assert full == int(vals["full_row_bytes"][0])
+    assert abs(full - int(vals["full_row_bytes"][2])) / full < 0.03
+    g = int(vals["uplink_gamma"][0])
+    assert g * entry == int(vals["uplink_bytes"][0]) < int(vals["uplink_bytes"][2])
+
+
+def test_minus_inf_logits_have_zero_weight():
+    V = 10
+    l = np.full((1, 2, V), -np.inf, np.float32)
+    l[0, :, [2, 7]] = 0.0
+    T = np.ones(1, np.float32)
+    qi, qp, qc, _ = oracle.compress(l[:, :1], T, top_k=4, top_p=1.0, k_max=4)
+    assert list(qi[0, 0, :2]) == [2, 7]
+    np.testing.assert_allclose(qp[0, 0], [0.5, 0.5, 0, 0])
+    for u2 in (0.1, 0.6, 0.99):
+        t, _ = oracle.residual_sample(l, T, np.array([1], np.int32), qi, qp, qc,
+                                      np.array([[0.5, u2]], np.float32))
+        assert t[0] in (2, 7)
+
+
+def test_invalid_inputs_are_flagged_not_sampled():
+    rng = _rng(37)
+    B, G, V = 4, 2, 16
+    ld = rng.normal(size=(B, G, V)).astype(np.float32)
+    lt = rng.normal(size=(B, G + 1, V)).astype(np.float32)
+    T = np.ones(B, np.float32)
+    ld[1, 0, 3] = np.nan
+    qi, qp, qc, tok = oracle.compress(ld, T, top_k=4, top_p=1.0, k_max=4,
+                                      u_draft=np.full((B, G), 0.5, np.float32))
+    assert qc[1, 0] == -1 and tok[1, 0] == -1 and np.all(qi[1, 0] == -1)
+    assert qc[0, 0] == 4 and qc[1, 1] == 4
+    lt[2, 1, 5] = np.inf
+    T2 = T.copy()
+    T2[3] = 0.0
+    u = np.full((B, G), 0.5, np.float32)
+    r = oracle.verify(lt, T2, np.where(tok < 0, 0, tok), qi, qp, qc, u,
+                      u_resample=np.full((B, 2), 0.5, np.float32))
+    assert r["accept_len"][0] >= 0 and r["token"][0] >= 0
+    for b in (1, 2, 3):           # bad count / +inf logit / zero temperature
+        assert r["accept_len"][b] == -1 and r["token"][b] == -1
+        assert np.all(r["p_draft"][b] == -1) and np.all(r["resid_mass"][b] == -1)

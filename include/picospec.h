@@ -1,0 +1,155 @@
+/*
+ * picospec.h -- C-ABI of the B200 (sm_100a) hot path of PicoSpec's separate rejection
+ * sampling with sparse compression (arXiv 2603.19133, Sec. 3.3).
+ *
+ * Conventions for every entry point
+ *   - Array arguments are DEVICE pointers owned by the caller unless a comment says "host".
+ *     The library never frees or keeps them beyond the asynchronous work it enqueues.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default
+ *     stream).  No entry point synchronises the stream except picospec_status.
+ *   - The library allocates device memory only inside picospec_create; the three hot calls
+ *     allocate nothing.  A context owns a workspace that the hot calls use as scratch, so
+ *     calls on one context must be ordered (one stream at a time); use one context per stream
+ *     for concurrent work.
+ *   - Logits are row-major with the vocabulary contiguous: element (b, i, v) of a
+ *     [B, R, V] tensor lives at base + ((b * R + i) * row_stride_elems + v), R = G for draft
+ *     logits and G + 1 for target logits.  row_stride_elems >= V.  Rows whose base address and
+ *     pitch are 16-byte aligned take the 128-bit load path; other rows are read element-wise.
+ *   - The return value reports errors the host can see (bad arguments, capacity, CUDA launch
+ *     errors).  Data errors found by kernels (NaN or +inf logits, a row of -inf only, a
+ *     temperature that is not finite and > 0, token / index / count / position out of range)
+ *     set bits of a sticky device status word and mark the affected outputs with -1; no kernel
+ *     traps or asserts.
+ *   - Decisions that floating point takes (accept test, top-p cut, inverse-CDF thresholds) are
+ *     taken in fp32-accumulated arithmetic when they are clear of their threshold by more than
+ *     the accumulated rounding error, and re-taken in double precision otherwise; the number of
+ *     rows that needed the double-precision pass is reported by picospec_status.
+ */
+#ifndef PICOSPEC_H_
+#define PICOSPEC_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define PICOSPEC_API __attribute__((visibility("default")))
+#else
+#define PICOSPEC_API
+#endif
+
+typedef struct picospec_ctx picospec_ctx; /* opaque: workspace, status word, capacities */
+
+typedef enum { PICOSPEC_F32 = 0, PICOSPEC_BF16 = 1 } picospec_dtype;
+
+typedef enum {
+    PICOSPEC_OK = 0,
+    PICOSPEC_EINVAL = -1,    /* null pointer, negative size, top_p <= 0, unknown dtype ...      */
+    PICOSPEC_ECUDA = -2,     /* a CUDA runtime call failed; see picospec_last_cuda_error        */
+    PICOSPEC_ECAPACITY = -3, /* B, G, V or k_max exceed what the context was created for        */
+    PICOSPEC_EDATA = -4      /* reported by picospec_status only: a kernel found bad data       */
+} picospec_err;
+
+/* bits of the device status word */
+#define PICOSPEC_ST_TEMPERATURE 1 /* temperature not finite or <= 0                              */
+#define PICOSPEC_ST_LOGIT 2       /* NaN or +inf logit, or a row with no finite logit            */
+#define PICOSPEC_ST_RANGE 4       /* draft token, sparse index, count or position out of range   */
+
+#define PICOSPEC_CHUNK 1024 /* vocabulary entries per level-1 chunk of the residual sampler      */
+#define PICOSPEC_MAX_K 1024 /* largest k_max a context accepts                                   */
+#define PICOSPEC_MAX_GAMMA 64
+
+/* Create a context on CUDA device `device` able to serve calls with B <= max_batch,
+ * G <= max_gamma, V <= max_vocab, k_max <= max_k.  Allocates the workspace (a few MB for the
+ * paper's vocabularies).  *out is host memory.  Returns PICOSPEC_OK or an error. */
+PICOSPEC_API int picospec_create(picospec_ctx** out, int device, int max_batch, int max_gamma, int max_vocab, int max_k);
+
+/* Free the workspace.  The caller makes sure no enqueued work still uses the context. */
+PICOSPEC_API int picospec_destroy(picospec_ctx* ctx);
+
+/* Static, never-freed description of an error code. */
+PICOSPEC_API const char* picospec_strerror(int err);
+
+/* cudaError_t of the last failing CUDA call made through this context (0 if none). */
+PICOSPEC_API int picospec_last_cuda_error(const picospec_ctx* ctx);
+
+/* Synchronise `cuda_stream`, then copy the sticky status word and the cumulative number of rows
+ * re-evaluated in double precision to HOST memory (either pointer may be NULL).  If `clear` is
+ * non-zero both are reset afterwards.  Returns PICOSPEC_EDATA if the status word is non-zero. */
+PICOSPEC_API int picospec_status(picospec_ctx* ctx, int* device_status_out, long long* slow_path_rows_out, int clear,
+                    void* cuda_stream);
+
+/* Half 1 -- draft-side sparse compression (Sec. 3.3, Eq. (4): keep the K most probable entries
+ * with their vocabulary indices; this build applies it to the drafter's distribution, adds the
+ * top-p cut and renormalises).
+ *
+ * For every row (b, i) of draft_logits [B, G, V]:
+ *   q      = softmax(logits / temperature[b])
+ *   order  = vocabulary sorted by (logit descending, index ascending)
+ *   k_eff  = min(top_k > 0 ? top_k : k_max, k_max, V)
+ *   n      = k_eff, or with top_p < 1 the smallest n >= 1 whose first n entries of `order`
+ *            reach cumulative probability >= top_p, capped at k_eff
+ *   q_idx[b,i,j]  = order[j],  q_prob[b,i,j] = q[order[j]] / sum_{j'<n} q[order[j']]   (j < n)
+ *   q_idx[b,i,j]  = -1,        q_prob[b,i,j] = 0                                      (j >= n)
+ *   q_count[b,i]  = n
+ * If u_draft and draft_tok are non-NULL, draft_tok[b,i] is drawn from the sparse row by inverse
+ * CDF in stored order with the uniform u_draft[b,i] in [0,1) (the drafter's own sampling step;
+ * the output law of the method is exact only if the candidate comes from this same q~).
+ * A row with bad data gets q_count = -1, q_idx = -1, q_prob = 0, draft_tok = -1.
+ *
+ * temperature [B] fp32 > 0; q_idx, q_prob [B, G, k_max]; q_count [B, G]; u_draft, draft_tok
+ * [B, G] or both NULL.  top_k = 0 disables top-k; top_p >= 1 disables top-p; top_p must be > 0.
+ */
+PICOSPEC_API int picospec_compress(picospec_ctx* ctx, const void* draft_logits, picospec_dtype dtype, int B, int G, int V,
+                      long long row_stride_elems, const float* temperature, int top_k, float top_p, int k_max,
+                      int* q_idx, float* q_prob, int* q_count, const float* u_draft, int* draft_tok,
+                      void* cuda_stream);
+
+/* Half 2a -- target-side verification (Sec. 3.3: the verifier decides each candidate from the
+ * probability the drafter gave it; Sec. 2.1: the speculative-sampling accept rule).
+ *
+ * For every sequence b, with p_i = softmax(target_logits[b, i, :] / temperature[b]), i in [0, G]:
+ *   x = draft_tok[b,i];  qx = q_prob of x in sparse row (b,i), 0 if absent
+ *   accept_i  = (qx == 0) or u_accept[b,i] < min(1, p_i(x) / qx)
+ *   p_draft[b,i]    = p_i(x)
+ *   resid_mass[b,i] = sum_v max(0, p_i(v) - q~_i(v))                       (every i < G)
+ *   accept_len[b]   = number of leading accepted positions, in [0, G]
+ *   *borderline_count = number, over the whole call, of deciding accept tests (every accepted
+ *                       one and the first rejected one of each sequence) with
+ *                       |p_i(x)/qx - u| <= 1e-6 * u
+ * If u_resample and token are non-NULL the call also performs half 2b at position
+ * accept_len[b] (residual at a rejected position, p itself at the bonus row G).
+ * A sequence with bad data gets accept_len = -1, token = -1, p_draft = resid_mass = -1.
+ *
+ * target_logits [B, G+1, V]; draft_tok [B, G]; q_idx, q_prob [B, G, k_max]; q_count [B, G];
+ * u_accept [B, G] fp32 in [0,1); accept_len [B]; p_draft, resid_mass [B, G] fp32;
+ * borderline_count [1] int32; u_resample [B, 2] fp32 in [0,1); token [B].
+ */
+PICOSPEC_API int picospec_verify(picospec_ctx* ctx, const void* target_logits, picospec_dtype dtype, int B, int G, int V,
+                    long long row_stride_elems, const float* temperature, const int* draft_tok, const int* q_idx,
+                    const float* q_prob, const int* q_count, int k_max, const float* u_accept, int* accept_len,
+                    float* p_draft, float* resid_mass, int* borderline_count, const float* u_resample,
+                    int* token, void* cuda_stream);
+
+/* Half 2b -- local resampling (Sec. 3.3: the corrected token is drawn from
+ * norm(max(0, P_j(x) - Q_j(x)))).
+ *
+ * For every sequence b, row j = pos[b] of its target logits: weights r_v = max(0, p_j(v) - q~_j(v))
+ * if j < G and the sparse row (b, j) is non-empty, else r_v = p_j(v) (bonus row; also the
+ * fallback when the residual is identically zero).  The token is drawn by a two-level inverse
+ * CDF with chunks of PICOSPEC_CHUNK vocabulary entries: u_resample[b,0] picks the first chunk c
+ * whose cumulative mass exceeds u0 * sum(r); u_resample[b,1] picks the first entry of that chunk
+ * whose cumulative weight inside the chunk exceeds u1 * mass(c).  Entries of zero weight are
+ * never drawn.  mass[b] (optional) = sum_v r_v.
+ *
+ * pos [B] in [0, G]; other arrays as in picospec_verify; token [B]; mass [B] fp32 or NULL.
+ */
+PICOSPEC_API int picospec_residual_sample(picospec_ctx* ctx, const void* target_logits, picospec_dtype dtype, int B, int G,
+                             int V, long long row_stride_elems, const float* temperature, const int* pos,
+                             const int* q_idx, const float* q_prob, const int* q_count, int k_max,
+                             const float* u_resample, int* token, float* mass, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PICOSPEC_H_ */

@@ -1,0 +1,195 @@
+"""Thin ctypes binding of the picospec C-ABI (include/picospec.h).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels of
+libpicospec.so.  torch supplies device memory and the current stream.  There is no CPU
+fallback: a missing library or a non-CUDA tensor raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+from . import buildlib as _build
+
+F32, BF16 = 0, 1
+OK, EINVAL, ECUDA, ECAPACITY, EDATA = 0, -1, -2, -3, -4
+CHUNK = 1024
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libpicospec.so (built in-tree by build.build()); fail loudly if it is absent."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if not os.path.exists(path):
+            path = _build.build()
+        L = ctypes.CDLL(path)
+        c_int, c_ll, c_f, vp = ctypes.c_int, ctypes.c_longlong, ctypes.c_float, ctypes.c_void_p
+        L.picospec_create.argtypes = [ctypes.POINTER(vp), c_int, c_int, c_int, c_int, c_int]
+        L.picospec_destroy.argtypes = [vp]
+        L.picospec_strerror.argtypes = [c_int]
+        L.picospec_strerror.restype = ctypes.c_char_p
+        L.picospec_last_cuda_error.argtypes = [vp]
+        L.picospec_status.argtypes = [vp, ctypes.POINTER(c_int), ctypes.POINTER(c_ll), c_int, vp]
+        L.picospec_compress.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, vp, c_int, c_f, c_int,
+                                        vp, vp, vp, vp, vp, vp]
+        L.picospec_verify.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp, c_int,
+                                      vp, vp, vp, vp, vp, vp, vp, vp]
+        L.picospec_residual_sample.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp,
+                                               c_int, vp, vp, vp, vp]
+        for f in ("picospec_create", "picospec_destroy", "picospec_last_cuda_error", "picospec_status",
+                  "picospec_compress", "picospec_verify", "picospec_residual_sample"):
+            getattr(L, f).restype = c_int
+        _lib = L
+    return _lib
+
+
+class PicospecError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {lib().picospec_strerror(code).decode()} ({code})")
+
+
+def _check(code: int, what: str):
+    if code != OK:
+        raise PicospecError(code, what)
+
+
+def _ptr(t: Optional[torch.Tensor], dtype: Optional[torch.dtype] = None, shape: Optional[Tuple[int, ...]] = None):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("picospec takes CUDA tensors only (there is no CPU path)")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"expected shape {tuple(shape)}, got {tuple(t.shape)}")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _logits(t: torch.Tensor):
+    """[B, R, V] logits with a contiguous vocabulary and uniformly pitched rows."""
+    if not t.is_cuda or t.dim() != 3 or t.stride(2) != 1:
+        raise ValueError("logits must be a CUDA tensor [B, R, V] with contiguous vocabulary")
+    B, R, V = t.shape
+    pitch = t.stride(1) if R > 1 else (t.stride(0) if B > 1 else V)
+    if (R > 1 and B > 1 and t.stride(0) != R * pitch) or pitch < V:
+        raise ValueError("rows must be uniformly pitched")
+    if t.dtype == torch.float32:
+        dt = F32
+    elif t.dtype == torch.bfloat16:
+        dt = BF16
+    else:
+        raise ValueError("logits must be float32 or bfloat16")
+    return ctypes.c_void_p(t.data_ptr()), dt, B, R, V, pitch
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Context:
+    """Owns the library's workspace on one device.  Calls on one context must be ordered on
+    one stream at a time; use one context per stream for concurrent work."""
+
+    def __init__(self, max_batch: int, max_gamma: int, max_vocab: int, max_k: int, device: Optional[int] = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("picospec needs a CUDA device")
+        self.device = torch.cuda.current_device() if device is None else int(device)
+        self._h = ctypes.c_void_p()
+        _check(lib().picospec_create(ctypes.byref(self._h), self.device, max_batch, max_gamma, max_vocab, max_k),
+               "picospec_create")
+        self.max_batch, self.max_gamma, self.max_vocab, self.max_k = max_batch, max_gamma, max_vocab, max_k
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            lib().picospec_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def status(self, clear: bool = False) -> Tuple[int, int]:
+        """Synchronise the current stream; return (status word, rows re-evaluated in double)."""
+        st, slow = ctypes.c_int(0), ctypes.c_longlong(0)
+        rc = lib().picospec_status(self._h, ctypes.byref(st), ctypes.byref(slow), int(clear), _stream())
+        if rc not in (OK, EDATA):
+            raise PicospecError(rc, "picospec_status")
+        return st.value, slow.value
+
+    # -- half 1 -------------------------------------------------------------------------
+    def compress(self, draft_logits: torch.Tensor, temperature: torch.Tensor, top_k: int, top_p: float,
+                 k_max: int, u_draft: Optional[torch.Tensor] = None, out=None):
+        """picospec_compress.  Returns (q_idx [B,G,k_max] i32, q_prob f32, q_count [B,G] i32,
+        draft_tok [B,G] i32 or None)."""
+        p, dt, B, G, V, pitch = _logits(draft_logits)
+        dev = draft_logits.device
+        if out is None:
+            q_idx = torch.empty((B, G, k_max), dtype=torch.int32, device=dev)
+            q_prob = torch.empty((B, G, k_max), dtype=torch.float32, device=dev)
+            q_count = torch.empty((B, G), dtype=torch.int32, device=dev)
+            tok = torch.empty((B, G), dtype=torch.int32, device=dev) if u_draft is not None else None
+        else:
+            q_idx, q_prob, q_count, tok = out
+        _check(lib().picospec_compress(
+            self._h, p, dt, B, G, V, pitch, _ptr(temperature, torch.float32, (B,)), int(top_k), float(top_p),
+            int(k_max), _ptr(q_idx, torch.int32, (B, G, k_max)), _ptr(q_prob, torch.float32, (B, G, k_max)),
+            _ptr(q_count, torch.int32, (B, G)), _ptr(u_draft, torch.float32, (B, G)),
+            _ptr(tok, torch.int32, (B, G)), _stream()), "picospec_compress")
+        return q_idx, q_prob, q_count, tok
+
+    # -- half 2a (+2b fused) ------------------------------------------------------------
+    def verify(self, target_logits: torch.Tensor, temperature: torch.Tensor, draft_tok: torch.Tensor,
+               q_idx: torch.Tensor, q_prob: torch.Tensor, q_count: torch.Tensor, u_accept: torch.Tensor,
+               u_resample: Optional[torch.Tensor] = None, out=None):
+        """picospec_verify.  Returns dict(accept_len [B], p_draft [B,G], resid_mass [B,G],
+        borderline_count [1], token [B] or None)."""
+        p, dt, B, G1, V, pitch = _logits(target_logits)
+        G = G1 - 1
+        k_max = q_idx.shape[-1]
+        dev = target_logits.device
+        if out is None:
+            out = {
+                "accept_len": torch.empty((B,), dtype=torch.int32, device=dev),
+                "p_draft": torch.empty((B, G), dtype=torch.float32, device=dev),
+                "resid_mass": torch.empty((B, G), dtype=torch.float32, device=dev),
+                "borderline_count": torch.empty((1,), dtype=torch.int32, device=dev),
+                "token": torch.empty((B,), dtype=torch.int32, device=dev) if u_resample is not None else None,
+            }
+        _check(lib().picospec_verify(
+            self._h, p, dt, B, G, V, pitch, _ptr(temperature, torch.float32, (B,)),
+            _ptr(draft_tok, torch.int32, (B, G)), _ptr(q_idx, torch.int32, (B, G, k_max)),
+            _ptr(q_prob, torch.float32, (B, G, k_max)), _ptr(q_count, torch.int32, (B, G)), int(k_max),
+            _ptr(u_accept, torch.float32, (B, G)), _ptr(out["accept_len"], torch.int32, (B,)),
+            _ptr(out["p_draft"], torch.float32, (B, G)), _ptr(out["resid_mass"], torch.float32, (B, G)),
+            _ptr(out["borderline_count"], torch.int32, (1,)), _ptr(u_resample, torch.float32, (B, 2)),
+            _ptr(out["token"], torch.int32, (B,)), _stream()), "picospec_verify")
+        return out
+
+    # -- half 2b ---------------------------------------------------------------------
+    def residual_sample(self, target_logits: torch.Tensor, temperature: torch.Tensor, pos: torch.Tensor,
+                        q_idx: torch.Tensor, q_prob: torch.Tensor, q_count: torch.Tensor,
+                        u_resample: torch.Tensor, want_mass: bool = True):
+        """picospec_residual_sample.  Returns (token [B] i32, mass [B] f32 or None)."""
+        p, dt, B, G1, V, pitch = _logits(target_logits)
+        G = G1 - 1
+        k_max = q_idx.shape[-1] if G > 0 else 1
+        dev = target_logits.device
+        token = torch.empty((B,), dtype=torch.int32, device=dev)
+        mass = torch.empty((B,), dtype=torch.float32, device=dev) if want_mass else None
+        _check(lib().picospec_residual_sample(
+            self._h, p, dt, B, G, V, pitch, _ptr(temperature, torch.float32, (B,)), _ptr(pos, torch.int32, (B,)),
+            _ptr(q_idx, torch.int32), _ptr(q_prob, torch.float32), _ptr(q_count, torch.int32), int(k_max),
+            _ptr(u_resample, torch.float32, (B, 2)), _ptr(token, torch.int32, (B,)),
+            _ptr(mass, torch.float32, (B,)), _stream()), "picospec_residual_sample")
+        return token, mass

@@ -1,0 +1,298 @@
+// C-ABI of the picospec library: context, argument checks, kernel launches.  See picospec.h.
+#include "../../include/picospec.h"
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdlib.h>
+
+#include "compress_kernels.cuh"
+#include "verify_kernels.cuh"
+
+using namespace picospec;
+
+struct picospec_ctx {
+    int device;
+    int max_batch, max_gamma, max_vocab, max_k;
+    int num_sms;
+    int last_cuda_error;
+    unsigned long long compress_calls;
+    // workspace
+    float2* stats;
+    double* dsum;
+    float* row_max;
+    int* queue;
+    int* counters;  // [0] verify queue count, [1],[2] compress queue counts (alternating)
+    unsigned* status;
+    unsigned long long* slow_rows;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) ok = false;
+        if (ok && prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        target = dev;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0 && prev != target) cudaSetDevice(prev);
+    }
+    int target;
+};
+
+int fail_cuda(picospec_ctx* ctx, cudaError_t e) {
+    if (ctx) ctx->last_cuda_error = (int)e;
+    return PICOSPEC_ECUDA;
+}
+
+bool rows_aligned(const void* base, long long row_stride, int elem) {
+    return ((uintptr_t)base % 16 == 0) && ((row_stride * elem) % 16 == 0);
+}
+
+template <typename T> void set_compress_attrs() {
+    cudaFuncSetAttribute(compress_kernel<T, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, COMPRESS_SMEM);
+    cudaFuncSetAttribute(compress_kernel<T, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, COMPRESS_SMEM);
+    cudaFuncSetAttribute(compress_kernel<T, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, COMPRESS_SMEM);
+    cudaFuncSetAttribute(compress_kernel<T, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, COMPRESS_SMEM);
+}
+
+template <typename T>
+cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool aligned, cudaStream_t s) {
+    const int rows = a.B * a.G;
+    const int grid = rows < ctx->num_sms * 2 ? rows : ctx->num_sms * 2;
+    const bool stats = a.top_p < 1.0f;
+    if (aligned) {
+        if (stats) compress_kernel<T, true, true><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+        else compress_kernel<T, true, false><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+    } else {
+        if (stats) compress_kernel<T, false, true><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+        else compress_kernel<T, false, false><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || !stats) return e;
+    // rows whose top-p cut was too close to call: exact normaliser, then redo the cut
+    PreciseArgs p;
+    p.logits = a.logits; p.row_stride = a.row_stride; p.V = a.V; p.nch = a.nch;
+    p.seq_rows = a.G; p.expand = 1; p.pos = nullptr; p.temperature = a.temperature;
+    p.queue = a.queue; p.queue_count = a.queue_count; p.row_max = a.row_max; p.dsum = a.dsum;
+    precise_chunk_sums_kernel<T><<<ctx->num_sms * 2, THREADS, 0, s>>>(p);
+    const int g2 = rows < ctx->num_sms ? rows : ctx->num_sms;
+    compress_precise_kernel<T><<<g2, THREADS, MAX_K * 8, s>>>(a);
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, cudaStream_t s) {
+    const long long items = (long long)(a.sample_only ? a.B : a.B * (a.G + 1)) * a.nch;
+    long long want = (items + WARPS - 1) / WARPS;
+    const int cap = ctx->num_sms * 4;
+    const int grid = (int)(want < cap ? want : cap);
+    if (aligned) chunk_stats_kernel<T, true><<<grid, THREADS, 0, s>>>(a);
+    else chunk_stats_kernel<T, false><<<grid, THREADS, 0, s>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const size_t dyn = (size_t)a.nch * sizeof(double);
+    verify_finish_kernel<T, false><<<a.B, THREADS, dyn, s>>>(a);
+    PreciseArgs p;
+    p.logits = a.logits; p.row_stride = a.row_stride; p.V = a.V; p.nch = a.nch;
+    p.seq_rows = a.G + 1; p.expand = a.sample_only ? 1 : a.G + 1; p.pos = a.sample_only ? a.pos : nullptr;
+    p.temperature = a.temperature; p.queue = a.queue; p.queue_count = a.queue_count;
+    p.row_max = a.row_max; p.dsum = a.dsum;
+    precise_chunk_sums_kernel<T><<<ctx->num_sms * 2, THREADS, 0, s>>>(p);
+    const int g2 = a.B < ctx->num_sms ? a.B : ctx->num_sms;
+    verify_finish_kernel<T, true><<<g2, THREADS, dyn, s>>>(a);
+    return cudaGetLastError();
+}
+
+int check_common(const picospec_ctx* ctx, const void* logits, int dtype, int B, int G, int V, long long row_stride,
+                 const float* temperature, int k_max) {
+    if (!ctx || !logits || !temperature) return PICOSPEC_EINVAL;
+    if (dtype != PICOSPEC_F32 && dtype != PICOSPEC_BF16) return PICOSPEC_EINVAL;
+    if (B < 0 || G < 0 || V <= 0 || k_max <= 0 || row_stride < V) return PICOSPEC_EINVAL;
+    if (B > ctx->max_batch || G > ctx->max_gamma || V > ctx->max_vocab || k_max > ctx->max_k)
+        return PICOSPEC_ECAPACITY;
+    return PICOSPEC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int picospec_create(picospec_ctx** out, int device, int max_batch, int max_gamma, int max_vocab, int max_k) {
+    if (!out) return PICOSPEC_EINVAL;
+    *out = nullptr;
+    if (device < 0 || max_batch <= 0 || max_gamma < 0 || max_gamma > PICOSPEC_MAX_GAMMA || max_vocab <= 0 ||
+        max_vocab > (1 << 22) || max_k <= 0 || max_k > PICOSPEC_MAX_K)
+        return PICOSPEC_EINVAL;
+    picospec_ctx* ctx = (picospec_ctx*)calloc(1, sizeof(picospec_ctx));
+    if (!ctx) return PICOSPEC_EINVAL;
+    ctx->device = device;
+    ctx->max_batch = max_batch;
+    ctx->max_gamma = max_gamma;
+    ctx->max_vocab = max_vocab;
+    ctx->max_k = max_k;
+    DeviceGuard g(device);
+    cudaError_t e = g.ok ? cudaSuccess : cudaErrorInvalidDevice;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, device);
+    const size_t rows = (size_t)max_batch * (max_gamma + 1);
+    const size_t nch = ((size_t)max_vocab + CHUNK - 1) / CHUNK;
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->stats, rows * nch * sizeof(float2));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->dsum, rows * nch * sizeof(double));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->row_max, rows * sizeof(float));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->queue, rows * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->counters, 4 * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->status, sizeof(unsigned));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->slow_rows, sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(ctx->counters, 0, 4 * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(unsigned));
+    if (e == cudaSuccess) e = cudaMemset(ctx->slow_rows, 0, sizeof(unsigned long long));
+    if (e == cudaSuccess) {
+        set_compress_attrs<float>();
+        set_compress_attrs<__nv_bfloat16>();
+        e = cudaGetLastError();
+    }
+    if (e != cudaSuccess) {
+        picospec_destroy(ctx);
+        return PICOSPEC_ECUDA;
+    }
+    *out = ctx;
+    return PICOSPEC_OK;
+}
+
+int picospec_destroy(picospec_ctx* ctx) {
+    if (!ctx) return PICOSPEC_EINVAL;
+    DeviceGuard g(ctx->device);
+    cudaFree(ctx->stats);
+    cudaFree(ctx->dsum);
+    cudaFree(ctx->row_max);
+    cudaFree(ctx->queue);
+    cudaFree(ctx->counters);
+    cudaFree(ctx->status);
+    cudaFree(ctx->slow_rows);
+    free(ctx);
+    return PICOSPEC_OK;
+}
+
+const char* picospec_strerror(int err) {
+    switch (err) {
+        case PICOSPEC_OK: return "ok";
+        case PICOSPEC_EINVAL: return "invalid argument";
+        case PICOSPEC_ECUDA: return "CUDA runtime error";
+        case PICOSPEC_ECAPACITY: return "problem size exceeds the context's capacity";
+        case PICOSPEC_EDATA: return "a kernel found bad data (see the status word)";
+        default: return "unknown error";
+    }
+}
+
+int picospec_last_cuda_error(const picospec_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+int picospec_status(picospec_ctx* ctx, int* device_status_out, long long* slow_path_rows_out, int clear,
+                    void* cuda_stream) {
+    if (!ctx) return PICOSPEC_EINVAL;
+    DeviceGuard g(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    unsigned st = 0;
+    unsigned long long slow = 0;
+    cudaError_t e = cudaMemcpyAsync(&st, ctx->status, sizeof(st), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&slow, ctx->slow_rows, sizeof(slow), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && clear) {
+        e = cudaMemsetAsync(ctx->status, 0, sizeof(unsigned), s);
+        if (e == cudaSuccess) e = cudaMemsetAsync(ctx->slow_rows, 0, sizeof(unsigned long long), s);
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    if (device_status_out) *device_status_out = (int)st;
+    if (slow_path_rows_out) *slow_path_rows_out = (long long)slow;
+    return st ? PICOSPEC_EDATA : PICOSPEC_OK;
+}
+
+int picospec_compress(picospec_ctx* ctx, const void* draft_logits, picospec_dtype dtype, int B, int G, int V,
+                      long long row_stride_elems, const float* temperature, int top_k, float top_p, int k_max,
+                      int* q_idx, float* q_prob, int* q_count, const float* u_draft, int* draft_tok,
+                      void* cuda_stream) {
+    int rc = check_common(ctx, draft_logits, (int)dtype, B, G, V, row_stride_elems, temperature, k_max);
+    if (rc != PICOSPEC_OK) return rc;
+    if (!q_idx || !q_prob || !q_count || top_k < 0 || !(top_p > 0.0f)) return PICOSPEC_EINVAL;
+    if ((u_draft == nullptr) != (draft_tok == nullptr)) return PICOSPEC_EINVAL;
+    if (B == 0 || G == 0) return PICOSPEC_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
+    CompressArgs a;
+    a.logits = draft_logits; a.row_stride = row_stride_elems;
+    a.B = B; a.G = G; a.V = V; a.nch = (V + CHUNK - 1) / CHUNK; a.k_max = k_max; a.top_k = top_k; a.top_p = top_p;
+    a.temperature = temperature; a.q_idx = q_idx; a.q_prob = q_prob; a.q_count = q_count;
+    a.u_draft = u_draft; a.draft_tok = draft_tok;
+    a.row_max = ctx->row_max; a.dsum = ctx->dsum; a.queue = ctx->queue;
+    const int cur = 1 + (int)(ctx->compress_calls & 1ull);
+    a.queue_count = ctx->counters + cur;
+    a.queue_count_next = ctx->counters + (3 - cur);
+    ctx->compress_calls++;
+    a.status = ctx->status; a.slow_rows = ctx->slow_rows;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e;
+    if (dtype == PICOSPEC_BF16)
+        e = launch_compress<__nv_bfloat16>(ctx, a, rows_aligned(draft_logits, row_stride_elems, 2), s);
+    else
+        e = launch_compress<float>(ctx, a, rows_aligned(draft_logits, row_stride_elems, 4), s);
+    return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
+}
+
+static int verify_common(picospec_ctx* ctx, VerifyArgs& a, picospec_dtype dtype, void* cuda_stream) {
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
+    a.nch = (a.V + CHUNK - 1) / CHUNK;
+    a.stats = ctx->stats; a.row_max = ctx->row_max; a.dsum = ctx->dsum; a.queue = ctx->queue;
+    a.queue_count = ctx->counters; a.status = ctx->status; a.slow_rows = ctx->slow_rows;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e;
+    if (dtype == PICOSPEC_BF16)
+        e = launch_verify<__nv_bfloat16>(ctx, a, rows_aligned(a.logits, a.row_stride, 2), s);
+    else
+        e = launch_verify<float>(ctx, a, rows_aligned(a.logits, a.row_stride, 4), s);
+    return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
+}
+
+int picospec_verify(picospec_ctx* ctx, const void* target_logits, picospec_dtype dtype, int B, int G, int V,
+                    long long row_stride_elems, const float* temperature, const int* draft_tok, const int* q_idx,
+                    const float* q_prob, const int* q_count, int k_max, const float* u_accept, int* accept_len,
+                    float* p_draft, float* resid_mass, int* borderline_count, const float* u_resample,
+                    int* token, void* cuda_stream) {
+    int rc = check_common(ctx, target_logits, (int)dtype, B, G, V, row_stride_elems, temperature, k_max);
+    if (rc != PICOSPEC_OK) return rc;
+    if (!accept_len || !borderline_count) return PICOSPEC_EINVAL;
+    if (G > 0 && (!draft_tok || !q_idx || !q_prob || !q_count || !u_accept || !p_draft || !resid_mass))
+        return PICOSPEC_EINVAL;
+    if ((u_resample == nullptr) != (token == nullptr)) return PICOSPEC_EINVAL;
+    if (B == 0) return PICOSPEC_OK;
+    VerifyArgs a;
+    a.logits = target_logits; a.row_stride = row_stride_elems;
+    a.B = B; a.G = G; a.V = V; a.k_max = k_max; a.sample_only = 0;
+    a.temperature = temperature; a.draft_tok = draft_tok; a.q_idx = q_idx; a.q_prob = q_prob; a.q_count = q_count;
+    a.u_accept = u_accept; a.pos = nullptr; a.u_resample = u_resample;
+    a.accept_len = accept_len; a.p_draft = p_draft; a.resid_mass = resid_mass; a.borderline = borderline_count;
+    a.token = token; a.mass = nullptr;
+    return verify_common(ctx, a, dtype, cuda_stream);
+}
+
+int picospec_residual_sample(picospec_ctx* ctx, const void* target_logits, picospec_dtype dtype, int B, int G,
+                             int V, long long row_stride_elems, const float* temperature, const int* pos,
+                             const int* q_idx, const float* q_prob, const int* q_count, int k_max,
+                             const float* u_resample, int* token, float* mass, void* cuda_stream) {
+    int rc = check_common(ctx, target_logits, (int)dtype, B, G, V, row_stride_elems, temperature, k_max);
+    if (rc != PICOSPEC_OK) return rc;
+    if (!pos || !u_resample || !token) return PICOSPEC_EINVAL;
+    if (G > 0 && (!q_idx || !q_prob || !q_count)) return PICOSPEC_EINVAL;
+    if (B == 0) return PICOSPEC_OK;
+    VerifyArgs a;
+    a.logits = target_logits; a.row_stride = row_stride_elems;
+    a.B = B; a.G = G; a.V = V; a.k_max = k_max; a.sample_only = 1;
+    a.temperature = temperature; a.draft_tok = nullptr; a.q_idx = q_idx; a.q_prob = q_prob; a.q_count = q_count;
+    a.u_accept = nullptr; a.pos = pos; a.u_resample = u_resample;
+    a.accept_len = nullptr; a.p_draft = nullptr; a.resid_mass = nullptr; a.borderline = nullptr;
+    a.token = token; a.mass = mass;
+    return verify_common(ctx, a, dtype, cuda_stream);
+}
+
+}  // extern "C"

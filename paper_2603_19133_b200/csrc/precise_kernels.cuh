@@ -1,0 +1,53 @@
+// Double-precision chunk sums for rows whose fp32 statistics were too close to a decision
+// threshold.  One warp per (queued row, chunk): sum of exp(l/T - max/T) over the chunk, exactly
+// the terms of the definition.  The whole grid shares the work, so a handful of flagged rows
+// costs microseconds; with an empty queue every CTA returns at once.
+#pragma once
+#include "common.cuh"
+
+namespace picospec {
+
+struct PreciseArgs {
+    const void* logits;
+    long long row_stride;
+    int V, nch;
+    int seq_rows;              // rows per sequence in the logits tensor (G or G+1)
+    int expand;                // rows per queue entry: entry e covers rows e*expand .. +expand-1
+    const int* pos;            // optional: entry b covers the single row b*seq_rows + pos[b]
+    const float* temperature;  // [B]
+    const int* queue;
+    const int* queue_count;
+    const float* row_max;      // [rows] exact row maxima from the fp32 pass
+    double* dsum;              // [rows, nch]
+};
+
+template <typename T>
+__global__ void __launch_bounds__(THREADS) precise_chunk_sums_kernel(PreciseArgs a) {
+    const int nq = *a.queue_count;
+    if (nq == 0) return;
+    const int lane = threadIdx.x & 31;
+    const long long gw = (long long)blockIdx.x * WARPS + (threadIdx.x >> 5);
+    const long long nw = (long long)gridDim.x * WARPS;
+    const long long total = (long long)nq * a.expand * a.nch;
+    for (long long item = gw; item < total; item += nw) {
+        const int c = (int)(item % a.nch);
+        const long long t = item / a.nch;
+        const int ri = (int)(t % a.expand);
+        const int e = a.queue[(int)(t / a.expand)];
+        const int src_row = a.pos ? e * a.seq_rows + a.pos[e] : e * a.expand + ri;
+        const int b = src_row / a.seq_rows;
+        const T* row = reinterpret_cast<const T*>(a.logits) + (long long)src_row * a.row_stride;
+        const double Td = (double)a.temperature[b];
+        const double m = (double)a.row_max[src_row] / Td;
+        double s = 0.0;
+        const int v0 = c * CHUNK;
+        for (int k = lane; k < CHUNK; k += 32) {
+            const int v = v0 + k;
+            if (v < a.V) s += exp((double)load_logit(row, v) / Td - m);
+        }
+        s = warp_sum(s);
+        if (lane == 0) a.dsum[(long long)src_row * a.nch + c] = s;
+    }
+}
+
+}  // namespace picospec

@@ -1,0 +1,497 @@
+// Target-side kernels: streaming chunk statistics, per-sequence finish (accept test, scan,
+// residual mass, two-level sampler) and the double-precision re-evaluation of flagged sequences.
+#pragma once
+#include "common.cuh"
+#include "precise_kernels.cuh"
+
+namespace picospec {
+
+struct VerifyArgs {
+    const void* logits;        // target logits [B, G+1, V]
+    long long row_stride;      // elements
+    int B, G, V, nch, k_max;
+    int sample_only;           // 1: residual_sample entry point (row pos[b] only)
+    const float* temperature;  // [B]
+    const int* draft_tok;      // [B,G]
+    const int* q_idx;          // [B,G,k_max]
+    const float* q_prob;
+    const int* q_count;        // [B,G]
+    const float* u_accept;     // [B,G]
+    const int* pos;            // [B] (sample_only)
+    const float* u_resample;   // [B,2] or null
+    int* accept_len;           // [B]
+    float* p_draft;            // [B,G]
+    float* resid_mass;         // [B,G]
+    int* borderline;           // [1]
+    int* token;                // [B] or null
+    float* mass;               // [B] or null (sample_only)
+    // workspace
+    float2* stats;             // [B*(G+1), nch]: (chunk max logit, sum of 2^(l*c32 - max*c32))
+    float* row_max;            // [B*(G+1)]
+    double* dsum;              // [B*(G+1), nch]: exact chunk sums of flagged sequences
+    int* queue;                // [B] flagged sequences
+    int* queue_count;          // [1]
+    unsigned* status;          // sticky status word
+    unsigned long long* slow_rows;  // cumulative rows re-evaluated in double precision
+};
+
+// ---------------------------------------------------------------------------------------------
+// Streaming pass: one warp per 1024-entry chunk, software-pipelined over two register buffers.
+// Per chunk: exact maximum logit and the fp32 sum of 2^((l - max) * log2e / T).
+// ---------------------------------------------------------------------------------------------
+template <typename T> struct ItemMeta {
+    const T* row;
+    int v0;
+    float c32;
+    long long slot;  // index into stats
+    bool valid;
+};
+
+template <typename T> __device__ __forceinline__ ItemMeta<T> decode_item(const VerifyArgs& a, long long item) {
+    ItemMeta<T> m;
+    const int r = (int)(item / a.nch);
+    const int c = (int)(item - (long long)r * a.nch);
+    int b, src_row;
+    m.valid = true;
+    if (a.sample_only) {
+        b = r;
+        const int j = a.pos[b];
+        if (j < 0 || j > a.G) m.valid = false;
+        src_row = b * (a.G + 1) + (m.valid ? j : 0);
+    } else {
+        b = r / (a.G + 1);
+        src_row = r;
+    }
+    const float Tb = a.temperature[b];
+    if (!temp_ok(Tb)) m.valid = false;
+    m.c32 = temp_scale(Tb);
+    m.row = reinterpret_cast<const T*>(a.logits) + (long long)src_row * a.row_stride;
+    m.v0 = c * CHUNK;
+    m.slot = (long long)src_row * a.nch + c;
+    return m;
+}
+
+template <typename T> __device__ __forceinline__ void chunk_stats_compute(const ChunkRegs<T>& regs, const ItemMeta<T>& m,
+                                                                          float2* stats, int lane) {
+    const float lm = regs.lane_max();
+    // NaN anywhere in the chunk: the exp-sum below turns NaN and the finish kernel reports it
+    const float cm = warp_max(lm);
+    const float off = __fmul_rn(cm, m.c32);
+    float s = 0.f;
+    if (cm > -CUDART_INF_F) s = lane_exp_sum(regs, m.c32, off);
+    if (lm != lm) s = CUDART_NAN_F;
+    s = warp_sum(s);
+    if (lane == 0) stats[m.slot] = make_float2(cm, s);
+}
+
+template <typename T, bool ALIGNED>
+__global__ void __launch_bounds__(THREADS, 4) chunk_stats_kernel(VerifyArgs a) {
+    const int lane = threadIdx.x & 31;
+    const long long gw = (long long)blockIdx.x * WARPS + (threadIdx.x >> 5);
+    const long long nw = (long long)gridDim.x * WARPS;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        *a.queue_count = 0;
+        if (a.borderline) *a.borderline = 0;
+    }
+    const long long total = (long long)(a.sample_only ? a.B : a.B * (a.G + 1)) * a.nch;
+    long long itA = gw;
+    if (itA >= total) return;
+    ChunkRegs<T> A, Bf;
+    ItemMeta<T> mA = decode_item<T>(a, itA), mB;
+    if (mA.valid) A.template load<ALIGNED>(mA.row, mA.v0, a.V, lane);
+    for (;;) {
+        const long long itB = itA + nw;
+        const bool hasB = itB < total;
+        if (hasB) {
+            mB = decode_item<T>(a, itB);
+            if (mB.valid) Bf.template load<ALIGNED>(mB.row, mB.v0, a.V, lane);
+        }
+        if (mA.valid) chunk_stats_compute<T>(A, mA, a.stats, lane);
+        if (!hasB) break;
+        itA = itB + nw;
+        const bool hasA = itA < total;
+        if (hasA) {
+            mA = decode_item<T>(a, itA);
+            if (mA.valid) A.template load<ALIGNED>(mA.row, mA.v0, a.V, lane);
+        }
+        if (mB.valid) chunk_stats_compute<T>(Bf, mB, a.stats, lane);
+        if (!hasA) break;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Finish: one CTA per sequence.
+// ---------------------------------------------------------------------------------------------
+struct FinishShared {
+    double Z[MAX_G1];     // normaliser on the scale of Weight<>
+    double Zraw[MAX_G1];  // the same sum on the streaming pass's own scale (fast path)
+    float mx[MAX_G1];
+    int bad;
+    int acc[MAX_G1], amb[MAX_G1], bord[MAX_G1];
+    double warp_tot[WARPS];
+    double red[WARPS];
+    int tok, last, flag;
+    int cstar;
+    double Rtot;
+    float qloc[CHUNK];
+};
+
+template <typename T, bool PRECISE>
+__device__ __forceinline__ void row_stats(const VerifyArgs& a, int src_row, float c32, int lane, double& Z,
+                                          double& Zraw, float& mx, bool& bad) {
+    // combine the chunk statistics of one row (called by a full warp)
+    bad = false;
+    if (PRECISE) {
+        mx = a.row_max[src_row];
+        double s = 0.0;
+        for (int c = lane; c < a.nch; c += 32) s += a.dsum[(long long)src_row * a.nch + c];
+        Z = warp_sum(s);
+    } else {
+        const float2* st = a.stats + (long long)src_row * a.nch;
+        float m = -CUDART_INF_F;
+        bool nan = false;
+        for (int c = lane; c < a.nch; c += 32) {
+            float2 v = st[c];
+            m = fmaxf(m, v.x);
+            nan |= (v.y != v.y);
+        }
+        m = warp_max(m);
+        nan = __any_sync(0xffffffffu, nan);
+        mx = m;
+        bad = nan || !(m > -CUDART_INF_F) || !(m < CUDART_INF_F);
+        double s = 0.0;
+        if (!bad) {
+            const double off = (double)__fmul_rn(m, c32);
+            for (int c = lane; c < a.nch; c += 32) {
+                float2 v = st[c];
+                if (v.x > -CUDART_INF_F) s += (double)v.y * exp2((double)__fmul_rn(v.x, c32) - off);
+            }
+        }
+        Zraw = warp_sum(s);
+        if (!(Zraw > 0.0)) bad = true;
+        Z = bad ? 0.0 : Zraw * stream_sum_scale(m, c32);
+    }
+}
+
+template <typename T, bool PRECISE>
+__global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
+    extern __shared__ double cm[];  // [nch] chunk masses of the sampled row
+    __shared__ FinishShared sh;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int G = a.G, G1 = a.G + 1;
+
+    const int nloop = PRECISE ? *a.queue_count : a.B;
+    for (int slot = blockIdx.x; slot < nloop; slot += gridDim.x) {
+        const int b = PRECISE ? a.queue[slot] : slot;
+        const float Tb = a.temperature[b];
+        const float c32 = temp_scale(Tb);
+        const T* seq = reinterpret_cast<const T*>(a.logits) + (long long)b * G1 * a.row_stride;
+        unsigned st_bits = 0;
+        if (!temp_ok(Tb)) st_bits |= ST_TEMPERATURE;
+        __syncthreads();
+        if (tid == 0) {
+            sh.bad = 0;
+            sh.flag = 0;
+        }
+        __syncthreads();
+
+        // ---- 1. normaliser of every row that is needed ------------------------------------
+        int jpos = -1;
+        if (a.sample_only) {
+            jpos = a.pos[b];
+            if (jpos < 0 || jpos > G) st_bits |= ST_RANGE;
+        }
+        if (!st_bits) {
+            for (int i = warp; i < G1; i += WARPS) {
+                if (a.sample_only && i != jpos) continue;
+                double Z, Zraw;
+                float mx;
+                bool bad;
+                row_stats<T, PRECISE>(a, b * G1 + i, c32, lane, Z, Zraw, mx, bad);
+                if (lane == 0) {
+                    sh.Z[i] = Z;
+                    sh.Zraw[i] = Zraw;
+                    sh.mx[i] = mx;
+                    if (!PRECISE) a.row_max[b * G1 + i] = mx;
+                    if (bad) atomicOr(&sh.bad, (int)ST_LOGIT);
+                }
+            }
+        }
+        __syncthreads();
+
+        // ---- 2. per draft position: p(x), q~(x), accept test, residual mass ----------------
+        if (!st_bits && !sh.bad && !a.sample_only) {
+            for (int i = warp; i < G; i += WARPS) {
+                const int ri = b * G + i;
+                const int x = a.draft_tok[ri];
+                const int n = a.q_count[ri];
+                bool range_bad = (x < 0 || x >= a.V || n < 0 || n > a.k_max);
+                const T* row = seq + (long long)i * a.row_stride;
+                Weight<PRECISE> wt;
+                wt.init(Tb, sh.mx[i]);
+                const double Z = sh.Z[i];
+                double smin = 0.0;
+                float qx = 0.f;
+                int kx = 0x7fffffff;
+                if (!range_bad) {
+                    const int* idx = a.q_idx + (long long)ri * a.k_max;
+                    const float* prob = a.q_prob + (long long)ri * a.k_max;
+                    for (int k = lane; k < n; k += 32) {
+                        const int v = idx[k];
+                        if (v < 0 || v >= a.V) {
+                            range_bad = true;
+                            continue;
+                        }
+                        const double qk = (double)prob[k];
+                        const double pk = wt(load_logit(row, v)) / Z;
+                        smin += fmin(pk, qk);
+                        if (v == x && k < kx) kx = k;
+                    }
+                }
+                range_bad = __any_sync(0xffffffffu, range_bad);
+                smin = warp_sum(smin);
+#pragma unroll
+                for (int d = 16; d > 0; d >>= 1) kx = min(kx, __shfl_xor_sync(0xffffffffu, kx, d));
+                if (lane == 0) {
+                    if (range_bad) {
+                        atomicOr(&sh.bad, (int)ST_RANGE);
+                    } else {
+                        if (kx != 0x7fffffff) qx = a.q_prob[(long long)ri * a.k_max + kx];
+                        const double px = wt(load_logit(row, x)) / Z;
+                        const double u = (double)a.u_accept[ri];
+                        int acc = 1, amb = 0, bord = 0;
+                        if (qx > 0.f) {
+                            const double ratio = px / (double)qx;
+                            acc = u < fmin(1.0, ratio);
+                            const double dist = fabs(ratio - u);
+                            if (PRECISE)
+                                bord = dist <= BORDER_REL * u;
+                            else
+                                amb = dist <= (BORDER_REL + GUARD_Z) * fmax(u, ratio);
+                        }
+                        sh.acc[i] = acc;
+                        sh.amb[i] = amb;
+                        sh.bord[i] = bord;
+                        double R = 1.0 - smin;
+                        if (R < 0.0) R = 0.0;
+                        a.p_draft[ri] = (float)px;
+                        a.resid_mass[ri] = (float)R;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        st_bits |= (unsigned)sh.bad;
+
+        // ---- 3. first-rejection scan -----------------------------------------------------
+        int alen = 0, nborder = 0;
+        bool flagged = false;
+        if (!st_bits && !a.sample_only) {
+            while (alen < G && sh.acc[alen]) ++alen;
+            const int last = alen < G ? alen : G - 1;
+            for (int i = 0; i <= last; ++i) {
+                flagged |= sh.amb[i] != 0;
+                nborder += sh.bord[i];
+            }
+        }
+
+        // ---- 4. residual / bonus sample --------------------------------------------------
+        int token = -1;
+        double Rtot = -1.0;
+        const bool want_token = a.token != nullptr;
+        if (!st_bits && want_token) {
+            const int j = a.sample_only ? jpos : alen;
+            const int rj = b * G + j;
+            int n = 0;
+            if (j < G) {
+                n = a.q_count[rj];
+                if (n < 0 || n > a.k_max) {
+                    n = 0;
+                    st_bits |= ST_RANGE;
+                }
+            }
+            const int* idx = a.q_idx + (long long)rj * a.k_max;
+            const float* prob = a.q_prob + (long long)rj * a.k_max;
+            const T* row = seq + (long long)j * a.row_stride;
+            Weight<PRECISE> wt;
+            wt.init(Tb, sh.mx[j]);
+            const double Z = sh.Z[j];
+            bool use_resid = n > 0;
+            for (int pass = 0; pass < 2 && !st_bits; ++pass) {
+                // chunk masses (in units where the row sums to one)
+                if (PRECISE) {
+                    for (int c = tid; c < a.nch; c += THREADS) cm[c] = a.dsum[(long long)(b * G1 + j) * a.nch + c] / Z;
+                } else {
+                    const float2* st = a.stats + (long long)(b * G1 + j) * a.nch;
+                    const double off = (double)__fmul_rn(sh.mx[j], c32);
+                    const double Zraw = sh.Zraw[j];
+                    for (int c = tid; c < a.nch; c += THREADS) {
+                        float2 v = st[c];
+                        cm[c] = v.x > -CUDART_INF_F ? (double)v.y * exp2((double)__fmul_rn(v.x, c32) - off) / Zraw : 0.0;
+                    }
+                }
+                __syncthreads();
+                if (use_resid) {
+                    bool rb = false;
+                    for (int k = tid; k < n; k += THREADS) {
+                        const int v = idx[k];
+                        if (v < 0 || v >= a.V) {
+                            rb = true;
+                            continue;
+                        }
+                        const double pk = wt(load_logit(row, v)) / Z;
+                        atomicAdd(&cm[v / CHUNK], -fmin(pk, (double)prob[k]));
+                    }
+                    if (rb) atomicOr(&sh.bad, (int)ST_RANGE);
+                }
+                __syncthreads();
+                // level 1 by warp 0: lanes own contiguous blocks of chunks
+                if (warp == 0) {
+                    const int per = (a.nch + 31) / 32;
+                    const int c0 = lane * per, c1 = min(a.nch, c0 + per);
+                    double s = 0.0;
+                    for (int c = c0; c < c1; ++c) {
+                        double m = cm[c];
+                        if (m < 0.0) {
+                            m = 0.0;
+                            cm[c] = 0.0;
+                        }
+                        s += m;
+                    }
+                    double incl = s;
+#pragma unroll
+                    for (int d = 1; d < 32; d <<= 1) {
+                        double y = __shfl_up_sync(0xffffffffu, incl, d);
+                        if (lane >= d) incl += y;
+                    }
+                    const double R = __shfl_sync(0xffffffffu, incl, 31);
+                    const double thr = (double)a.u_resample[2 * b] * R;
+                    double run = incl - s;
+                    int first = 0x7fffffff, lastpos = -1;
+                    double mind = 1e300;
+                    for (int c = c0; c < c1; ++c) {
+                        const double m = cm[c];
+                        run += m;
+                        if (m > 0.0) lastpos = c;
+                        if (run > thr && first == 0x7fffffff) first = c;
+                        mind = fmin(mind, fabs(run - thr));
+                    }
+#pragma unroll
+                    for (int d = 16; d > 0; d >>= 1) {
+                        first = min(first, __shfl_xor_sync(0xffffffffu, first, d));
+                        lastpos = max(lastpos, __shfl_xor_sync(0xffffffffu, lastpos, d));
+                        mind = fmin(mind, __shfl_xor_sync(0xffffffffu, mind, d));
+                    }
+                    if (lane == 0) {
+                        sh.cstar = first != 0x7fffffff ? first : lastpos;
+                        sh.Rtot = R;
+                        // every prefix and the total carry an absolute error <= GUARD_Z
+                        if (!PRECISE && mind <= GUARD_Z) sh.flag = 1;
+                    }
+                }
+                __syncthreads();
+                Rtot = sh.Rtot;
+                if (!use_resid) break;
+                // the residual may vanish (q~ >= p everywhere): then the draw is from p itself
+                const double tiny = PRECISE ? 1e-12 : 4.0 * GUARD_Z;
+                if (Rtot > tiny) break;
+                if (!PRECISE) {
+                    if (tid == 0) sh.flag = 1;   // too close to zero to call in fp32
+                    break;
+                }
+                use_resid = false;  // precise: residual is zero, fall back to p
+                __syncthreads();
+            }
+            st_bits |= (unsigned)sh.bad;
+            const int cs = st_bits ? -1 : sh.cstar;
+            if (!st_bits && cs >= 0) {
+                // level 2: the 1024 entries of chunk cs, four consecutive entries per thread
+                const int v0 = cs * CHUNK;
+                for (int k = tid; k < CHUNK; k += THREADS) sh.qloc[k] = 0.f;
+                if (tid == 0) {
+                    sh.tok = 0x7fffffff;
+                    sh.last = -1;
+                }
+                __syncthreads();
+                if (use_resid)
+                    for (int k = tid; k < n; k += THREADS) {
+                        const int v = idx[k];
+                        if (v >= v0 && v < v0 + CHUNK) sh.qloc[v - v0] = prob[k];
+                    }
+                __syncthreads();
+                double r[4], cum[4], qsum = 0.0, loc = 0.0;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int v = v0 + tid * 4 + e;
+                    double w = 0.0;
+                    if (v < a.V) w = wt(load_logit(row, v)) / Z;
+                    const double q = (double)sh.qloc[tid * 4 + e];
+                    qsum += q;
+                    double d = w - q;
+                    r[e] = d > 0.0 ? d : 0.0;
+                    loc += r[e];
+                    cum[e] = loc;
+                }
+                double M;
+                const double incl = block_scan_incl(loc, sh.warp_tot, M);
+                const double base = incl - loc;
+                double Q;
+                block_scan_incl(qsum, sh.warp_tot, Q);
+                const double thr2 = (double)a.u_resample[2 * b + 1] * M;
+                int mine = 0x7fffffff, mylast = -1;
+#pragma unroll
+                for (int e = 3; e >= 0; --e) {
+                    if (base + cum[e] > thr2) mine = v0 + tid * 4 + e;
+                    if (r[e] > 0.0 && mylast < 0) mylast = v0 + tid * 4 + e;
+                }
+                if (mine != 0x7fffffff) atomicMin(&sh.tok, mine);
+                if (mylast >= 0) atomicMax(&sh.last, mylast);
+                __syncthreads();
+                token = sh.tok != 0x7fffffff ? sh.tok : sh.last;
+                if (!PRECISE && use_resid && Q > 0.0) {
+                    // with q~ present the thresholds depend on the normaliser: error <= GUARD_Z * Q
+                    const double E2 = 2.0 * GUARD_Z * Q;
+                    if (sh.tok == 0x7fffffff) {
+                        if (tid == 0) sh.flag = 1;
+                    } else if (mine == sh.tok) {
+                        const int e = mine - (v0 + tid * 4);
+                        const double hi = base + cum[e] - thr2;
+                        const double lo = thr2 - (base + cum[e] - r[e]);
+                        if (hi < E2 || lo < E2) sh.flag = 1;
+                    }
+                }
+                __syncthreads();
+            }
+            flagged |= sh.flag != 0;
+        }
+
+        // ---- 5. outputs --------------------------------------------------------------------
+        if (tid == 0) {
+            if (st_bits) {
+                atomicOr(a.status, st_bits);
+                if (!a.sample_only) {
+                    a.accept_len[b] = -1;
+                    for (int i = 0; i < G; ++i) {
+                        a.p_draft[b * G + i] = -1.f;
+                        a.resid_mass[b * G + i] = -1.f;
+                    }
+                }
+                if (want_token) a.token[b] = -1;
+                if (a.mass) a.mass[b] = -1.f;
+            } else {
+                if (!a.sample_only) a.accept_len[b] = alen;
+                if (want_token) a.token[b] = token;
+                if (a.mass) a.mass[b] = (float)Rtot;
+                if (PRECISE) {
+                    if (nborder && a.borderline) atomicAdd(a.borderline, nborder);
+                } else if (flagged) {
+                    const int q = atomicAdd(a.queue_count, 1);
+                    a.queue[q] = b;
+                    atomicAdd(a.slow_rows, (unsigned long long)(a.sample_only ? 1 : G1));
+                }
+            }
+        }
+    }
+}
+
+}  // namespace picospec

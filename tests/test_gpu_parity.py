@@ -1,0 +1,365 @@
+"""GPU parity: the CUDA path, called through the C-ABI, against the CPU oracle on the same
+seeded input bits.  Integer outputs (support indices, counts, draft tokens, accept lengths,
+emitted tokens, borderline count) must be bit-exact; probabilities and residual masses must
+agree to 1e-5 relative."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+
+pytestmark = pytest.mark.gpu
+
+RTOL = 1e-5          # stated tolerance on q_prob, p_draft, resid_mass
+ATOL_MASS = 3e-7     # residual masses below ~1e-2 cancel against the fp32-accumulated normaliser
+
+
+@pytest.fixture(scope="module")
+def ps():
+    import paper_2603_19133_b200 as ps
+    ps.lib()
+    return ps
+
+
+_ctx_cache = {}
+
+
+def _ctx(ps, B, G, V, K):
+    key = (max(B, 1), G, V, K)
+    if key not in _ctx_cache:
+        _ctx_cache.clear()
+        _ctx_cache[key] = ps.Context(max(B, 1), G, V, K)
+    return _ctx_cache[key]
+
+
+def _np(t):
+    return t.detach().float().cpu().numpy() if t.is_floating_point() else t.detach().cpu().numpy()
+
+
+def _cuda(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    return t if dtype is None else t.to(dtype)
+
+
+def run_both(ps, w, inputs, check_compress=True, nthreads=None, draft_tok_override=None, seq_subset=None):
+    """Run compress -> verify (+ fused sample) on both sides and compare.  The sparse rows and
+    draft tokens fed to BOTH verifies are the oracle's."""
+    nthreads = nthreads or oracle.cores()
+    B, G, V, K = w.B, w.G, w.V, w.k_max
+    ctx = _ctx(ps, B, G, V, K)
+    dl, tl, T = inputs["draft_logits"], inputs["target_logits"], inputs["temperature"]
+    sub = slice(None) if seq_subset is None else seq_subset
+    # ---- oracle (on the sampled sequences) -------------------------------------------------
+    o_qi, o_qp, o_qc, o_tok = oracle.compress(_np(dl[sub]), _np(T[sub]), w.top_k, w.top_p, K,
+                                              _np(inputs["u_draft"][sub]), nthreads=nthreads)
+    if draft_tok_override is not None:
+        o_tok = draft_tok_override
+    o = oracle.verify(_np(tl[sub]), _np(T[sub]), o_tok, o_qi, o_qp, o_qc, _np(inputs["u_accept"][sub]),
+                      _np(inputs["u_resample"][sub]), nthreads=nthreads)
+    # ---- GPU ------------------------------------------------------------------------------------
+    if check_compress:
+        g_qi, g_qp, g_qc, g_tok = ctx.compress(dl, T, w.top_k, w.top_p, K, inputs["u_draft"])
+        torch.cuda.synchronize()
+        assert np.array_equal(_np(g_qc[sub]), o_qc), "q_count"
+        assert np.array_equal(_np(g_qi[sub]), o_qi), "q_idx"
+        if draft_tok_override is None:
+            assert np.array_equal(_np(g_tok[sub]), o_tok), "draft_tok"
+        np.testing.assert_allclose(_np(g_qp[sub]), o_qp, rtol=RTOL, atol=0)
+    if seq_subset is None:
+        qi, qp, qc, tok = _cuda(o_qi), _cuda(o_qp), _cuda(o_qc), _cuda(o_tok)
+    else:
+        # full-size GPU call: the sampled sequences carry the oracle's sparse rows, the others the GPU's
+        qi, qp, qc, tok = g_qi.clone(), g_qp.clone(), g_qc.clone(), g_tok.clone()
+        qi[sub], qp[sub], qc[sub], tok[sub] = _cuda(o_qi), _cuda(o_qp), _cuda(o_qc), _cuda(o_tok)
+    g = ctx.verify(tl, T, tok, qi, qp, qc, inputs["u_accept"], inputs["u_resample"])
+    st, slow = ctx.status(clear=True)
+    assert np.array_equal(_np(g["accept_len"][sub]), o["accept_len"]), "accept_len"
+    assert np.array_equal(_np(g["token"][sub]), o["token"]), "token"
+    if seq_subset is None:
+        assert int(g["borderline_count"].item()) == o["borderline_count"], "borderline_count"
+    ok = o["accept_len"] >= 0
+    np.testing.assert_allclose(_np(g["p_draft"][sub])[ok], o["p_draft"][ok], rtol=RTOL, atol=0)
+    np.testing.assert_allclose(_np(g["resid_mass"][sub])[ok], o["resid_mass"][ok], rtol=RTOL, atol=ATOL_MASS)
+    bad = ~ok
+    if bad.any():
+        assert np.all(_np(g["p_draft"][sub])[bad] == -1) and np.all(_np(g["resid_mass"][sub])[bad] == -1)
+    return {"status": st, "slow_rows": slow, "oracle": o, "gpu": g}
+
+
+# ---------------------------------------------------------------------------------------------
+# the benchmark configurations
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("name", ["config1", "config2", "config3"])
+def test_config_full_size(ps, name):
+    w = gen.WORKLOADS[name]
+    inputs = gen.make_inputs(w, seed=1000 * int(name[-1]), device="cuda")
+    r = run_both(ps, w, inputs)
+    assert r["status"] == 0
+
+
+def test_config4_full_size_launch_sampled_sequences(ps):
+    # the configuration the benchmark times, in its launch shape; the oracle checks a sample of
+    # sequences one by one (sequences are independent)
+    w = gen.WORKLOADS["config4"]
+    inputs = gen.make_inputs(w, seed=4000, device="cuda")
+    sub = np.arange(0, w.B, 8)
+    r = run_both(ps, w, inputs, seq_subset=sub)
+    assert r["status"] == 0
+
+
+@pytest.mark.parametrize("V,k", [(32000, 8), (128256, 64), (151936, 512), (262144, 1024), (32000, 1024)])
+def test_config5_sweep_points_reduced_batch(ps, V, k):
+    w = gen.sweep_workload(V, k, B=24)
+    inputs = gen.make_inputs(w, seed=5000 + k, device="cuda")
+    r = run_both(ps, w, inputs)
+    assert r["status"] == 0
+
+
+def test_config5_full_batch_sampled(ps):
+    w = gen.sweep_workload(128256, 64, B=512)
+    inputs = gen.make_inputs(w, seed=5512, device="cuda")
+    r = run_both(ps, w, inputs, seq_subset=np.arange(3, 512, 32))
+    assert r["status"] == 0
+
+
+# ---------------------------------------------------------------------------------------------
+# shapes: ragged tails, unaligned rows, padded pitch, K >= V
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("V,B,G,K,dtype,top_k,top_p", [
+    (1000, 3, 2, 16, "bf16", 16, 1.0),      # less than one chunk
+    (1001, 3, 2, 16, "bf16", 0, 0.9),       # odd V: rows not 16-byte aligned -> element-wise loads
+    (4097, 2, 3, 40, "f32", 40, 1.0),       # one entry into the fifth chunk
+    (4099, 2, 3, 40, "f32", 0, 0.8),        # unaligned fp32 rows
+    (9000, 5, 1, 1024, "bf16", 0, 0.999),   # wide sparse rows
+    (300, 2, 2, 512, "f32", 0, 1.0),        # K >= V: dense q~
+    (20000, 4, 4, 64, "bf16", 50, 0.7),     # top-k and top-p together
+    (8192, 2, 0, 8, "bf16", 8, 1.0),        # gamma = 0: bonus row only
+])
+def test_small_shapes(ps, V, B, G, K, dtype, top_k, top_p):
+    w = gen.Workload("t", V=V, B=B, G=G, dtype=dtype, s=1.1, sigma_d=1.5, corr=0.8, sigma_t=1.0,
+                     T=None, top_k=top_k, top_p=top_p, k_max=K)
+    inputs = gen.make_inputs(w, seed=V + K, device="cuda")
+    if G == 0:
+        ctx = _ctx(ps, B, G, V, K)
+        e = torch.empty
+        g = ctx.verify(inputs["target_logits"], inputs["temperature"], e((B, 0), dtype=torch.int32, device="cuda"),
+                       e((B, 0, K), dtype=torch.int32, device="cuda"), e((B, 0, K), dtype=torch.float32, device="cuda"),
+                       e((B, 0), dtype=torch.int32, device="cuda"), e((B, 0), dtype=torch.float32, device="cuda"),
+                       inputs["u_resample"])
+        o = oracle.verify(_np(inputs["target_logits"]), _np(inputs["temperature"]), np.zeros((B, 0), np.int32),
+                          np.zeros((B, 0, K), np.int32), np.zeros((B, 0, K), np.float32), np.zeros((B, 0), np.int32),
+                          np.zeros((B, 0), np.float32), _np(inputs["u_resample"]))
+        assert np.array_equal(_np(g["accept_len"]), o["accept_len"])
+        assert np.array_equal(_np(g["token"]), o["token"])
+        return
+    r = run_both(ps, w, inputs)
+    assert r["status"] == 0
+
+
+def test_padded_pitch_and_offset_base(ps):
+    # rows pitched wider than V, and a base pointer that is only 2-byte aligned
+    V, B, G, K = 5000, 3, 2, 32
+    w = gen.Workload("t", V=V, B=B, G=G, dtype="bf16", s=1.1, sigma_d=1.5, corr=0.8, sigma_t=1.0,
+                     T=0.9, top_k=K, top_p=1.0, k_max=K)
+    inp = gen.make_inputs(w, seed=77, device="cuda")
+    for pitch, offset in ((V + 24, 0), (V + 3, 0), (V, 1)):
+        def repitch(t):
+            Bq, R, _ = t.shape
+            flat = torch.full((Bq * R * pitch + 8,), float("nan"), dtype=t.dtype, device="cuda")
+            view = flat[offset:offset + Bq * R * pitch].view(Bq, R, pitch)[:, :, :V]
+            view.copy_(t)
+            return view
+        inputs = dict(inp)
+        inputs["draft_logits"] = repitch(inp["draft_logits"])
+        inputs["target_logits"] = repitch(inp["target_logits"])
+        ctx = _ctx(ps, B, G, V, K)
+        o_qi, o_qp, o_qc, o_tok = oracle.compress(_np(inp["draft_logits"]), _np(inp["temperature"]), K, 1.0, K,
+                                                  _np(inp["u_draft"]))
+        g_qi, g_qp, g_qc, g_tok = ctx.compress(inputs["draft_logits"], inp["temperature"], K, 1.0, K, inp["u_draft"])
+        assert np.array_equal(_np(g_qi), o_qi) and np.array_equal(_np(g_tok), o_tok)
+        o = oracle.verify(_np(inp["target_logits"]), _np(inp["temperature"]), o_tok, o_qi, o_qp, o_qc,
+                          _np(inp["u_accept"]), _np(inp["u_resample"]))
+        g = ctx.verify(inputs["target_logits"], inp["temperature"], g_tok, g_qi, g_qp, g_qc, inp["u_accept"],
+                       inp["u_resample"])
+        assert np.array_equal(_np(g["accept_len"]), o["accept_len"])
+        assert np.array_equal(_np(g["token"]), o["token"])
+        np.testing.assert_allclose(_np(g["p_draft"]), o["p_draft"], rtol=RTOL)
+        assert ctx.status(clear=True)[0] == 0
+
+
+# ---------------------------------------------------------------------------------------------
+# degenerate inputs
+# ---------------------------------------------------------------------------------------------
+
+def test_all_equal_logits_and_ties(ps):
+    V, B, G, K = 3000, 2, 2, 8
+    dl = torch.full((B, G, V), 1.5, dtype=torch.bfloat16, device="cuda")
+    dl[1] = torch.randint(-3, 4, (G, V), device="cuda").to(torch.bfloat16)     # heavy ties
+    tl = torch.zeros((B, G + 1, V), dtype=torch.bfloat16, device="cuda")
+    tl[1] = torch.randint(-2, 3, (G + 1, V), device="cuda").to(torch.bfloat16)
+    w = gen.Workload("t", V=V, B=B, G=G, dtype="bf16", s=0, sigma_d=0, corr=0, sigma_t=0, T=1.0,
+                     top_k=K, top_p=1.0, k_max=K)
+    g = torch.Generator(device="cuda").manual_seed(5)
+    inputs = {"draft_logits": dl, "target_logits": tl, "temperature": torch.ones(B, device="cuda"),
+              "u_draft": torch.rand((B, G), generator=g, device="cuda"),
+              "u_accept": torch.rand((B, G), generator=g, device="cuda"),
+              "u_resample": torch.rand((B, 2), generator=g, device="cuda")}
+    r = run_both(ps, w, inputs)
+    assert r["status"] == 0
+
+
+def test_minus_inf_logits(ps):
+    V, B, G, K = 2500, 2, 1, 4
+    dl = torch.full((B, G, V), float("-inf"), dtype=torch.float32, device="cuda")
+    dl[:, :, [5, 1200, 2400]] = torch.tensor([0.5, 1.0, -0.5], device="cuda")
+    tl = torch.full((B, G + 1, V), float("-inf"), dtype=torch.float32, device="cuda")
+    tl[:, :, [5, 700, 2400]] = torch.tensor([0.2, 0.1, 1.0], device="cuda")
+    w = gen.Workload("t", V=V, B=B, G=G, dtype="f32", s=0, sigma_d=0, corr=0, sigma_t=0, T=1.0,
+                     top_k=K, top_p=1.0, k_max=K)
+    inputs = {"draft_logits": dl, "target_logits": tl, "temperature": torch.ones(B, device="cuda"),
+              "u_draft": torch.tensor([[0.1], [0.9]], device="cuda"),
+              "u_accept": torch.tensor([[0.99], [0.5]], device="cuda"),
+              "u_resample": torch.tensor([[0.3, 0.6], [0.8, 0.2]], device="cuda")}
+    r = run_both(ps, w, inputs)
+    assert r["status"] == 0
+
+
+def test_q_equal_p_accepts_everything(ps):
+    # draft == target and K = V: q~ = p up to fp32 storage, every draft accepted, residual ~ 0,
+    # the bonus row is sampled
+    V, B, G = 700, 4, 3
+    w = gen.Workload("t", V=V, B=B, G=G, dtype="f32", s=1.0, sigma_d=1.0, corr=1.0, sigma_t=0.0, T=0.9,
+                     top_k=0, top_p=1.0, k_max=1024)
+    inputs = gen.make_inputs(w, seed=3, device="cuda")
+    inputs["u_accept"] = inputs["u_accept"] * 0.99
+    r = run_both(ps, w, inputs)
+    assert np.all(_np(r["gpu"]["accept_len"]) == G)
+    assert np.all(np.abs(_np(r["gpu"]["resid_mass"])) < 1e-6)
+
+
+def test_draft_token_outside_support_is_accepted(ps):
+    V, B, G, K = 4000, 3, 2, 4
+    w = gen.Workload("t", V=V, B=B, G=G, dtype="bf16", s=1.1, sigma_d=1.5, corr=0.8, sigma_t=1.0, T=1.0,
+                     top_k=K, top_p=1.0, k_max=K)
+    inputs = gen.make_inputs(w, seed=9, device="cuda")
+    qi, _, _, _ = oracle.compress(_np(inputs["draft_logits"]), _np(inputs["temperature"]), K, 1.0, K)
+    tok = np.zeros((B, G), np.int32)
+    for b in range(B):
+        for i in range(G):
+            tok[b, i] = next(v for v in range(V) if v not in qi[b, i])
+    r = run_both(ps, w, inputs, check_compress=False, draft_tok_override=tok)
+    assert np.all(_np(r["gpu"]["accept_len"]) == G)
+
+
+def test_bad_data_sets_status_and_marks_outputs(ps):
+    V, B, G, K = 3000, 5, 2, 8
+    w = gen.Workload("t", V=V, B=B, G=G, dtype="bf16", s=1.1, sigma_d=1.5, corr=0.8, sigma_t=1.0, T=1.0,
+                     top_k=K, top_p=0.9, k_max=K)
+    inputs = gen.make_inputs(w, seed=21, device="cuda")
+    inputs["draft_logits"][1, 0, 17] = float("nan")
+    inputs["target_logits"][2, 1, 2999] = float("inf")
+    inputs["temperature"][3] = 0.0
+    inputs["target_logits"][4, 2, 1500] = float("nan")
+    ctx = _ctx(ps, B, G, V, K)
+    o_qi, o_qp, o_qc, o_tok = oracle.compress(_np(inputs["draft_logits"]), _np(inputs["temperature"]), K, 0.9, K,
+                                              _np(inputs["u_draft"]))
+    g_qi, g_qp, g_qc, g_tok = ctx.compress(inputs["draft_logits"], inputs["temperature"], K, 0.9, K, inputs["u_draft"])
+    st, _ = ctx.status(clear=True)
+    assert st & 2 and st & 1
+    assert np.array_equal(_np(g_qc), o_qc) and np.array_equal(_np(g_qi), o_qi) and np.array_equal(_np(g_tok), o_tok)
+    assert _np(g_qc)[1, 0] == -1 and np.all(_np(g_qc)[3] == -1)
+    tok = np.where(o_tok < 0, 0, o_tok).astype(np.int32)
+    o = oracle.verify(_np(inputs["target_logits"]), _np(inputs["temperature"]), tok, o_qi, o_qp, o_qc,
+                      _np(inputs["u_accept"]), _np(inputs["u_resample"]))
+    g = ctx.verify(inputs["target_logits"], inputs["temperature"], _cuda(tok), g_qi, g_qp, g_qc, inputs["u_accept"],
+                   inputs["u_resample"])
+    st, _ = ctx.status(clear=True)
+    assert st & 1 and st & 2 and st & 4          # temperature, logit, count out of range (-1)
+    assert np.array_equal(_np(g["accept_len"]), o["accept_len"])
+    assert np.array_equal(_np(g["token"]), o["token"])
+    assert list(o["accept_len"][1:]) == [-1, -1, -1, -1] and o["accept_len"][0] >= 0
+    # out-of-range token
+    tok2 = tok.copy()
+    tok2[0, 1] = V
+    g = ctx.verify(inputs["target_logits"], inputs["temperature"], _cuda(tok2), g_qi, g_qp, g_qc, inputs["u_accept"],
+                   inputs["u_resample"])
+    st, _ = ctx.status(clear=True)
+    assert st & 4 and _np(g["accept_len"])[0] == -1 and _np(g["token"])[0] == -1
+
+
+def test_host_side_argument_errors(ps):
+    ctx = ps.Context(4, 2, 1000, 8)
+    l = torch.zeros((2, 2, 1000), dtype=torch.bfloat16, device="cuda")
+    T = torch.ones(2, device="cuda")
+    with pytest.raises(ps.PicospecError) as e:
+        ctx.compress(l, T, 4, 0.0, 8)                       # top_p <= 0
+    assert e.value.code == -1
+    with pytest.raises(ps.PicospecError) as e:
+        ctx.compress(l, T, 4, 1.0, 16)                      # k_max beyond capacity
+    assert e.value.code == -3
+    big = torch.zeros((5, 2, 1000), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(ps.PicospecError) as e:
+        ctx.compress(big, torch.ones(5, device="cuda"), 4, 1.0, 8)
+    assert e.value.code == -3
+    with pytest.raises(ValueError):
+        ctx.compress(l.cpu(), T, 4, 1.0, 8)                 # no CPU path
+    ctx.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# stand-alone residual sampling
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("name,B", [("config2", 8), ("config3", 24)])
+def test_residual_sample_standalone(ps, name, B):
+    w = gen.scaled(gen.WORKLOADS[name], B=B)
+    inputs = gen.make_inputs(w, seed=808, device="cuda")
+    ctx = _ctx(ps, w.B, w.G, w.V, w.k_max)
+    o_qi, o_qp, o_qc, _ = oracle.compress(_np(inputs["draft_logits"]), _np(inputs["temperature"]), w.top_k, w.top_p,
+                                          w.k_max, nthreads=oracle.cores())
+    rng = np.random.default_rng(1)
+    pos = rng.integers(0, w.G + 1, size=B).astype(np.int32)
+    pos[0], pos[-1] = 0, w.G
+    o_tok, o_mass = oracle.residual_sample(_np(inputs["target_logits"]), _np(inputs["temperature"]), pos, o_qi, o_qp,
+                                           o_qc, _np(inputs["u_resample"]), nthreads=oracle.cores())
+    g_tok, g_mass = ctx.residual_sample(inputs["target_logits"], inputs["temperature"], _cuda(pos), _cuda(o_qi),
+                                        _cuda(o_qp), _cuda(o_qc), inputs["u_resample"])
+    st, _ = ctx.status(clear=True)
+    assert st == 0
+    assert np.array_equal(_np(g_tok), o_tok)
+    np.testing.assert_allclose(_np(g_mass), o_mass, rtol=RTOL, atol=ATOL_MASS)
+    # an out-of-range position is reported, not sampled
+    pos[1] = w.G + 1
+    g_tok, g_mass = ctx.residual_sample(inputs["target_logits"], inputs["temperature"], _cuda(pos), _cuda(o_qi),
+                                        _cuda(o_qp), _cuda(o_qc), inputs["u_resample"])
+    st, _ = ctx.status(clear=True)
+    assert st & 4 and _np(g_tok)[1] == -1
+    assert np.array_equal(np.delete(_np(g_tok), 1), np.delete(o_tok, 1))
+
+
+# ---------------------------------------------------------------------------------------------
+# the double-precision path really decides near-threshold cases the way the oracle does
+# ---------------------------------------------------------------------------------------------
+
+def test_near_threshold_uniforms_are_decided_exactly(ps):
+    # place every accept uniform within a few fp32 ulps of the oracle's ratio p(x)/q~(x): all of
+    # them must go through the double-precision pass and still match, borderline count included
+    w = gen.scaled(gen.WORKLOADS["config2"], B=16)
+    inputs = gen.make_inputs(w, seed=99, device="cuda")
+    dl, tl, T = _np(inputs["draft_logits"]), _np(inputs["target_logits"]), _np(inputs["temperature"])
+    qi, qp, qc, tok = oracle.compress(dl, T, w.top_k, w.top_p, w.k_max, _np(inputs["u_draft"]), nthreads=oracle.cores())
+    o0 = oracle.verify(tl, T, tok, qi, qp, qc, _np(inputs["u_accept"]), nthreads=oracle.cores())
+    qx = np.zeros((w.B, w.G))
+    for b in range(w.B):
+        for i in range(w.G):
+            qx[b, i] = qp[b, i][list(qi[b, i]).index(tok[b, i])]
+    ratio = np.minimum(o0["p_draft"] / qx, 0.999)
+    rng = np.random.default_rng(4)
+    u = (ratio * (1 + rng.integers(-3, 4, size=ratio.shape) * 6e-8)).astype(np.float32)
+    inputs["u_accept"] = _cuda(u)
+    r = run_both(ps, w, inputs, check_compress=False)
+    assert r["slow_rows"] > 0
+    assert r["oracle"]["borderline_count"] > 0

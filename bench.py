@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the separate-rejection-sampling hot path on B200.
+
+One "step" is one pass of the whole path over one batch of synthetic input: draft-side sparse
+compression (picospec_compress, with the draft-token draw) followed by target-side verification
+with the fused residual / bonus sample (picospec_verify).  The headline metric is verified
+draft positions per second (B * gamma per step); the roofline entry is the achieved HBM
+bandwidth of the verify streaming kernel.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config4] [--impl ours|reference]
+
+N > 1 is launched under torchrun, one rank per GPU; every rank runs its own batch (the path
+shards by sequence, no collective on the data path), so scaling is weak.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import gen  # noqa: E402
+
+METRIC = "verified_draft_positions_per_sec"
+UNIT = "positions/s"
+
+# DRAM traffic of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum per launch)
+# from the ncu captures summarised under profiles/; None until a capture exists for the workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.idx = device_index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+
+        def pump():
+            for line in self.proc.stdout:
+                self.rows.append(line.strip())
+
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                 f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def _np(t):
+    return t.detach().float().cpu().numpy() if t.is_floating_point() else t.detach().cpu().numpy()
+
+
+# -------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on the host cores
+# -------------------------------------------------------------------------------------------------
+
+def oracle_step_time(w, inputs_cpu, nthreads):
+    """One pass of the whole path (compress + verify with fused sample) by the oracle; seconds."""
+    import oracle
+    t0 = time.perf_counter()
+    qi, qp, qc, tok = oracle.compress(inputs_cpu["draft_logits"], inputs_cpu["temperature"], w.top_k, w.top_p,
+                                      w.k_max, inputs_cpu["u_draft"], nthreads=nthreads)
+    oracle.verify(inputs_cpu["target_logits"], inputs_cpu["temperature"], tok, qi, qp, qc, inputs_cpu["u_accept"],
+                  inputs_cpu["u_resample"], nthreads=nthreads)
+    return time.perf_counter() - t0
+
+
+def oracle_sample(w, seed, sample_B):
+    ws = gen.scaled(w, B=sample_B)
+    inp = gen.make_inputs(ws, seed=seed, device="cpu")
+    return ws, {k: _np(v) for k, v in inp.items()}
+
+
+def run_reference(args):
+    rank, _, world = _dist_env()
+    if rank != 0:
+        return
+    import oracle
+    w = gen.WORKLOADS[args.workload]
+    cores = oracle.cores()
+    sample_B = min(w.B, args.ref_sample)
+    ws, inp = oracle_sample(w, 4242, sample_B)
+    for _ in range(min(args.warmup, 1)):
+        oracle_step_time(ws, inp, cores)
+    times = [oracle_step_time(ws, inp, cores) for _ in range(args.steps)]
+    t = sum(times)
+    value = ws.B * ws.G * args.steps / t
+    sample = f"{sample_B} of {w.B} sequences of {w.name} per step, all {cores} host threads (OpenMP over rows)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "V": w.V, "B": ws.B, "gamma": w.G, "logits": w.dtype, "k_max": w.k_max},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# -------------------------------------------------------------------------------------------------
+# our arm
+# -------------------------------------------------------------------------------------------------
+
+class Step:
+    """Pre-allocated outputs and the two calls of one step on device-resident inputs."""
+
+    def __init__(self, ps, ctx, w, inputs):
+        self.ctx, self.w, self.inp = ctx, w, inputs
+        dev = inputs["draft_logits"].device
+        B, G, K = w.B, w.G, w.k_max
+        i32, f32 = torch.int32, torch.float32
+        self.c_out = (torch.empty((B, G, K), dtype=i32, device=dev), torch.empty((B, G, K), dtype=f32, device=dev),
+                      torch.empty((B, G), dtype=i32, device=dev), torch.empty((B, G), dtype=i32, device=dev))
+        self.v_out = {"accept_len": torch.empty((B,), dtype=i32, device=dev),
+                      "p_draft": torch.empty((B, G), dtype=f32, device=dev),
+                      "resid_mass": torch.empty((B, G), dtype=f32, device=dev),
+                      "borderline_count": torch.empty((1,), dtype=i32, device=dev),
+                      "token": torch.empty((B,), dtype=i32, device=dev)}
+        self.launches_per_step = (3 if w.top_p < 1.0 else 1) + 4
+
+    def compress(self, inp=None):
+        inp = inp or self.inp
+        w = self.w
+        return self.ctx.compress(inp["draft_logits"], inp["temperature"], w.top_k, w.top_p, w.k_max, inp["u_draft"],
+                                 out=self.c_out)
+
+    def verify(self, inp=None):
+        inp = inp or self.inp
+        qi, qp, qc, tok = self.c_out
+        return self.ctx.verify(inp["target_logits"], inp["temperature"], tok, qi, qp, qc, inp["u_accept"],
+                               inp["u_resample"], out=self.v_out)
+
+    def __call__(self, inp=None):
+        self.compress(inp)
+        self.verify(inp)
+
+
+def timed_loop(fn, steps, warmup, sync):
+    for _ in range(warmup):
+        fn()
+    sync()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    sync()
+    return e0.elapsed_time(e1) * 1e-3
+
+
+def algorithmic_bytes(w):
+    """Bytes the method itself has to move per launch of each streaming kernel."""
+    nch = (w.V + 1023) // 1024
+    rows_t, rows_d = w.B * (w.G + 1), w.B * w.G
+    verify_stream = rows_t * w.V * w.bytes_per_logit + rows_t * nch * 8
+    compress_stream = rows_d * w.V * w.bytes_per_logit + rows_d * (w.k_max * 8 + 8)
+    return verify_stream, compress_stream
+
+
+def bench_workload(ps, w, args, rank, world, device, with_e2e, with_clocks):
+    ctx = ps.Context(w.B, w.G, w.V, w.k_max)
+    # rotate through enough distinct input sets that consecutive steps never find their logits in L2
+    per_set = (w.B * (2 * w.G + 1)) * w.V * w.bytes_per_logit
+    nsets = max(1, min(12, -(-(512 << 20) // per_set))) if per_set < (512 << 20) else 1
+    sets = [gen.make_inputs(w, seed=1000 * (rank + 1) + 17 * i + sum(map(ord, w.name)), device=device)
+            for i in range(nsets)]
+    step = Step(ps, ctx, w, sets[0])
+    state = {"i": 0}
+
+    def one():
+        step(sets[state["i"] % nsets])
+        state["i"] += 1
+
+    def sync():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+            torch.cuda.synchronize()
+
+    ctx.status(clear=True)
+    ctx.profile_enable(1)
+    sampler = ClockSampler(torch.cuda.current_device()) if with_clocks else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.15)
+    t = timed_loop(one, args.steps, args.warmup, sync)
+    clocks = sampler.stop() if sampler else None
+    ms_vs, n_vs = ctx.profile_read(1)
+    ms_cs, n_cs = ctx.profile_read(0)
+    ctx.profile_enable(0)
+    st, slow = ctx.status(clear=True)
+    if world > 1:
+        tt = torch.tensor([t], device=device, dtype=torch.float64)
+        torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
+        t = float(tt.item())
+    # the same loop without the event brackets, for the record
+    t_plain = timed_loop(one, args.steps, min(args.warmup, 3), sync)
+
+    vbytes, cbytes = algorithmic_bytes(w)
+    peak, peak_kind = _peaks()
+    vs_time = ms_vs / max(n_vs, 1) * 1e-3
+    cs_time = ms_cs / max(n_cs, 1) * 1e-3
+    res = {
+        "seconds": t, "seconds_unbracketed": t_plain, "status": st,
+        "slow_rows_per_step": slow / float(args.steps + args.warmup),
+        "value": world * w.B * w.G * args.steps / t,
+        "rows_streamed_per_sec": world * w.B * (2 * w.G + 1) * args.steps / t,
+        "verify_stream": {"avg_us": vs_time * 1e6, "launches": n_vs, "alg_bytes": vbytes,
+                          "GBps": vbytes / vs_time / 1e9 if vs_time > 0 else None},
+        "compress_stream": {"avg_us": cs_time * 1e6, "launches": n_cs, "alg_bytes": cbytes,
+                            "GBps": cbytes / cs_time / 1e9 if cs_time > 0 else None},
+        "peak": peak, "peak_kind": peak_kind, "clocks": clocks, "nsets": nsets,
+        "launches_per_step": step.launches_per_step,
+    }
+
+    if with_e2e:
+        # end to end: host-resident inputs (pinned), copied in every step; results read back
+        host = {k: v.cpu().pin_memory() for k, v in sets[0].items()}
+        dev = {k: torch.empty_like(v) for k, v in sets[0].items()}
+        h_out = {k: torch.empty_like(v, device="cpu").pin_memory() for k, v in step.v_out.items()}
+        h2d = sum(v.numel() * v.element_size() for v in host.values())
+        d2h = sum(v.numel() * v.element_size() for v in h_out.values())
+
+        def one_e2e():
+            for k in host:
+                dev[k].copy_(host[k], non_blocking=True)
+            step(dev)
+            for k in h_out:
+                h_out[k].copy_(step.v_out[k], non_blocking=True)
+            torch.cuda.current_stream().synchronize()      # the caller reads the result
+
+        k_e2e = max(2, min(args.steps, 10))
+        t0 = time.perf_counter()
+        te = timed_loop(one_e2e, k_e2e, 1, sync)
+        if world > 1:
+            tt = torch.tensor([te], device=device, dtype=torch.float64)
+            torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
+            te = float(tt.item())
+        res["e2e"] = {"value": world * w.B * w.G * k_e2e / te, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                      "d2h_bytes_per_step": d2h, "steps": k_e2e, "wall_s": time.perf_counter() - t0}
+        del host, dev, h_out
+    ctx.close()
+    del sets, step
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_ours(args):
+    rank, local_rank, world = _dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=device)
+    import paper_2603_19133_b200 as ps
+    ps.lib()
+    w = gen.WORKLOADS[args.workload]
+    if args.batch > 0:
+        w = gen.scaled(w, B=args.batch)
+    main = bench_workload(ps, w, args, rank, world, device, with_e2e=True, with_clocks=(rank == 0))
+
+    others = {}
+    if args.all_configs and world == 1:
+        for name in ("config1", "config2", "config3"):
+            if name == args.workload:
+                continue
+            r = bench_workload(ps, gen.WORKLOADS[name], args, rank, world, device, with_e2e=False, with_clocks=False)
+            others[name] = {"positions_per_sec": r["value"], "ms_per_step": 1e3 * r["seconds"] / args.steps,
+                            "verify_stream_us": r["verify_stream"]["avg_us"],
+                            "verify_stream_GBps": r["verify_stream"]["GBps"],
+                            "verify_stream_frac_of_peak": (r["verify_stream"]["GBps"] or 0) / r["peak"],
+                            "compress_stream_us": r["compress_stream"]["avg_us"],
+                            "compress_stream_GBps": r["compress_stream"]["GBps"],
+                            "input_sets_rotated": r["nsets"], "slow_rows_per_step": r["slow_rows_per_step"]}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        cores = oracle.cores()
+        sample_B = min(w.B, args.ref_sample)
+        ws, inp = oracle_sample(w, 4242, sample_B)
+        tcpu = oracle_step_time(ws, inp, cores)
+        cpu_baseline = {"value": ws.B * ws.G / tcpu, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"{sample_B} of {w.B} sequences of {w.name}, one pass, {tcpu:.2f} s, "
+                                  f"all {cores} host threads (OpenMP over rows)"}
+
+    if rank == 0:
+        vs = main["verify_stream"]
+        line = {
+            "metric": METRIC, "value": main["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * main["seconds"] / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "V": w.V, "B_per_gpu": w.B, "gamma": w.G, "logits": w.dtype,
+                       "top_k": w.top_k, "top_p": w.top_p, "k_max": w.k_max,
+                       "step": "picospec_compress + picospec_verify (fused residual/bonus sample)",
+                       "l2": f"inputs larger than L2: {main['nsets']} input set(s) of "
+                             f"{(w.B * (2 * w.G + 1)) * w.V * w.bytes_per_logit / 1e6:.0f} MB rotated",
+                       "parallelism": f"dp{world} (sequences sharded, no collective)"},
+            "roofline": {"bound": "hbm", "kernel": "chunk_stats_kernel (picospec_verify streaming pass)",
+                         "achieved": vs["GBps"], "peak": main["peak"], "unit": "GB/s",
+                         "frac": (vs["GBps"] or 0) / main["peak"], "peak_kind": f"of {main['peak_kind']}",
+                         "frac_of_8TBps_nominal": (vs["GBps"] or 0) / 8000.0,
+                         "avg_launch_us": vs["avg_us"], "launches_timed": vs["launches"],
+                         "algorithmic_bytes_per_launch": vs["alg_bytes"],
+                         "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+            "kernels": {"compress_stream": main["compress_stream"]},
+            "e2e": {k: main["e2e"][k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step")},
+            "gpu_launches": main["launches_per_step"] * args.steps,
+            "cpu_baseline": cpu_baseline,
+            "clocks": main["clocks"],
+            "ms_per_step_without_event_brackets": 1e3 * main["seconds_unbracketed"] / args.steps,
+            "rows_streamed_per_sec": main["rows_streamed_per_sec"],
+            "slow_path_rows_per_step": main["slow_rows_per_step"],
+            "device_status": main["status"],
+            "other_configs": others,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        torch.distributed.barrier()
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config4", choices=sorted(gen.WORKLOADS))
+    ap.add_argument("--ref-sample", type=int, default=64, help="sequences per step of the CPU oracle legs")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override B of the workload (profiling on a small case)")
+    ap.add_argument("--all-configs", action="store_true", default=True)
+    ap.add_argument("--only-main", dest="all_configs", action="store_false")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

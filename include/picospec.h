@@ -73,6 +73,24 @@ PICOSPEC_API const char* picospec_strerror(int err);
 /* cudaError_t of the last failing CUDA call made through this context (0 if none). */
 PICOSPEC_API int picospec_last_cuda_error(const picospec_ctx* ctx);
 
+/* Optional per-kernel timing, for benchmarks.  level 0 = off (default), 1 = bracket the two
+ * streaming kernels (one per hot call) with CUDA events on the caller's stream, 2 = bracket every
+ * kernel group.  Enabling creates the events (host objects; no device memory) and resets the
+ * counters; call it outside timed or captured regions.  The paper has no counterpart. */
+#define PICOSPEC_PROF_COMPRESS_STREAM 0  /* compress: streaming select kernel                    */
+#define PICOSPEC_PROF_VERIFY_STREAM 1    /* verify / residual_sample: streaming statistics kernel */
+#define PICOSPEC_PROF_VERIFY_FINISH 2    /* verify: per-sequence finish kernel                   */
+#define PICOSPEC_PROF_VERIFY_PRECISE 3   /* verify: double-precision re-evaluation kernels       */
+#define PICOSPEC_PROF_COMPRESS_PRECISE 4 /* compress: double-precision re-evaluation kernels     */
+#define PICOSPEC_PROF_KINDS 5
+PICOSPEC_API int picospec_profile_enable(picospec_ctx* ctx, int level);
+
+/* Synchronise `cuda_stream`, then return the summed device time (ms, HOST pointer) and the number
+ * of launches (HOST pointer) recorded for `kind` since the last read (at most the last 128
+ * launches are kept), and reset that counter. */
+PICOSPEC_API int picospec_profile_read(picospec_ctx* ctx, int kind, float* total_ms_out, int* launches_out,
+                                       void* cuda_stream);
+
 /* Synchronise `cuda_stream`, then copy the sticky status word and the cumulative number of rows
  * re-evaluated in double precision to HOST memory (either pointer may be NULL).  If `clear` is
  * non-zero both are reset afterwards.  Returns PICOSPEC_EDATA if the status word is non-zero. */

@@ -42,7 +42,9 @@ def lib() -> ctypes.CDLL:
                                       vp, vp, vp, vp, vp, vp, vp, vp]
         L.picospec_residual_sample.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp,
                                                c_int, vp, vp, vp, vp]
-        for f in ("picospec_create", "picospec_destroy", "picospec_last_cuda_error", "picospec_status",
+        L.picospec_profile_enable.argtypes = [vp, c_int]
+        L.picospec_profile_read.argtypes = [vp, c_int, ctypes.POINTER(c_f), ctypes.POINTER(c_int), vp]
+        for f in ("picospec_profile_enable", "picospec_profile_read", "picospec_create", "picospec_destroy", "picospec_last_cuda_error", "picospec_status",
                   "picospec_compress", "picospec_verify", "picospec_residual_sample"):
             getattr(L, f).restype = c_int
         _lib = L
@@ -126,6 +128,17 @@ class Context:
         if rc not in (OK, EDATA):
             raise PicospecError(rc, "picospec_status")
         return st.value, slow.value
+
+    def profile_enable(self, level: int):
+        """0 = off, 1 = time the two streaming kernels, 2 = time every kernel group."""
+        _check(lib().picospec_profile_enable(self._h, int(level)), "picospec_profile_enable")
+
+    def profile_read(self, kind: int) -> Tuple[float, int]:
+        """(summed device ms, launches) recorded for one kernel kind since the last read."""
+        ms, n = ctypes.c_float(0), ctypes.c_int(0)
+        _check(lib().picospec_profile_read(self._h, int(kind), ctypes.byref(ms), ctypes.byref(n), _stream()),
+               "picospec_profile_read")
+        return ms.value, n.value
 
     # -- half 1 -------------------------------------------------------------------------
     def compress(self, draft_logits: torch.Tensor, temperature: torch.Tensor, top_k: int, top_p: float,

@@ -10,12 +10,18 @@
 
 using namespace picospec;
 
+#define PROF_RING 128
+
 struct picospec_ctx {
     int device;
     int max_batch, max_gamma, max_vocab, max_k;
     int num_sms;
     int last_cuda_error;
     unsigned long long compress_calls;
+    // optional per-kernel timing (picospec_profile_*): rings of event pairs per kernel kind
+    int prof_level;
+    cudaEvent_t prof_ev[PICOSPEC_PROF_KINDS][PROF_RING][2];
+    long long prof_count[PICOSPEC_PROF_KINDS];
     // workspace
     float2* stats;
     double* dsum;
@@ -42,6 +48,24 @@ struct DeviceGuard {
     int target;
 };
 
+// Brackets one kernel launch with a pair of events when profiling is enabled for its kind.
+struct ProfScope {
+    picospec_ctx* ctx;
+    int kind;
+    cudaStream_t s;
+    bool on;
+    ProfScope(picospec_ctx* c, int k, int min_level, cudaStream_t st) : ctx(c), kind(k), s(st) {
+        on = c->prof_level >= min_level;
+        if (on) cudaEventRecord(c->prof_ev[k][c->prof_count[k] % PROF_RING][0], s);
+    }
+    ~ProfScope() {
+        if (on) {
+            cudaEventRecord(ctx->prof_ev[kind][ctx->prof_count[kind] % PROF_RING][1], s);
+            ctx->prof_count[kind]++;
+        }
+    }
+};
+
 int fail_cuda(picospec_ctx* ctx, cudaError_t e) {
     if (ctx) ctx->last_cuda_error = (int)e;
     return PICOSPEC_ECUDA;
@@ -63,15 +87,19 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
     const int rows = a.B * a.G;
     const int grid = rows < ctx->num_sms * 2 ? rows : ctx->num_sms * 2;
     const bool stats = a.top_p < 1.0f;
-    if (aligned) {
-        if (stats) compress_kernel<T, true, true><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
-        else compress_kernel<T, true, false><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
-    } else {
-        if (stats) compress_kernel<T, false, true><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
-        else compress_kernel<T, false, false><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+    {
+        ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_STREAM, 1, s);
+        if (aligned) {
+            if (stats) compress_kernel<T, true, true><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+            else compress_kernel<T, true, false><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+        } else {
+            if (stats) compress_kernel<T, false, true><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+            else compress_kernel<T, false, false><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+        }
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || !stats) return e;
+    ProfScope ps2(ctx, PICOSPEC_PROF_COMPRESS_PRECISE, 2, s);
     // rows whose top-p cut was too close to call: exact normaliser, then redo the cut
     PreciseArgs p;
     p.logits = a.logits; p.row_stride = a.row_stride; p.V = a.V; p.nch = a.nch;
@@ -89,12 +117,19 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
     long long want = (items + WARPS - 1) / WARPS;
     const int cap = ctx->num_sms * 4;
     const int grid = (int)(want < cap ? want : cap);
-    if (aligned) chunk_stats_kernel<T, true><<<grid, THREADS, 0, s>>>(a);
-    else chunk_stats_kernel<T, false><<<grid, THREADS, 0, s>>>(a);
+    {
+        ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_STREAM, 1, s);
+        if (aligned) chunk_stats_kernel<T, true><<<grid, THREADS, 0, s>>>(a);
+        else chunk_stats_kernel<T, false><<<grid, THREADS, 0, s>>>(a);
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const size_t dyn = (size_t)a.nch * sizeof(double);
-    verify_finish_kernel<T, false><<<a.B, THREADS, dyn, s>>>(a);
+    {
+        ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_FINISH, 2, s);
+        verify_finish_kernel<T, false><<<a.B, THREADS, dyn, s>>>(a);
+    }
+    ProfScope ps3(ctx, PICOSPEC_PROF_VERIFY_PRECISE, 2, s);
     PreciseArgs p;
     p.logits = a.logits; p.row_stride = a.row_stride; p.V = a.V; p.nch = a.nch;
     p.seq_rows = a.G + 1; p.expand = a.sample_only ? 1 : a.G + 1; p.pos = a.sample_only ? a.pos : nullptr;
@@ -164,6 +199,7 @@ int picospec_create(picospec_ctx** out, int device, int max_batch, int max_gamma
 int picospec_destroy(picospec_ctx* ctx) {
     if (!ctx) return PICOSPEC_EINVAL;
     DeviceGuard g(ctx->device);
+    picospec_profile_enable(ctx, 0);
     cudaFree(ctx->stats);
     cudaFree(ctx->dsum);
     cudaFree(ctx->row_max);
@@ -187,6 +223,50 @@ const char* picospec_strerror(int err) {
 }
 
 int picospec_last_cuda_error(const picospec_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+int picospec_profile_enable(picospec_ctx* ctx, int level) {
+    if (!ctx || level < 0 || level > 2) return PICOSPEC_EINVAL;
+    DeviceGuard g(ctx->device);
+    const bool have = ctx->prof_ev[0][0][0] != nullptr;
+    if (level > 0 && !have) {
+        for (int k = 0; k < PICOSPEC_PROF_KINDS; ++k)
+            for (int i = 0; i < PROF_RING; ++i)
+                for (int j = 0; j < 2; ++j) {
+                    cudaError_t e = cudaEventCreate(&ctx->prof_ev[k][i][j]);
+                    if (e != cudaSuccess) return fail_cuda(ctx, e);
+                }
+    }
+    if (level == 0 && have) {
+        for (int k = 0; k < PICOSPEC_PROF_KINDS; ++k)
+            for (int i = 0; i < PROF_RING; ++i)
+                for (int j = 0; j < 2; ++j) {
+                    cudaEventDestroy(ctx->prof_ev[k][i][j]);
+                    ctx->prof_ev[k][i][j] = nullptr;
+                }
+    }
+    for (int k = 0; k < PICOSPEC_PROF_KINDS; ++k) ctx->prof_count[k] = 0;
+    ctx->prof_level = level;
+    return PICOSPEC_OK;
+}
+
+int picospec_profile_read(picospec_ctx* ctx, int kind, float* total_ms_out, int* launches_out, void* cuda_stream) {
+    if (!ctx || kind < 0 || kind >= PICOSPEC_PROF_KINDS || !total_ms_out || !launches_out) return PICOSPEC_EINVAL;
+    DeviceGuard g(ctx->device);
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    const long long n = ctx->prof_count[kind] < PROF_RING ? ctx->prof_count[kind] : PROF_RING;
+    float total = 0.f;
+    for (long long i = 0; i < n; ++i) {
+        float ms = 0.f;
+        e = cudaEventElapsedTime(&ms, ctx->prof_ev[kind][i][0], ctx->prof_ev[kind][i][1]);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        total += ms;
+    }
+    *total_ms_out = total;
+    *launches_out = (int)n;
+    ctx->prof_count[kind] = 0;
+    return PICOSPEC_OK;
+}
 
 int picospec_status(picospec_ctx* ctx, int* device_status_out, long long* slow_path_rows_out, int clear,
                     void* cuda_stream) {

@@ -1,0 +1,141 @@
+"""CPU-side checks: the C-ABI library loads and exports what the header declares, the binding
+refuses to run without CUDA, the input generator is deterministic, and the sequence sharding
+used for more than one GPU reproduces the single-process result (gloo, world_size 2)."""
+import ctypes
+import os
+import re
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+import torch
+
+import gen
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "picospec.h")).read()
+    return sorted(set(re.findall(r"PICOSPEC_API\s+[\w\s\*]+?\b(picospec_\w+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2603_19133_b200 import buildlib
+    lib = ctypes.CDLL(buildlib.build())
+    names = _declared_symbols()
+    assert {"picospec_compress", "picospec_verify", "picospec_residual_sample", "picospec_create",
+            "picospec_destroy", "picospec_status", "picospec_strerror"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in picospec.h but not exported"
+    lib.picospec_strerror.restype = ctypes.c_char_p
+    assert lib.picospec_strerror(0) == b"ok"
+    assert b"capacity" in lib.picospec_strerror(-3)
+
+
+def test_only_the_c_abi_is_exported():
+    from paper_2603_19133_b200 import buildlib
+    out = subprocess.run(["nm", "-D", "--defined-only", buildlib.build()], capture_output=True, text=True).stdout
+    exported = [ln.split()[-1] for ln in out.splitlines() if " T " in ln]
+    assert sorted(exported) == _declared_symbols()
+
+
+def test_host_argument_checks_need_no_gpu():
+    from paper_2603_19133_b200 import buildlib
+    lib = ctypes.CDLL(buildlib.build())
+    h = ctypes.c_void_p()
+    assert lib.picospec_create(None, 0, 1, 1, 1000, 8) == -1
+    assert lib.picospec_create(ctypes.byref(h), 0, 0, 1, 1000, 8) == -1          # max_batch <= 0
+    assert lib.picospec_create(ctypes.byref(h), 0, 1, 1, 1000, 5000) == -1       # max_k too large
+    assert lib.picospec_destroy(None) == -1
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="checks the behaviour without a GPU")
+def test_no_cpu_fallback():
+    import paper_2603_19133_b200 as ps
+    with pytest.raises(RuntimeError):
+        ps.Context(1, 1, 1000, 8)
+
+
+def test_product_package_never_touches_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2603_19133_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower(), f"{f} mentions the oracle"
+
+
+def test_generator_is_deterministic_and_shaped():
+    w = gen.scaled(gen.WORKLOADS["config2"], B=2, V=5000)
+    a, b = gen.make_inputs(w, 5), gen.make_inputs(w, 5)
+    c = gen.make_inputs(w, 6)
+    for k in a:
+        assert torch.equal(a[k], b[k])
+    assert not torch.equal(a["draft_logits"], c["draft_logits"])
+    assert a["draft_logits"].shape == (2, w.G, 5000) and a["draft_logits"].dtype == torch.bfloat16
+    assert a["target_logits"].shape == (2, w.G + 1, 5000)
+    for k in ("u_draft", "u_accept", "u_resample"):
+        assert a[k].dtype == torch.float32 and float(a[k].min()) >= 0 and float(a[k].max()) < 1
+    # long tail: the largest logit stands well above the median
+    l = a["draft_logits"].float()
+    assert float((l.max(-1).values - l.median(-1).values).min()) > 5
+    w4 = gen.scaled(gen.WORKLOADS["config4"], B=3, V=3000)
+    d = gen.make_inputs(w4, 1)
+    T = d["temperature"].numpy()
+    assert np.all((T >= 0.5) & (T <= 1.2)) and len(set(T.tolist())) == 3
+
+
+def test_shard_ranges_partition_the_batch():
+    from paper_2603_19133_b200.shard import shard_range
+    for B in (0, 1, 7, 8, 256, 511):
+        for world in (1, 2, 3, 8):
+            ranges = [shard_range(B, r, world) for r in range(world)]
+            assert ranges[0][0] == 0 and ranges[-1][1] == B
+            assert all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))
+            sizes = [b1 - b0 for b0, b1 in ranges]
+            assert max(sizes) - min(sizes) <= 1
+
+
+_WORKER = r'''
+import os, sys
+sys.path.insert(0, sys.argv[1])
+import numpy as np, torch, torch.distributed as dist
+import gen, oracle
+from paper_2603_19133_b200.shard import shard_range, gather_sequences, max_over_ranks
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+w = gen.Workload("t", V=3000, B=7, G=3, dtype="bf16", s=1.1, sigma_d=1.5, corr=0.8, sigma_t=1.0, T=None,
+                 top_k=0, top_p=0.9, k_max=16)
+inp = gen.make_inputs(w, 11)                       # every rank generates the same global batch
+f = lambda t: t.float().numpy() if t.is_floating_point() else t.numpy()
+b0, b1 = shard_range(w.B, rank, world)
+loc = {k: f(v[b0:b1]) for k, v in inp.items()}
+# the CPU stand-in for the per-rank GPU call: each rank works on its own block of sequences only
+qi, qp, qc, tok = oracle.compress(loc["draft_logits"], loc["temperature"], w.top_k, w.top_p, w.k_max, loc["u_draft"])
+r = oracle.verify(loc["target_logits"], loc["temperature"], tok, qi, qp, qc, loc["u_accept"], loc["u_resample"])
+alen = gather_sequences(torch.from_numpy(r["accept_len"]), w.B)
+token = gather_sequences(torch.from_numpy(r["token"]), w.B)
+pd = gather_sequences(torch.from_numpy(r["p_draft"]), w.B)
+t = max_over_ranks(1.0 + rank)
+if rank == 0:
+    full = {k: f(v) for k, v in inp.items()}
+    qi, qp, qc, tok = oracle.compress(full["draft_logits"], full["temperature"], w.top_k, w.top_p, w.k_max, full["u_draft"])
+    ref = oracle.verify(full["target_logits"], full["temperature"], tok, qi, qp, qc, full["u_accept"], full["u_resample"])
+    assert np.array_equal(alen.numpy(), ref["accept_len"]) and np.array_equal(token.numpy(), ref["token"])
+    assert np.array_equal(pd.numpy(), ref["p_draft"])
+    assert t == float(world)
+    print("SHARD_OK")
+dist.destroy_process_group()
+'''
+
+
+def test_sequence_sharding_world_size_2_gloo(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(_WORKER)
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", "29571", str(script), ROOT]
+    run = subprocess.run(cmd, capture_output=True, text=True, timeout=300)
+    assert run.returncode == 0, run.stdout[-2000:] + run.stderr[-2000:]
+    assert "SHARD_OK" in run.stdout

@@ -167,6 +167,42 @@ PICOSPEC_API int picospec_residual_sample(picospec_ctx* ctx, const void* target_
                              const int* q_idx, const float* q_prob, const int* q_count, int k_max,
                              const float* u_resample, int* token, float* mass, void* cuda_stream);
 
+/* Verification without any allocation -- the paper has no counterpart; this entry point exists
+ * for callers that cannot obtain device memory at all.  Two kinds of caller are meant: a plugin
+ * inside a serving engine that has already claimed the whole of the GPU's memory for its own
+ * pools (cudaMalloc fails there, and so would picospec_create, which allocates the workspace),
+ * and a latency-critical loop that must not take the device-wide synchronisation cudaMalloc and
+ * cudaFree imply.  Such callers pass their own input and output buffers as usual and need no
+ * context.
+ *
+ * Same computation, arguments and outputs as picospec_verify (including the fused half 2b when
+ * u_resample and token are non-NULL), minus the context.  The workspace the kernels need between
+ * their passes lives in a fixed array inside the library's device image (about 1 MB, held by
+ * every GPU that loads the library until the process exits), so the problem must fit it:
+ *     B * (G + 1) <= PICOSPEC_STATIC_MAX_ROWS   and   V <= PICOSPEC_STATIC_MAX_VOCAB
+ * (k_max <= PICOSPEC_MAX_K, G <= PICOSPEC_MAX_GAMMA as everywhere); anything larger is rejected
+ * with PICOSPEC_ECAPACITY before any work is enqueued.
+ *
+ * device_status_out (DEVICE pointer to one int, or NULL) receives this call's status bits
+ * (PICOSPEC_ST_*) once the enqueued work has run; slow_rows_out (DEVICE pointer to one
+ * long long, or NULL) the number of rows this call re-evaluated in double precision.
+ *
+ * The call makes no cudaMalloc / cudaFree and calls nothing that allocates.  Its first use on a
+ * device looks up the address of the fixed array for that device (a host-side query, done once
+ * per device with that device current); make that first call outside any stream capture.
+ * Every call on a device shares the one array and the array keeps what the previous call left
+ * in it; the call clears the few words that must start at zero itself.  Two calls whose work
+ * overlaps on the GPU (different streams, or several host threads) race on the array: order
+ * them on one stream. */
+#define PICOSPEC_STATIC_MAX_ROWS 256
+#define PICOSPEC_STATIC_MAX_VOCAB 262144
+PICOSPEC_API int picospec_verify_static(const void* target_logits, picospec_dtype dtype, int B, int G, int V,
+                           long long row_stride_elems, const float* temperature, const int* draft_tok,
+                           const int* q_idx, const float* q_prob, const int* q_count, int k_max,
+                           const float* u_accept, int* accept_len, float* p_draft, float* resid_mass,
+                           int* borderline_count, const float* u_resample, int* token,
+                           int* device_status_out, long long* slow_rows_out, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

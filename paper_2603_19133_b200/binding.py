@@ -44,6 +44,9 @@ def lib() -> ctypes.CDLL:
                                                c_int, vp, vp, vp, vp]
         L.picospec_profile_enable.argtypes = [vp, c_int]
         L.picospec_profile_read.argtypes = [vp, c_int, ctypes.POINTER(c_f), ctypes.POINTER(c_int), vp]
+        L.picospec_verify_static.argtypes = [vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp, c_int,
+                                             vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.picospec_verify_static.restype = c_int
         for f in ("picospec_profile_enable", "picospec_profile_read", "picospec_create", "picospec_destroy", "picospec_last_cuda_error", "picospec_status",
                   "picospec_compress", "picospec_verify", "picospec_residual_sample"):
             getattr(L, f).restype = c_int
@@ -95,6 +98,35 @@ def _logits(t: torch.Tensor):
 
 def _stream() -> ctypes.c_void_p:
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+STATIC_MAX_ROWS, STATIC_MAX_VOCAB = 256, 262144
+
+
+def verify_static(target_logits: torch.Tensor, temperature: torch.Tensor, draft_tok: torch.Tensor,
+                  q_idx: torch.Tensor, q_prob: torch.Tensor, q_count: torch.Tensor, u_accept: torch.Tensor,
+                  u_resample: Optional[torch.Tensor], out: dict):
+    """picospec_verify_static: picospec_verify for callers that cannot allocate device memory (an
+    engine plugin on a GPU whose memory is already claimed, a loop that must avoid cudaMalloc's
+    synchronisation).  It needs no Context; its workspace is a fixed array inside the library, so
+    B * (G + 1) <= STATIC_MAX_ROWS and V <= STATIC_MAX_VOCAB.  Nothing is allocated here either:
+    every output is a tensor the caller made beforehand and passes in `out`
+    (accept_len [B], p_draft [B,G], resid_mass [B,G], borderline_count [1], token [B] or None,
+    and optionally device_status [1] int32, slow_rows [1] int64).  Calls on one device share
+    the workspace: keep them on one stream.  Returns `out`."""
+    p, dt, B, G1, V, pitch = _logits(target_logits)
+    G = G1 - 1
+    k_max = q_idx.shape[-1]
+    _check(lib().picospec_verify_static(
+        p, dt, B, G, V, pitch, _ptr(temperature, torch.float32, (B,)),
+        _ptr(draft_tok, torch.int32, (B, G)), _ptr(q_idx, torch.int32, (B, G, k_max)),
+        _ptr(q_prob, torch.float32, (B, G, k_max)), _ptr(q_count, torch.int32, (B, G)), int(k_max),
+        _ptr(u_accept, torch.float32, (B, G)), _ptr(out["accept_len"], torch.int32, (B,)),
+        _ptr(out["p_draft"], torch.float32, (B, G)), _ptr(out["resid_mass"], torch.float32, (B, G)),
+        _ptr(out["borderline_count"], torch.int32, (1,)), _ptr(u_resample, torch.float32, (B, 2)),
+        _ptr(out.get("token"), torch.int32, (B,)), _ptr(out.get("device_status"), torch.int32, (1,)),
+        _ptr(out.get("slow_rows"), torch.int64, (1,)), _stream()), "picospec_verify_static")
+    return out
 
 
 class Context:

@@ -2,8 +2,11 @@
 #include "../../include/picospec.h"
 
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 #include <stdlib.h>
+
+#include <mutex>
 
 #include "compress_kernels.cuh"
 #include "verify_kernels.cuh"
@@ -376,3 +379,104 @@ int picospec_residual_sample(picospec_ctx* ctx, const void* target_logits, picos
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// picospec_verify_static: the verify kernels on a workspace that is part of the device image.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int STATIC_ROWS = PICOSPEC_STATIC_MAX_ROWS;
+constexpr int STATIC_NCH = (PICOSPEC_STATIC_MAX_VOCAB + CHUNK - 1) / CHUNK;
+
+struct StaticWorkspace {
+    float2 stats[STATIC_ROWS * STATIC_NCH];
+    double dsum[STATIC_ROWS * STATIC_NCH];
+    float row_max[STATIC_ROWS];
+    int queue[STATIC_ROWS];
+    // the words below must read zero when a call starts; one memset covers them
+    int counters[4];
+    unsigned status;
+    unsigned pad;
+    unsigned long long slow_rows;
+};
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never an address a kernel
+// could use; the per-device address is looked up below.
+static __device__ __align__(256) unsigned char g_static_workspace[sizeof(StaticWorkspace)];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+StaticWorkspace* g_static_ptr[STATIC_MAX_DEVICES];   // device address of the array, per device
+int g_static_sms[STATIC_MAX_DEVICES];
+
+// Once per device, with that device current: the device address of the array and the SM count.
+cudaError_t static_workspace(int device, StaticWorkspace** ws, int* sms) {
+    if (device < 0 || device >= STATIC_MAX_DEVICES) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[device]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_static_workspace);
+        if (e != cudaSuccess) return e;
+        int n = 0;
+        e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device);
+        if (e != cudaSuccess) return e;
+        g_static_sms[device] = n;
+        g_static_ptr[device] = static_cast<StaticWorkspace*>(p);
+    }
+    *ws = g_static_ptr[device];
+    *sms = g_static_sms[device];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int picospec_verify_static(const void* target_logits, picospec_dtype dtype, int B, int G, int V,
+                                      long long row_stride_elems, const float* temperature, const int* draft_tok,
+                                      const int* q_idx, const float* q_prob, const int* q_count, int k_max,
+                                      const float* u_accept, int* accept_len, float* p_draft, float* resid_mass,
+                                      int* borderline_count, const float* u_resample, int* token,
+                                      int* device_status_out, long long* slow_rows_out, void* cuda_stream) {
+    if (!target_logits || !temperature) return PICOSPEC_EINVAL;
+    if (dtype != PICOSPEC_F32 && dtype != PICOSPEC_BF16) return PICOSPEC_EINVAL;
+    if (B < 0 || G < 0 || V <= 0 || k_max <= 0 || row_stride_elems < V) return PICOSPEC_EINVAL;
+    if (!accept_len || !borderline_count) return PICOSPEC_EINVAL;
+    if (G > 0 && (!draft_tok || !q_idx || !q_prob || !q_count || !u_accept || !p_draft || !resid_mass))
+        return PICOSPEC_EINVAL;
+    if ((u_resample == nullptr) != (token == nullptr)) return PICOSPEC_EINVAL;
+    if (G > PICOSPEC_MAX_GAMMA || k_max > PICOSPEC_MAX_K || V > PICOSPEC_STATIC_MAX_VOCAB ||
+        (long long)B * (G + 1) > STATIC_ROWS)
+        return PICOSPEC_ECAPACITY;
+    if (B == 0) return PICOSPEC_OK;
+
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return PICOSPEC_ECUDA;
+    StaticWorkspace* ws = nullptr;
+    picospec_ctx local = {};          // host-side launch parameters only; owns nothing
+    local.device = device;
+    if (static_workspace(device, &ws, &local.num_sms) != cudaSuccess) return PICOSPEC_ECUDA;
+
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const size_t tail = sizeof(StaticWorkspace) - offsetof(StaticWorkspace, counters);
+    if (cudaMemsetAsync(ws->counters, 0, tail, s) != cudaSuccess) return PICOSPEC_ECUDA;
+
+    VerifyArgs a;
+    a.logits = target_logits; a.row_stride = row_stride_elems;
+    a.B = B; a.G = G; a.V = V; a.k_max = k_max; a.sample_only = 0;
+    a.nch = (V + CHUNK - 1) / CHUNK;
+    a.temperature = temperature; a.draft_tok = draft_tok; a.q_idx = q_idx; a.q_prob = q_prob; a.q_count = q_count;
+    a.u_accept = u_accept; a.pos = nullptr; a.u_resample = u_resample;
+    a.accept_len = accept_len; a.p_draft = p_draft; a.resid_mass = resid_mass; a.borderline = borderline_count;
+    a.token = token; a.mass = nullptr;
+    a.stats = ws->stats; a.row_max = ws->row_max; a.dsum = ws->dsum; a.queue = ws->queue;
+    a.queue_count = ws->counters; a.status = &ws->status; a.slow_rows = &ws->slow_rows;
+    cudaError_t e;
+    if (dtype == PICOSPEC_BF16)
+        e = launch_verify<__nv_bfloat16>(&local, a, rows_aligned(a.logits, a.row_stride, 2), s);
+    else
+        e = launch_verify<float>(&local, a, rows_aligned(a.logits, a.row_stride, 4), s);
+    if (e == cudaSuccess && device_status_out)
+        e = cudaMemcpyAsync(device_status_out, &ws->status, sizeof(int), cudaMemcpyDeviceToDevice, s);
+    if (e == cudaSuccess && slow_rows_out)
+        e = cudaMemcpyAsync(slow_rows_out, &ws->slow_rows, sizeof(long long), cudaMemcpyDeviceToDevice, s);
+    return e == cudaSuccess ? PICOSPEC_OK : PICOSPEC_ECUDA;
+}

@@ -54,6 +54,7 @@ typedef enum {
 #define PICOSPEC_ST_TEMPERATURE 1 /* temperature not finite or <= 0                              */
 #define PICOSPEC_ST_LOGIT 2       /* NaN or +inf logit, or a row with no finite logit            */
 #define PICOSPEC_ST_RANGE 4       /* draft token, sparse index, count or position out of range   */
+#define PICOSPEC_ST_INTERNAL 8    /* a bounded wait inside a kernel ran out (outputs not valid)  */
 
 #define PICOSPEC_CHUNK 1024 /* vocabulary entries per level-1 chunk of the residual sampler      */
 #define PICOSPEC_MAX_K 1024 /* largest k_max a context accepts                                   */

@@ -114,13 +114,40 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
     return cudaGetLastError();
 }
 
+// Opt-in shared-memory sizes of the staged kernels: once per device and process.
+cudaError_t ensure_kernel_attrs(int device) {
+    static std::mutex mu;
+    static bool done[64];
+    if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (done[device]) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(chunk_stats_bulk_kernel<__nv_bfloat16>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         TileGeom<__nv_bfloat16>::SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(chunk_stats_bulk_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TileGeom<float>::SMEM_BYTES);
+    if (e == cudaSuccess) done[device] = true;
+    return e;
+}
+
 template <typename T>
 cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, cudaStream_t s) {
     const long long items = (long long)(a.sample_only ? a.B : a.B * (a.G + 1)) * a.nch;
     long long want = (items + WARPS - 1) / WARPS;
     const int cap = ctx->num_sms * 4;
     const int grid = (int)(want < cap ? want : cap);
-    {
+    const bool staged = aligned && ((size_t)a.V * sizeof(T)) % 16 == 0;
+    if (staged) {
+        cudaError_t ea = ensure_kernel_attrs(ctx->device);
+        if (ea != cudaSuccess) return ea;
+        const int tiles_per_row = (a.nch + TILE_CHUNKS - 1) / TILE_CHUNKS;
+        const long long tiles = (long long)(a.sample_only ? a.B : a.B * (a.G + 1)) * tiles_per_row;
+        const int gcap = ctx->num_sms * 2;
+        const int g = (int)(tiles < gcap ? tiles : gcap);
+        ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_STREAM, 1, s);
+        chunk_stats_bulk_kernel<T><<<g, STREAM_THREADS, TileGeom<T>::SMEM_BYTES, s>>>(a, tiles_per_row, tiles);
+    } else {
         ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_STREAM, 1, s);
         if (aligned) chunk_stats_kernel<T, true><<<grid, THREADS, 0, s>>>(a);
         else chunk_stats_kernel<T, false><<<grid, THREADS, 0, s>>>(a);

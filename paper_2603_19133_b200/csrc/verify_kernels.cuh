@@ -3,6 +3,7 @@
 #pragma once
 #include "common.cuh"
 #include "precise_kernels.cuh"
+#include "stream_pipeline.cuh"
 
 namespace picospec {
 
@@ -116,6 +117,116 @@ __global__ void __launch_bounds__(THREADS, 4) chunk_stats_kernel(VerifyArgs a) {
         }
         if (mB.valid) chunk_stats_compute<T>(Bf, mB, a.stats, lane);
         if (!hasA) break;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Streaming pass through shared memory (rows whose base, pitch and length are multiples of 16
+// bytes).  A tile is TILE_CHUNKS consecutive chunks of one row; CTA c takes tiles c, c + grid,
+// c + 2 grid, ...  Warp 8 lane 0 is the producer: it keeps STAGES bulk copies in flight.  Each of
+// the 8 consumer warps moves its chunk of a landed tile to registers, hands the stage back and
+// then reduces the chunk to (maximum logit, fp32 sum of 2^((l - max) * log2e / T)).
+// ---------------------------------------------------------------------------------------------
+struct TileDesc {
+    int src_row;   // row of the logits tensor
+    int c0;        // first chunk of the tile
+    float c32;     // log2(e) / T of the row's sequence
+    int valid;     // 0: bad temperature or position, nothing was copied
+};
+
+template <typename T>
+__global__ void __launch_bounds__(STREAM_THREADS, 2) chunk_stats_bulk_kernel(VerifyArgs a, int tiles_per_row,
+                                                                             long long total_tiles) {
+    extern __shared__ __align__(1024) unsigned char stage_mem[];
+    constexpr int STAGES = StreamCfg<T>::STAGES;
+    constexpr int TILE_BYTES = TileGeom<T>::TILE_BYTES;
+    __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES];
+    __shared__ TileDesc desc[STAGES];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], WARPS);
+        }
+        mbar_init_fence();
+        if (blockIdx.x == 0) {
+            *a.queue_count = 0;
+            if (a.borderline) *a.borderline = 0;
+        }
+    }
+    __syncthreads();
+
+    if (warp == WARPS) {
+        // ---- producer ---------------------------------------------------------------------
+        if (lane != 0) return;
+        const uint64_t pol = l2_evict_first_policy();
+        long long t = blockIdx.x;
+        for (uint32_t i = 0; t < total_tiles; ++i, t += gridDim.x) {
+            const int s = (int)(i % STAGES);
+            const uint32_t round = i / STAGES;
+            if (round > 0 && !mbar_wait(&empty[s], (round - 1) & 1)) {
+                atomicOr(a.status, ST_INTERNAL);
+                break;
+            }
+            const int r = (int)(t / tiles_per_row);
+            const int tc = (int)(t - (long long)r * tiles_per_row);
+            TileDesc d;
+            d.valid = 1;
+            int b;
+            if (a.sample_only) {
+                b = r;
+                const int j = a.pos[b];
+                if (j < 0 || j > a.G) d.valid = 0;
+                d.src_row = b * (a.G + 1) + (d.valid ? j : 0);
+            } else {
+                b = r / (a.G + 1);
+                d.src_row = r;
+            }
+            const float Tb = a.temperature[b];
+            if (!temp_ok(Tb)) d.valid = 0;
+            d.c32 = temp_scale(Tb);
+            d.c0 = tc * TILE_CHUNKS;
+            desc[s] = d;
+            if (d.valid) {
+                const int v0 = d.c0 * CHUNK;
+                const int v1 = min(a.V, v0 + TILE_CHUNKS * CHUNK);
+                const uint32_t bytes = (uint32_t)(v1 - v0) * (uint32_t)sizeof(T);
+                const T* src = reinterpret_cast<const T*>(a.logits) + (long long)d.src_row * a.row_stride + v0;
+                mbar_arrive_expect_tx(&full[s], bytes);
+                bulk_load(stage_mem + s * TILE_BYTES, src, bytes, &full[s], pol);
+            } else {
+                mbar_arrive(&full[s]);
+            }
+        }
+        return;
+    }
+
+    // ---- consumers ------------------------------------------------------------------------
+    long long t = blockIdx.x;
+    for (uint32_t i = 0; t < total_tiles; ++i, t += gridDim.x) {
+        const int s = (int)(i % STAGES);
+        const uint32_t round = i / STAGES;
+        if (!mbar_wait(&full[s], round & 1)) {
+            if (lane == 0) atomicOr(a.status, ST_INTERNAL);
+            break;
+        }
+        const TileDesc d = desc[s];
+        const int c = d.c0 + warp;
+        const bool work = d.valid && c < a.nch;
+        ChunkRegs<T> regs;
+        if (work) load_staged(regs, stage_mem + s * TILE_BYTES + warp * (CHUNK * (int)sizeof(T)), c * CHUNK, a.V, lane);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[s]);
+        if (work) {
+            const float lm = regs.lane_max();
+            const float cm = warp_max(lm);
+            const float off = __fmul_rn(cm, d.c32);
+            float sum = 0.f;
+            if (cm > -CUDART_INF_F) sum = lane_exp_sum2(regs, d.c32, off);
+            if (lm != lm) sum = CUDART_NAN_F;     // NaN in the chunk: the finish kernel reports it
+            sum = warp_sum(sum);
+            if (lane == 0) a.stats[(long long)d.src_row * a.nch + c] = make_float2(cm, sum);
+        }
     }
 }
 

@@ -179,7 +179,7 @@ class Step:
                       "resid_mass": torch.empty((B, G), dtype=f32, device=dev),
                       "borderline_count": torch.empty((1,), dtype=i32, device=dev),
                       "token": torch.empty((B,), dtype=i32, device=dev)}
-        self.launches_per_step = (3 if w.top_p < 1.0 else 1) + 4
+        self.launches_per_step = (5 if w.top_p < 1.0 else 3) + 4
 
     def compress(self, inp=None):
         inp = inp or self.inp

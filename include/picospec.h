@@ -78,12 +78,14 @@ PICOSPEC_API int picospec_last_cuda_error(const picospec_ctx* ctx);
  * streaming kernels (one per hot call) with CUDA events on the caller's stream, 2 = bracket every
  * kernel group.  Enabling creates the events (host objects; no device memory) and resets the
  * counters; call it outside timed or captured regions.  The paper has no counterpart. */
-#define PICOSPEC_PROF_COMPRESS_STREAM 0  /* compress: streaming select kernel                    */
+#define PICOSPEC_PROF_COMPRESS_STREAM 0  /* compress: streaming filter (or direct select) kernel  */
 #define PICOSPEC_PROF_VERIFY_STREAM 1    /* verify / residual_sample: streaming statistics kernel */
 #define PICOSPEC_PROF_VERIFY_FINISH 2    /* verify: per-sequence finish kernel                   */
 #define PICOSPEC_PROF_VERIFY_PRECISE 3   /* verify: double-precision re-evaluation kernels       */
 #define PICOSPEC_PROF_COMPRESS_PRECISE 4 /* compress: double-precision re-evaluation kernels     */
-#define PICOSPEC_PROF_KINDS 5
+#define PICOSPEC_PROF_COMPRESS_REDO 5    /* compress: direct kernel on rows handed over by the staged one */
+#define PICOSPEC_PROF_COMPRESS_FINISH 6  /* compress: per-row sort / cut / emit kernel of the staged path   */
+#define PICOSPEC_PROF_KINDS 7
 PICOSPEC_API int picospec_profile_enable(picospec_ctx* ctx, int level);
 
 /* Synchronise `cuda_stream`, then return the summed device time (ms, HOST pointer) and the number

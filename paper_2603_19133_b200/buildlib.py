@@ -30,7 +30,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         stale = any(os.path.getmtime(p) > t for p in _deps())
     if stale:
         nvcc = os.environ.get("NVCC", "nvcc")
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + SOURCES
+        extra = os.environ.get("PICOSPEC_NVCC_FLAGS", "").split()     # e.g. -DPICOSPEC_STAGES_BF16=3
+        cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + SOURCES
         res = subprocess.run(cmd, capture_output=True, text=True)
         if verbose or res.returncode != 0:
             sys.stderr.write(res.stdout + res.stderr)

@@ -56,8 +56,26 @@ __device__ __forceinline__ int warp_sum(int v) {
     return v;
 }
 
-// Inclusive scan of one double per thread over a 256-thread CTA.  warp_tot: 8 doubles of shared
-// memory.  Contains two __syncthreads.
+// Barrier over the 256 worker threads (warps 0..7) of a CTA.  Kernels that carry an extra producer
+// warp cannot use __syncthreads in code their workers share with plain 256-thread kernels, so the
+// cooperative routines below all synchronise on named barrier 1.
+__device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// The same barrier, returning the OR of `pred` over the 256 workers.
+__device__ __forceinline__ bool workers_sync_or(bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, 256, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred)
+        : "memory");
+    return r != 0;
+}
+
+// Inclusive scan of one double per thread over the 256 worker threads.  warp_tot: 8 doubles of
+// shared memory.  Contains two barriers.
 __device__ __forceinline__ double block_scan_incl(double x, double* warp_tot, double& total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
@@ -66,7 +84,7 @@ __device__ __forceinline__ double block_scan_incl(double x, double* warp_tot, do
         if (lane >= d) x += y;
     }
     if (lane == 31) warp_tot[warp] = x;
-    __syncthreads();
+    workers_sync();
     double base = 0.0, tot = 0.0;
 #pragma unroll
     for (int w = 0; w < WARPS; ++w) {
@@ -74,7 +92,7 @@ __device__ __forceinline__ double block_scan_incl(double x, double* warp_tot, do
         if (w < warp) base += t;
         tot += t;
     }
-    __syncthreads();
+    workers_sync();
     total = tot;
     return x + base;
 }

@@ -9,6 +9,8 @@ namespace picospec {
 
 typedef unsigned long long u64;
 
+struct CsRowMeta;   // per-row record the staged filter kernel leaves for its finish kernel
+
 constexpr int ITER_ELEMS = WARPS * CHUNK;            // entries one CTA iteration can push at most
 constexpr int CAND_CAP = ITER_ELEMS + 2 * MAX_K;     // candidate buffer (keys)
 constexpr int COMPRESS_SMEM = CAND_CAP * 8 + MAX_K * 8;   // candidate keys + staging / sorted keys
@@ -32,6 +34,14 @@ struct CompressArgs {
     int* queue_count_next;     // cleared by this call for the next one
     unsigned* status;
     unsigned long long* slow_rows;
+    // rows the staged kernel hands to the direct kernel (candidate buffer overflow)
+    int* redo_rows;            // [B*G]
+    int* redo_count;           // zero on entry of the staged kernel
+    int* redo_count_next;      // cleared for the next call
+    int use_redo_list;         // direct kernel: 1 = process redo_rows[0 .. *redo_count) only
+    // staged path: survivors of the filter kernel, [B*G, cs_survivor_cap(k_max)] keys + one record per row
+    unsigned long long* surv_keys;
+    CsRowMeta* surv_meta;
 };
 
 // Monotone map float -> uint32 (larger float, larger key); -0 is folded onto +0 so that the two
@@ -82,7 +92,7 @@ __device__ u64 radix_select_kth(const u64* keys, int count, int k, CompressShare
         // orderable form is the complement); the top byte of the index part is 0xFF
         const bool logit_low = LOGIT16 && (shift == 40 || shift == 32);
         if (logit_low || shift == 24) {
-            __syncthreads();
+            workers_sync();
             if (tid == 0) {
                 const u64 digit = (shift == 24 || !(sh.prefix >> 63)) ? 0xFFull : 0x00ull;
                 sh.prefix |= digit << shift;
@@ -91,13 +101,13 @@ __device__ u64 radix_select_kth(const u64* keys, int count, int k, CompressShare
             continue;
         }
         sh.hist[tid] = 0;
-        __syncthreads();
+        workers_sync();
         const u64 prefix = sh.prefix;
         for (int i = tid; i < count; i += THREADS) {
             const u64 key = keys[i];
             if ((key & mask) == prefix) atomicAdd(&sh.hist[(int)((key >> shift) & 0xFF)], 1);
         }
-        __syncthreads();
+        workers_sync();
         if (warp == 0) {
             int loc[8], s = 0;
 #pragma unroll
@@ -126,33 +136,34 @@ __device__ u64 radix_select_kth(const u64* keys, int count, int k, CompressShare
             }
         }
         mask |= 0xFFull << shift;
-        __syncthreads();
+        workers_sync();
     }
-    __syncthreads();
+    workers_sync();
     return sh.prefix;
 }
 
 // Keep the k largest keys of cand[0..count): afterwards cand[0..k) holds them (unordered).
 template <bool LOGIT16>
-__device__ void keep_top_k(u64* cand, u64* keep, int count, int k, CompressShared& sh) {
+__device__ u64 keep_top_k(u64* cand, u64* keep, int count, int k, CompressShared& sh) {
     const u64 kth = radix_select_kth<LOGIT16>(cand, count, k, sh);
-    __syncthreads();
+    workers_sync();
     if (threadIdx.x == 0) sh.count = 0;
-    __syncthreads();
+    workers_sync();
     for (int i = threadIdx.x; i < count; i += THREADS) {
         const u64 key = cand[i];
         if (key >= kth) keep[atomicAdd(&sh.count, 1)] = key;   // keys are distinct: exactly k pass
     }
-    __syncthreads();
+    workers_sync();
     for (int i = threadIdx.x; i < k; i += THREADS) cand[i] = keep[i];
-    __syncthreads();
+    workers_sync();
+    return kth;
 }
 
 // Descending bitonic sort of keys[0..n2), n2 a power of two.
 __device__ void bitonic_sort_desc(u64* keys, int n2) {
     for (int size = 2; size <= n2; size <<= 1) {
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            __syncthreads();
+            workers_sync();
             for (int i = threadIdx.x; i < (n2 >> 1); i += THREADS) {
                 const int pos = 2 * i - (i & (stride - 1));
                 const int j = pos + stride;
@@ -165,7 +176,7 @@ __device__ void bitonic_sort_desc(u64* keys, int n2) {
             }
         }
     }
-    __syncthreads();
+    workers_sync();
 }
 
 __device__ __forceinline__ void emit_invalid_row(const CompressArgs& a, int row) {
@@ -214,7 +225,7 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
         for (int e = 3; e >= 0; --e)
             if (tid * 4 + e < k_eff && base + cum[e] >= thrZ) mine = tid * 4 + e;
         if (mine != 0x7fffffff) atomicMin(&sh.first, mine);
-        __syncthreads();
+        workers_sync();
         const int jn = sh.first;   // rank of the entry that reaches top_p, if any
         if (jn != 0x7fffffff && jn == mine) {
             sh.n = jn + 1;
@@ -230,13 +241,13 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
         if (!PRECISE && jn == 0x7fffffff && tid == 0) {
             // never reached: n = k_eff either way, nothing to decide
         }
-        __syncthreads();
+        workers_sync();
     }
     const int n = sh.n;
 #pragma unroll
     for (int e = 0; e < 4; ++e)
         if (tid * 4 + e == n - 1) sh.Wn = base + cum[e];
-    __syncthreads();
+    workers_sync();
     const double Wn = sh.Wn;
     // stored probabilities, and their running sum for the draft draw
     float pf[4];
@@ -281,7 +292,7 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
         }
         if (mine != 0x7fffffff) atomicMin(&sh.first, mine);
         if (mylast >= 0) atomicMax(&sh.last, mylast);
-        __syncthreads();
+        workers_sync();
         if (tid == 0) {
             const int j = sh.first != 0x7fffffff ? sh.first : sh.last;
             a.draft_tok[row] = j >= 0 ? key_index(keys[j]) : -1;
@@ -295,7 +306,7 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
             atomicAdd(a.slow_rows, 1ull);
         }
     }
-    __syncthreads();
+    workers_sync();
 }
 
 template <typename T, bool ALIGNED, bool STATS>
@@ -312,12 +323,14 @@ __global__ void __launch_bounds__(THREADS, 2) compress_kernel(CompressArgs a) {
     if (k_eff > a.k_max) k_eff = a.k_max;
     if (k_eff > a.V) k_eff = a.V;
 
-    if (blockIdx.x == 0 && tid == 0) *a.queue_count_next = 0;
+    if (blockIdx.x == 0 && tid == 0 && !a.use_redo_list) *a.queue_count_next = 0;
+    const int nwork = a.use_redo_list ? *a.redo_count : rows;
 
-    for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+    for (int wi = blockIdx.x; wi < nwork; wi += gridDim.x) {
+        const int row = a.use_redo_list ? a.redo_rows[wi] : wi;
         const int b = row / a.G;
         const float Tb = a.temperature[b];
-        __syncthreads();
+        workers_sync();
         if (!temp_ok(Tb)) {
             emit_invalid_row(a, row);
             if (tid == 0) atomicOr(a.status, ST_TEMPERATURE);
@@ -330,7 +343,7 @@ __global__ void __launch_bounds__(THREADS, 2) compress_kernel(CompressArgs a) {
             sh.thr = -CUDART_INF_F;
             sh.nan = 0;
         }
-        __syncthreads();
+        workers_sync();
 
         // running softmax statistics of this warp: fp32 lane sums relative to the warp's running
         // maximum; when the maximum rises the sums are folded into a double and rescaled exactly
@@ -375,23 +388,23 @@ __global__ void __launch_bounds__(THREADS, 2) compress_kernel(CompressArgs a) {
                     }
                 }
             }
-            __syncthreads();
+            workers_sync();
             if (sh.count > CAND_CAP - ITER_ELEMS) {
                 const int count = sh.count;
-                __syncthreads();
+                workers_sync();
                 keep_top_k<LOGIT16>(cand, keep, count, k_eff, sh);
                 // sh.count == k_eff now; the k-th key's logit is the new admission threshold
                 float mn = CUDART_INF_F;
                 for (int i = tid; i < k_eff; i += THREADS) mn = fminf(mn, key_logit(cand[i]));
                 mn = -warp_max(-mn);
                 if (lane == 0) sh.wM[warp] = mn;
-                __syncthreads();
+                workers_sync();
                 if (tid == 0) {
                     float m = sh.wM[0];
                     for (int w = 1; w < WARPS; ++w) m = fminf(m, sh.wM[w]);
                     sh.thr = m;
                 }
-                __syncthreads();
+                workers_sync();
             }
         };
         for (int it = 0; it < iters; it += 2) {
@@ -407,7 +420,7 @@ __global__ void __launch_bounds__(THREADS, 2) compress_kernel(CompressArgs a) {
                 sh.wM[warp] = runM;
                 sh.wS[warp] = folded + s;   // relative to runOff = fp32(runM * c32)
             }
-            __syncthreads();
+            workers_sync();
             float m = sh.wM[0];
             for (int w = 1; w < WARPS; ++w) m = fmaxf(m, sh.wM[w]);
             if (m > -CUDART_INF_F && m < CUDART_INF_F) {
@@ -417,11 +430,11 @@ __global__ void __launch_bounds__(THREADS, 2) compress_kernel(CompressArgs a) {
                 Z *= stream_sum_scale(m, c32);
             }
         }
-        __syncthreads();
+        workers_sync();
 
         // ---- final selection and order --------------------------------------------------------
         int count = sh.count;
-        __syncthreads();
+        workers_sync();
         if (count > k_eff) {
             keep_top_k<LOGIT16>(cand, keep, count, k_eff, sh);
             count = k_eff;
@@ -458,7 +471,7 @@ __global__ void __launch_bounds__(THREADS) compress_precise_kernel(CompressArgs 
         const int row = a.queue[slot];
         const int b = row / a.G;
         const T* rowp = reinterpret_cast<const T*>(a.logits) + (long long)row * a.row_stride;
-        __syncthreads();
+        workers_sync();
         for (int j = tid; j < k_eff; j += THREADS) {
             const int v = a.q_idx[(long long)row * a.k_max + j];
             keep[j] = make_key(load_logit(rowp, v), v);
@@ -467,10 +480,10 @@ __global__ void __launch_bounds__(THREADS) compress_precise_kernel(CompressArgs 
         for (int c = tid; c < a.nch; c += THREADS) s += a.dsum[(long long)row * a.nch + c];
         s = warp_sum(s);
         if (lane == 0) sh.wS[warp] = s;
-        __syncthreads();
+        workers_sync();
         double Z = 0.0;
         for (int w = 0; w < WARPS; ++w) Z += sh.wS[w];
-        __syncthreads();
+        workers_sync();
         finish_row<true>(a, row, keep, k_eff, a.temperature[b], Z, sh);
     }
 }

@@ -9,6 +9,7 @@
 #include <mutex>
 
 #include "compress_kernels.cuh"
+#include "compress_stream_kernel.cuh"
 #include "verify_kernels.cuh"
 
 using namespace picospec;
@@ -30,7 +31,10 @@ struct picospec_ctx {
     double* dsum;
     float* row_max;
     int* queue;
-    int* counters;  // [0] verify queue count, [1],[2] compress queue counts (alternating)
+    int* counters;  // [0] verify queue, [1],[2] compress queue (alternating), [3],[4] compress redo list (alternating)
+    int* redo_rows; // rows the staged compress kernel hands to the direct kernel
+    unsigned long long* surv_keys;  // staged compress: survivors per row
+    CsRowMeta* surv_meta;
     unsigned* status;
     unsigned long long* slow_rows;
 };
@@ -85,20 +89,79 @@ template <typename T> void set_compress_attrs() {
     cudaFuncSetAttribute(compress_kernel<T, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, COMPRESS_SMEM);
 }
 
+// Opt-in shared-memory sizes of the staged kernels: once per device and process.
+cudaError_t ensure_kernel_attrs(int device) {
+    static std::mutex mu;
+    static bool done[64];
+    if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (done[device]) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(chunk_stats_bulk_kernel<__nv_bfloat16>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         TileGeom<__nv_bfloat16>::SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(chunk_stats_bulk_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TileGeom<float>::SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(compress_filter_kernel<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 CsGeom<__nv_bfloat16>::SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(compress_filter_kernel<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 CsGeom<__nv_bfloat16>::SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(compress_filter_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 CsGeom<float>::SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(compress_filter_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 CsGeom<float>::SMEM_BYTES);
+    if (e == cudaSuccess) done[device] = true;
+    return e;
+}
+
+template <typename T, bool ALIGNED>
+void launch_compress_direct(const CompressArgs& a, int grid, bool stats, cudaStream_t s) {
+    if (stats) compress_kernel<T, ALIGNED, true><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+    else compress_kernel<T, ALIGNED, false><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+}
+
 template <typename T>
 cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool aligned, cudaStream_t s) {
     const int rows = a.B * a.G;
     const int grid = rows < ctx->num_sms * 2 ? rows : ctx->num_sms * 2;
     const bool stats = a.top_p < 1.0f;
-    {
-        ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_STREAM, 1, s);
-        if (aligned) {
-            if (stats) compress_kernel<T, true, true><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
-            else compress_kernel<T, true, false><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
-        } else {
-            if (stats) compress_kernel<T, false, true><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
-            else compress_kernel<T, false, false><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+    // staged kernel: 16-byte aligned rows of at least one full tile
+    const bool staged = aligned && ((size_t)a.V * sizeof(T)) % 16 == 0 && a.V >= TILE_CHUNKS * CHUNK;
+    if (staged) {
+        cudaError_t ea = ensure_kernel_attrs(ctx->device);
+        if (ea != cudaSuccess) return ea;
+        const int tiles_per_row = (a.nch + TILE_CHUNKS - 1) / TILE_CHUNKS;
+        const int per_sm = CsGeom<T>::SMEM_BYTES > 110 * 1024 ? 1 : 2;
+        const int g = rows < ctx->num_sms * per_sm ? rows : ctx->num_sms * per_sm;
+        {
+            ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_STREAM, 1, s);
+            if (stats) compress_filter_kernel<T, true><<<g, STREAM_THREADS, CsGeom<T>::SMEM_BYTES, s>>>(a, tiles_per_row);
+            else compress_filter_kernel<T, false><<<g, STREAM_THREADS, CsGeom<T>::SMEM_BYTES, s>>>(a, tiles_per_row);
         }
+        cudaError_t e0 = cudaGetLastError();
+        if (e0 != cudaSuccess) return e0;
+        {
+            int n2 = 1;
+            while (n2 < cs_survivor_cap(a.k_max)) n2 <<= 1;
+            ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_FINISH, 2, s);
+            if (stats) compress_finish_kernel<T, true><<<rows, THREADS, (size_t)n2 * 8, s>>>(a);
+            else compress_finish_kernel<T, false><<<rows, THREADS, (size_t)n2 * 8, s>>>(a);
+        }
+        e0 = cudaGetLastError();
+        if (e0 != cudaSuccess) return e0;
+        // rows whose candidates did not fit (normally none: every CTA returns at once)
+        CompressArgs r = a;
+        r.use_redo_list = 1;
+        ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_REDO, 2, s);
+        launch_compress_direct<T, true>(r, grid, stats, s);
+    } else {
+        ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_STREAM, 1, s);
+        if (aligned) launch_compress_direct<T, true>(a, grid, stats, s);
+        else launch_compress_direct<T, false>(a, grid, stats, s);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || !stats) return e;
@@ -114,23 +177,6 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
     return cudaGetLastError();
 }
 
-// Opt-in shared-memory sizes of the staged kernels: once per device and process.
-cudaError_t ensure_kernel_attrs(int device) {
-    static std::mutex mu;
-    static bool done[64];
-    if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
-    std::lock_guard<std::mutex> lock(mu);
-    if (done[device]) return cudaSuccess;
-    cudaError_t e = cudaFuncSetAttribute(chunk_stats_bulk_kernel<__nv_bfloat16>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         TileGeom<__nv_bfloat16>::SMEM_BYTES);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(chunk_stats_bulk_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 TileGeom<float>::SMEM_BYTES);
-    if (e == cudaSuccess) done[device] = true;
-    return e;
-}
-
 template <typename T>
 cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, cudaStream_t s) {
     const long long items = (long long)(a.sample_only ? a.B : a.B * (a.G + 1)) * a.nch;
@@ -143,7 +189,7 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
         if (ea != cudaSuccess) return ea;
         const int tiles_per_row = (a.nch + TILE_CHUNKS - 1) / TILE_CHUNKS;
         const long long tiles = (long long)(a.sample_only ? a.B : a.B * (a.G + 1)) * tiles_per_row;
-        const int gcap = ctx->num_sms * 2;
+        const int gcap = ctx->num_sms * StreamCfg<T>::CTAS_PER_SM;
         const int g = (int)(tiles < gcap ? tiles : gcap);
         ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_STREAM, 1, s);
         chunk_stats_bulk_kernel<T><<<g, STREAM_THREADS, TileGeom<T>::SMEM_BYTES, s>>>(a, tiles_per_row, tiles);
@@ -207,10 +253,13 @@ int picospec_create(picospec_ctx** out, int device, int max_batch, int max_gamma
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->dsum, rows * nch * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->row_max, rows * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->queue, rows * sizeof(int));
-    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->counters, 4 * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->counters, 8 * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->redo_rows, rows * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_keys, rows * (size_t)cs_survivor_cap(max_k) * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_meta, rows * sizeof(CsRowMeta));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->status, sizeof(unsigned));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->slow_rows, sizeof(unsigned long long));
-    if (e == cudaSuccess) e = cudaMemset(ctx->counters, 0, 4 * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(ctx->counters, 0, 8 * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(unsigned));
     if (e == cudaSuccess) e = cudaMemset(ctx->slow_rows, 0, sizeof(unsigned long long));
     if (e == cudaSuccess) {
@@ -235,6 +284,9 @@ int picospec_destroy(picospec_ctx* ctx) {
     cudaFree(ctx->row_max);
     cudaFree(ctx->queue);
     cudaFree(ctx->counters);
+    cudaFree(ctx->redo_rows);
+    cudaFree(ctx->surv_keys);
+    cudaFree(ctx->surv_meta);
     cudaFree(ctx->status);
     cudaFree(ctx->slow_rows);
     free(ctx);
@@ -338,6 +390,12 @@ int picospec_compress(picospec_ctx* ctx, const void* draft_logits, picospec_dtyp
     const int cur = 1 + (int)(ctx->compress_calls & 1ull);
     a.queue_count = ctx->counters + cur;
     a.queue_count_next = ctx->counters + (3 - cur);
+    a.redo_rows = ctx->redo_rows;
+    a.redo_count = ctx->counters + 2 + cur;           // [3] / [4]
+    a.redo_count_next = ctx->counters + 2 + (3 - cur);
+    a.use_redo_list = 0;
+    a.surv_keys = ctx->surv_keys;
+    a.surv_meta = ctx->surv_meta;
     ctx->compress_calls++;
     a.status = ctx->status; a.slow_rows = ctx->slow_rows;
     cudaStream_t s = (cudaStream_t)cuda_stream;

@@ -117,11 +117,27 @@ constexpr int TILE_CHUNKS = WARPS;               // one chunk per consumer warp
 constexpr int STREAM_THREADS = THREADS + 32;     // consumer warps + the producer warp
 
 template <typename T> struct StreamCfg;
+// Tunables (overridable at build time): stages per CTA and CTAs per SM of the staged kernels.
+// bf16 rows carry twice the arithmetic per byte, so they get more resident warps per SM.
+#ifndef PICOSPEC_STAGES_BF16
+#define PICOSPEC_STAGES_BF16 4                   // 4 x 16 KB in flight per CTA
+#endif
+#ifndef PICOSPEC_STAGES_F32
+#define PICOSPEC_STAGES_F32 3                    // 3 x 32 KB in flight per CTA
+#endif
+#ifndef PICOSPEC_CTAS_PER_SM_BF16
+#define PICOSPEC_CTAS_PER_SM_BF16 3
+#endif
+#ifndef PICOSPEC_CTAS_PER_SM_F32
+#define PICOSPEC_CTAS_PER_SM_F32 2
+#endif
 template <> struct StreamCfg<__nv_bfloat16> {
-    static constexpr int STAGES = 4;             // 4 x 16 KB in flight per CTA
+    static constexpr int STAGES = PICOSPEC_STAGES_BF16;
+    static constexpr int CTAS_PER_SM = PICOSPEC_CTAS_PER_SM_BF16;
 };
 template <> struct StreamCfg<float> {
-    static constexpr int STAGES = 3;             // 3 x 32 KB in flight per CTA
+    static constexpr int STAGES = PICOSPEC_STAGES_F32;
+    static constexpr int CTAS_PER_SM = PICOSPEC_CTAS_PER_SM_F32;
 };
 template <typename T> struct TileGeom {
     static constexpr int TILE_BYTES = TILE_CHUNKS * CHUNK * (int)sizeof(T);
@@ -134,23 +150,29 @@ template <typename T> struct TileGeom {
 __device__ __forceinline__ void load_staged(ChunkRegs<__nv_bfloat16>& r, const unsigned char* chunk, int v0, int V,
                                             int lane) {
     const uint4* p = reinterpret_cast<const uint4*>(chunk) + lane;
-    const bool whole = v0 + CHUNK <= V;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-        uint4 q = p[j * 32];
-        if (!whole && v0 + j * 256 + lane * 8 >= V) q = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+        const uint4 q = p[j * 32];
         r.w[4 * j + 0] = q.x; r.w[4 * j + 1] = q.y; r.w[4 * j + 2] = q.z; r.w[4 * j + 3] = q.w;
+    }
+    if (v0 + CHUNK > V) {   // ragged last chunk of a row (warp-uniform)
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (v0 + j * 256 + lane * 8 >= V) r.w[4 * j + 0] = r.w[4 * j + 1] = r.w[4 * j + 2] = r.w[4 * j + 3] = 0xFF80FF80u;
     }
 }
 __device__ __forceinline__ void load_staged(ChunkRegs<float>& r, const unsigned char* chunk, int v0, int V, int lane) {
     const uint4* p = reinterpret_cast<const uint4*>(chunk) + lane;
-    const bool whole = v0 + CHUNK <= V;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        uint4 q = p[j * 32];
-        if (!whole && v0 + j * 128 + lane * 4 >= V) q = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
+        const uint4 q = p[j * 32];
         r.f[4 * j + 0] = __uint_as_float(q.x); r.f[4 * j + 1] = __uint_as_float(q.y);
         r.f[4 * j + 2] = __uint_as_float(q.z); r.f[4 * j + 3] = __uint_as_float(q.w);
+    }
+    if (v0 + CHUNK > V) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (v0 + j * 128 + lane * 4 >= V) r.f[4 * j + 0] = r.f[4 * j + 1] = r.f[4 * j + 2] = r.f[4 * j + 3] = -CUDART_INF_F;
     }
 }
 

@@ -135,7 +135,7 @@ struct TileDesc {
 };
 
 template <typename T>
-__global__ void __launch_bounds__(STREAM_THREADS, 2) chunk_stats_bulk_kernel(VerifyArgs a, int tiles_per_row,
+__global__ void __launch_bounds__(STREAM_THREADS, StreamCfg<T>::CTAS_PER_SM) chunk_stats_bulk_kernel(VerifyArgs a, int tiles_per_row,
                                                                              long long total_tiles) {
     extern __shared__ __align__(1024) unsigned char stage_mem[];
     constexpr int STAGES = StreamCfg<T>::STAGES;

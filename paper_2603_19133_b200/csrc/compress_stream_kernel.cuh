@@ -4,18 +4,23 @@
 // compress_filter_kernel streams the rows (one CTA per row at a time, tiles of 8 chunks staged in
 // shared memory by bulk async copies; the producer lane runs ahead into the next row) and keeps
 // every element that can still be among the k largest:
-//   - workers hold a running lower bound `thr` on the k-th largest logit of the row;
+//   - the CTA holds a running lower bound `thr` on the k-th largest logit of the row;
 //   - per chunk a lane compares the maximum of each 16-byte vector it holds with thr; vectors
 //     that reach it are parked in a per-warp ring in shared memory, and whenever 32 are parked the
-//     warp tests their elements with all lanes busy and appends the survivors (64-bit keys: logit,
-//     then lower index first) to the CTA's candidate buffer with one shared atomic per batch;
+//     warp tests their elements with all lanes busy (one element position per step, positions by
+//     ballot) and appends the survivors (64-bit keys: logit, then lower index first) to the warp's
+//     own region of the candidate buffer: no atomics with a return value, no CTA barrier;
 //   - every stored candidate is counted in a two-level histogram over the top 12 bits of the
 //     orderable logit; thr is the lower edge of the highest bin whose suffix count reaches k, so
-//     it is always a valid bound; it is refreshed after tiles 1, 2, 4, 8, ... and when the buffer
-//     fills.  The first tile of a row gets its bound from the maxima of small groups of elements;
-//   - the buffer is compacted against thr when it fills; if that is not enough an exact radix
-//     select runs; a row whose candidates still do not fit (heavy ties, adversarial order) is
-//     handed to the direct kernel through a redo list;
+//     it is a valid bound whenever it is computed, by any warp, from whatever has been counted so
+//     far.  Warp 0 refreshes it after tiles 1, 2, 4, 8, ...; a warp whose region fills refreshes
+//     it and drops its candidates below it;
+//   - the first tile of a row gets its bound without the histogram: every warp finds, by a
+//     16-step bisection over its own chunk, a value that at least ceil(k/8) of its small groups
+//     of elements reach with their maximum; the smallest of the eight values is reached by at
+//     least k elements of the tile (one CTA barrier, the only one inside a row);
+//   - a row whose candidates do not fit (heavy ties, adversarial order) is handed to the direct
+//     kernel through a redo list;
 //   - with top-p the same pass accumulates the softmax normaliser relative to the first tile's
 //     maximum (a row whose later logits overflow that reference also goes to the redo list).
 // At the end of a row the candidates at or above thr (at least k, normally k plus a few dozen) go
@@ -29,8 +34,20 @@
 
 namespace picospec {
 
-constexpr int CS_CAND_CAP = 4096;    // candidate keys held in shared memory
-constexpr int CS_SOFT = 2560;        // compaction trigger (leaves room for one tile's pushes)
+// Tunables (overridable at build time).
+#ifndef PICOSPEC_CS_CAND_CAP
+#define PICOSPEC_CS_CAND_CAP 4096
+#endif
+#ifndef PICOSPEC_CS_STAGES_BF16
+#define PICOSPEC_CS_STAGES_BF16 3
+#endif
+#ifndef PICOSPEC_CS_CTAS
+#define PICOSPEC_CS_CTAS 2
+#endif
+constexpr int CS_CAND_CAP = PICOSPEC_CS_CAND_CAP;          // candidate keys held in shared memory
+constexpr int CS_REGION = CS_CAND_CAP / WARPS;             // each worker warp appends to its own region
+constexpr int CS_REGION_SOFT = CS_REGION - CS_REGION / 4;  // a region this full is compacted against thr
+constexpr int CS_BIN_SHIFT = 20;
 constexpr int CS_BINS = 4096;        // histogram bins: top 12 bits of the orderable logit
 constexpr int CS_SUPER = CS_BINS / 32;
 constexpr int CS_QCAP = 64;          // per-warp ring of parked vectors
@@ -47,8 +64,8 @@ struct CsRowMeta {
 };
 
 template <typename T> struct CsCfg;
-template <> struct CsCfg<__nv_bfloat16> { static constexpr int STAGES = 3; };   // 3 x 16 KB
-template <> struct CsCfg<float> { static constexpr int STAGES = 2; };           // 2 x 32 KB
+template <> struct CsCfg<__nv_bfloat16> { static constexpr int STAGES = PICOSPEC_CS_STAGES_BF16; };   // x 16 KB
+template <> struct CsCfg<float> { static constexpr int STAGES = 2; };                                 // x 32 KB
 template <typename T> struct CsGeom {
     static constexpr int TILE_BYTES = TILE_CHUNKS * CHUNK * (int)sizeof(T);
     static constexpr int STAGE_BYTES = CsCfg<T>::STAGES * TILE_BYTES;
@@ -60,21 +77,19 @@ template <typename T> struct CsGeom {
 __host__ __device__ __forceinline__ int cs_survivor_cap(int k_max) { return 2 * k_max > 512 ? 2 * k_max : 512; }
 
 struct CsShared {
-    float thr;          // current lower bound on the k-th largest logit
-    int thr_bin;        // its bin
-    unsigned top_key;   // largest orderable logit seen in the row
-    int count;          // candidates appended (may run past CS_CAND_CAP: then overflow is set)
-    int overflow;
+    unsigned thr_key;   // orderable form of the current lower bound on the k-th largest logit
+    unsigned thr0_key;  // first-tile bound: minimum over the warps' own bounds
+    unsigned top_key;   // largest orderable logit of the first tile
+    int overflow;       // a region ran out of room: the row goes to the redo list
     int nan;
     int abort;          // a bounded wait ran out somewhere in the CTA
-    int m;              // scratch: survivor count
+    int m;              // survivors written at the end of the row
     double wsum[WARPS];
 };
 
-__device__ __forceinline__ int coarse_bin(float l) { return (int)(orderable(l) >> 20); }
-__device__ __forceinline__ float bin_lower_edge(int bin) {
-    // bins 0..7 hold -inf and the negative NaN patterns: no finite edge
-    return bin <= 7 ? -CUDART_INF_F : from_orderable((uint32_t)bin << 20);
+// threshold (a float) of an orderable key; keys below 0x00800000 are -inf and the negative NaN patterns
+__device__ __forceinline__ float thr_of_key(unsigned key) {
+    return key < 0x00800000u ? -CUDART_INF_F : from_orderable(key);
 }
 
 // ---- per-dtype pieces --------------------------------------------------------------------------
@@ -87,17 +102,9 @@ __device__ __forceinline__ float vec_elem(const uint4& q, int e, const __nv_bflo
 __device__ __forceinline__ float vec_elem(const uint4& q, int e, const float*) {
     return __uint_as_float(e < 2 ? (e == 0 ? q.x : q.y) : (e == 2 ? q.z : q.w));
 }
-__device__ __forceinline__ uint4 vec_words(const ChunkRegs<__nv_bfloat16>& r, int j) {
-    return make_uint4(r.w[4 * j], r.w[4 * j + 1], r.w[4 * j + 2], r.w[4 * j + 3]);
-}
-__device__ __forceinline__ uint4 vec_words(const ChunkRegs<float>& r, int j) {
-    return make_uint4(__float_as_uint(r.f[4 * j]), __float_as_uint(r.f[4 * j + 1]), __float_as_uint(r.f[4 * j + 2]),
-                      __float_as_uint(r.f[4 * j + 3]));
-}
-__device__ __forceinline__ float fmax_nan(float a, float b) { return (a != a || b != b) ? CUDART_NAN_F : fmaxf(a, b); }
 
-// Per-lane view of a chunk for the filter: which vectors may hold an element >= thr (a superset:
-// the element test decides), the lane's maximum (NaN if the lane holds a NaN).
+// Per-lane view of a chunk for the filter: a bit per vector that may hold an element >= thr (a
+// superset: the element test decides) and the lane's maximum (NaN if the lane holds a NaN).
 template <typename T> struct ChunkScan;
 template <> struct ChunkScan<__nv_bfloat16> {
     __nv_bfloat162 vmax[4];      // per vector: (max of even elements, max of odd elements)
@@ -117,13 +124,16 @@ template <> struct ChunkScan<__nv_bfloat16> {
         lane_max = __uint_as_float(*reinterpret_cast<uint32_t*>(&a) << 16);
     }
     // thr as a packed pair: the smallest bf16 >= thr when thr is negative or a bf16 itself (every
-    // threshold this kernel produces); otherwise a slightly lower value, which only adds vectors
-    static __device__ __forceinline__ uint32_t pack_thr(float thr) {
+    // threshold this kernel produces); otherwise a slightly lower value, which only adds vectors.
+    // A NaN maximum counts as a hit; the element test drops it.
+    __device__ __forceinline__ unsigned hit_mask(float thr) const {
         const uint32_t h = __float_as_uint(thr) >> 16;
-        return h | (h << 16);
-    }
-    __device__ __forceinline__ bool hit(int j, uint32_t thr2) const {
-        return !__hblt2(vmax[j], *reinterpret_cast<const __nv_bfloat162*>(&thr2));   // not (both halves < thr)
+        const uint32_t t2 = h | (h << 16);
+        const __nv_bfloat162 t = *reinterpret_cast<const __nv_bfloat162*>(&t2);
+        unsigned m = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) m |= (__hblt2(vmax[j], t) ? 0u : 1u) << j;     // not (both halves < thr)
+        return m;
     }
 };
 template <> struct ChunkScan<float> {
@@ -141,53 +151,63 @@ template <> struct ChunkScan<float> {
         }
         lane_max = nan ? CUDART_NAN_F : lm;
     }
-    static __device__ __forceinline__ uint32_t pack_thr(float thr) { return __float_as_uint(thr); }
-    __device__ __forceinline__ bool hit(int j, uint32_t thr2) const { return vmax[j] >= __uint_as_float(thr2); }
+    __device__ __forceinline__ unsigned hit_mask(float thr) const {
+        unsigned m = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) m |= (vmax[j] >= thr ? 1u : 0u) << j;
+        return m;
+    }
 };
 
+// 16-bit orderable keys of the maxima of groups of 2 consecutive elements of the lane's chunk
+// (NaN is ignored here; the lane maximum reports it).
+__device__ __forceinline__ void pair_keys(const ChunkRegs<__nv_bfloat16>& r, unsigned (&key)[16]) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k)
+        key[k] = orderable(fmaxf(__uint_as_float(r.w[k] << 16), __uint_as_float(r.w[k] & 0xffff0000u))) >> 16;
+}
+__device__ __forceinline__ void pair_keys(const ChunkRegs<float>& r, unsigned (&key)[16]) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) key[k] = orderable(fmaxf(r.f[2 * k], r.f[2 * k + 1])) >> 16;
+}
+
+// Warp-wide bisection: the largest 16-bit key t such that at least `need` of the warp's G*32 group
+// keys are >= t (the need-th largest key).  G in {4, 8, 16} keys per lane.
+template <int G>
+__device__ __forceinline__ unsigned warp_kth_key(const unsigned (&key)[16], int need) {
+    unsigned prefix = 0;
+#pragma unroll 1
+    for (int bit = 15; bit >= 0; --bit) {
+        const unsigned trial = prefix | (1u << bit);
+        int c = 0;
+#pragma unroll
+        for (int x = 0; x < G; ++x) c += key[x] >= trial ? 1 : 0;
+        if (__reduce_add_sync(0xffffffffu, c) >= need) prefix = trial;
+    }
+    return prefix;
+}
+
+// First-tile bound of one warp: group size g (elements) in {2, 4, 8 (bf16 only)}.
+template <typename T>
+__device__ __forceinline__ unsigned first_tile_key(const ChunkRegs<T>& regs, int g, int need) {
+    unsigned key[16];
+    pair_keys(regs, key);
+    if (g == 2) return warp_kth_key<16>(key, need);
+#pragma unroll
+    for (int x = 0; x < 8; ++x) key[x] = max(key[2 * x], key[2 * x + 1]);
+    if (g == 4) return warp_kth_key<8>(key, need);
+#pragma unroll
+    for (int x = 0; x < 4; ++x) key[x] = max(key[2 * x], key[2 * x + 1]);
+    return warp_kth_key<4>(key, need);
+}
+
 // two-level histogram update
-__device__ __forceinline__ void hist_add(unsigned* hist, int bin, unsigned v) {
-    atomicAdd(&hist[bin], v);
-    atomicAdd(&hist[CS_BINS + (bin >> 5)], v);
+__device__ __forceinline__ void hist_add(unsigned* hist, int bin) {
+    atomicAdd(&hist[bin], 1u);
+    atomicAdd(&hist[CS_BINS + (bin >> 5)], 1u);
 }
 
-// Count (sign = +1) or take back (sign = -1) the maxima of groups of `g` consecutive elements of
-// the lane's chunk (first tile of a row).  bf16: g in {8, 4, 2}; fp32: g in {4, 2}.
-__device__ __forceinline__ void count_group_maxima(const ChunkRegs<__nv_bfloat16>& r, int g, unsigned* hist, unsigned v) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        float m4[2];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const uint32_t w0 = r.w[4 * j + 2 * h], w1 = r.w[4 * j + 2 * h + 1];
-            const float m0 = fmax_nan(__uint_as_float(w0 << 16), __uint_as_float(w0 & 0xffff0000u));
-            const float m1 = fmax_nan(__uint_as_float(w1 << 16), __uint_as_float(w1 & 0xffff0000u));
-            if (g == 2) {
-                if (m0 == m0) hist_add(hist, coarse_bin(m0), v);
-                if (m1 == m1) hist_add(hist, coarse_bin(m1), v);
-            }
-            m4[h] = fmax_nan(m0, m1);
-            if (g == 4 && m4[h] == m4[h]) hist_add(hist, coarse_bin(m4[h]), v);
-        }
-        const float m8 = fmax_nan(m4[0], m4[1]);
-        if (g == 8 && m8 == m8) hist_add(hist, coarse_bin(m8), v);
-    }
-}
-__device__ __forceinline__ void count_group_maxima(const ChunkRegs<float>& r, int g, unsigned* hist, unsigned v) {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const float m0 = fmax_nan(r.f[4 * j], r.f[4 * j + 1]), m1 = fmax_nan(r.f[4 * j + 2], r.f[4 * j + 3]);
-        if (g == 2) {
-            if (m0 == m0) hist_add(hist, coarse_bin(m0), v);
-            if (m1 == m1) hist_add(hist, coarse_bin(m1), v);
-        } else {
-            const float m = fmax_nan(m0, m1);
-            if (m == m) hist_add(hist, coarse_bin(m), v);
-        }
-    }
-}
-
-// Warp 0: raise thr to the lower edge of the highest bin whose suffix count reaches k.
+// One warp: raise thr to the lower edge of the highest bin whose suffix count reaches k.
 __device__ __forceinline__ void refresh_threshold(const unsigned* hist, CsShared& cs, int k, int lane) {
     // level 1: lane l owns super-bins 4l .. 4l+3 (super-bin s covers bins 32 s .. 32 s + 31)
     const uint4 sv = *reinterpret_cast<const uint4*>(&hist[CS_BINS + 4 * lane]);
@@ -218,8 +238,7 @@ __device__ __forceinline__ void refresh_threshold(const unsigned* hist, CsShared
         }
     }
     // level 2: the 32 bins of super-bin s, lane l reads bin 32 s + l
-    const unsigned h = hist[32 * s + lane];
-    unsigned bs = h;
+    unsigned bs = hist[32 * s + lane];
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
         const unsigned y = __shfl_down_sync(0xffffffffu, bs, d);
@@ -227,64 +246,35 @@ __device__ __forceinline__ void refresh_threshold(const unsigned* hist, CsShared
     }
     const unsigned hit2 = __ballot_sync(0xffffffffu, above + bs >= (unsigned)k);
     const int found = hit2 ? 32 * s + (31 - __clz(hit2)) : 32 * s;
-    if (lane == 0 && found > cs.thr_bin) {
-        cs.thr_bin = found;
-        cs.thr = bin_lower_edge(found);
-    }
+    if (lane == 0) atomicMax(&cs.thr_key, (unsigned)found << CS_BIN_SHIFT);
 }
 
-// Drop the candidates below thr (all 256 workers).  Survivors go to `dst` (shared or global; may be
-// `cand` itself), at most dst_cap of them are written.  Returns how many there are.
-__device__ __forceinline__ int compact_candidates(const u64* cand, int n, u64* dst, int dst_cap, CsShared& cs) {
-    constexpr int PER = CS_CAND_CAP / THREADS;
-    const int tid = threadIdx.x;
-    const uint32_t thr_key = orderable(cs.thr);
-    u64 mine[PER];
-#pragma unroll
-    for (int e = 0; e < PER; ++e) {
-        const int i = tid + e * THREADS;
-        mine[e] = i < n ? cand[i] : 0ull;
+// Warp-local: drop the entries of this warp's region below thr (stable, in place).
+__device__ __forceinline__ int compact_region(u64* region, int n, unsigned thr_key, int lane) {
+    int out = 0;
+    for (int base = 0; base < n; base += 32) {
+        const int i = base + lane;
+        const u64 key = i < n ? region[i] : 0ull;
+        const bool keep = i < n && (unsigned)(key >> 32) >= thr_key;
+        const unsigned m = __ballot_sync(0xffffffffu, keep);
+        if (keep) region[out + __popc(m & ((1u << lane) - 1u))] = key;
+        out += __popc(m);
     }
-    if (tid == 0) cs.m = 0;
-    workers_sync();
-    int cnt = 0;
-#pragma unroll
-    for (int e = 0; e < PER; ++e) cnt += (mine[e] != 0ull && (uint32_t)(mine[e] >> 32) >= thr_key) ? 1 : 0;
-    const int lane = tid & 31;
-    int incl = cnt;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const int y = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += y;
-    }
-    const int total = __shfl_sync(0xffffffffu, incl, 31);
-    int base = 0;
-    if (lane == 0 && total) base = atomicAdd(&cs.m, total);
-    base = __shfl_sync(0xffffffffu, base, 0);
-    int pos = base + incl - cnt;
-#pragma unroll
-    for (int e = 0; e < PER; ++e)
-        if (mine[e] != 0ull && (uint32_t)(mine[e] >> 32) >= thr_key) {
-            if (pos < dst_cap) dst[pos] = mine[e];
-            ++pos;
-        }
-    workers_sync();
-    return cs.m;
+    __syncwarp();
+    return out;
 }
 
 template <typename T, bool STATS>
-__global__ void __launch_bounds__(STREAM_THREADS, 2) compress_filter_kernel(CompressArgs a, int tiles_per_row) {
+__global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_filter_kernel(CompressArgs a, int tiles_per_row) {
     extern __shared__ __align__(1024) unsigned char dyn[];
     constexpr int STAGES = CsCfg<T>::STAGES;
     constexpr int TILE_BYTES = CsGeom<T>::TILE_BYTES;
     constexpr int VEC = ChunkRegs<T>::VEC, NVEC = ChunkRegs<T>::NVEC;
-    constexpr bool LOGIT16 = sizeof(T) == 2;
     unsigned char* stage_mem = dyn;
     u64* cand = reinterpret_cast<u64*>(dyn + CsGeom<T>::STAGE_BYTES);
     unsigned* hist = reinterpret_cast<unsigned*>(cand + CS_CAND_CAP);          // bins, then super-bins
     unsigned char* qmem = reinterpret_cast<unsigned char*>(hist + CS_BINS + CS_SUPER);
     __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES];
-    __shared__ CompressShared sh;
     __shared__ CsShared cs;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -304,13 +294,13 @@ __global__ void __launch_bounds__(STREAM_THREADS, 2) compress_filter_kernel(Comp
             *a.queue_count_next = 0;
             *a.redo_count_next = 0;
         }
-        cs.thr = -CUDART_INF_F;
-        cs.thr_bin = 0;
+        cs.thr_key = 0u;
+        cs.thr0_key = 0xffffffffu;
         cs.top_key = 0u;
-        cs.count = 0;
         cs.overflow = 0;
         cs.nan = 0;
         cs.abort = 0;
+        cs.m = 0;
     }
     for (int i = tid; i < CS_BINS + CS_SUPER; i += STREAM_THREADS) hist[i] = 0u;
     __syncthreads();
@@ -347,10 +337,12 @@ __global__ void __launch_bounds__(STREAM_THREADS, 2) compress_filter_kernel(Comp
     // ---- workers ------------------------------------------------------------------------------
     uint4* qvec = reinterpret_cast<uint4*>(qmem) + warp * CS_QCAP;
     int* qidx = reinterpret_cast<int*>(qmem + WARPS * CS_QCAP * 16) + warp * CS_QCAP;
+    u64* region = cand + warp * CS_REGION;
     const unsigned lt_mask = (1u << lane) - 1u;
-    // group size of the first-tile bound: at least 4 k groups in the tile
+    // first-tile bound: groups of g elements, at least 4 k groups in the tile
     int g = VEC;
     while (g > 2 && (TILE_CHUNKS * CHUNK) / g < 4 * k_eff) g >>= 1;
+    const int need = (k_eff + WARPS - 1) / WARPS;
 
     bool dead = false;      // this warp stopped waiting on copies; it still joins every barrier
     uint32_t i = 0;
@@ -360,52 +352,43 @@ __global__ void __launch_bounds__(STREAM_THREADS, 2) compress_filter_kernel(Comp
         const bool valid = temp_ok(Tb);
         const float c32 = temp_scale(Tb);
         float ref_off = 0.f, acc = 0.f;
-        int qhead = 0, qn = 0;
-        bool skip = false;   // row overflowed: consume its tiles without work
+        int qhead = 0, qn = 0;      // ring of parked vectors
+        int wcount = 0;             // candidates in this warp's region
+        bool full_region = false;   // the region ran out of room (row goes to the redo list)
 
-        // tests up to 32 parked vectors with all lanes busy and appends the survivors
+        // Tests up to 32 parked vectors, one element position per step with every lane on its own
+        // vector, and appends the survivors to the warp's region.
         auto drain = [&](int n) {
-            const bool active = lane < n;
             const int slot = (qhead + lane) & (CS_QCAP - 1);
             uint4 q = make_uint4(0, 0, 0, 0);
             int vb = a.V;
-            if (active) {
+            if (lane < n) {
                 q = qvec[slot];
                 vb = qidx[slot];
             }
-            const float thr = *(volatile float*)&cs.thr;
-            unsigned pass = 0;
-            if (vb < a.V) {
+            const bool active = vb < a.V;
+            const float thr = thr_of_key(*(volatile unsigned*)&cs.thr_key);
+            const int before = wcount;
 #pragma unroll
-                for (int e = 0; e < VEC; ++e)
-                    if (vec_elem(q, e, (const T*)nullptr) >= thr) pass |= 1u << e;
-            }
-            const int cnt = __popc(pass);
-            int incl = cnt;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int y = __shfl_up_sync(0xffffffffu, incl, d);
-                if (lane >= d) incl += y;
-            }
-            const int total = __shfl_sync(0xffffffffu, incl, 31);
-            if (total) {
-                int base = 0;
-                if (lane == 0) base = atomicAdd(&cs.count, total);
-                base = __shfl_sync(0xffffffffu, base, 0);
-                int pos = base + incl - cnt;
-                while (pass) {
-                    const int e = __ffs(pass) - 1;
-                    pass &= pass - 1;
-                    if (pos < CS_CAND_CAP) {
-                        const float l = vec_elem(q, e, (const T*)nullptr);
-                        cand[pos] = make_key(l, vb + e);
-                        hist_add(hist, coarse_bin(l), 1u);
-                    } else {
-                        cs.overflow = 1;
-                    }
-                    ++pos;
+            for (int e = 0; e < VEC; ++e) {
+                const float l = vec_elem(q, e, (const T*)nullptr) + 0.0f;     // -0 becomes +0
+                const bool p = active && l >= thr;
+                const unsigned m = __ballot_sync(0xffffffffu, p);
+                const int pos = wcount + __popc(m & lt_mask);
+                if (p && pos < CS_REGION) {
+                    const uint32_t bits = __float_as_uint(l);
+                    const uint32_t okey = bits ^ ((uint32_t)((int32_t)bits >> 31) | 0x80000000u);
+                    region[pos] = ((u64)okey << 32) | (u64)(~(uint32_t)(vb + e));
                 }
+                wcount += __popc(m);
             }
+            if (wcount > CS_REGION) {
+                full_region = true;
+                wcount = CS_REGION;
+            }
+            __syncwarp();
+            // count the new entries in the histogram
+            for (int x = before + lane; x < wcount; x += 32) hist_add(hist, (int)(region[x] >> (32 + CS_BIN_SHIFT)));
             qhead = (qhead + n) & (CS_QCAP - 1);
             qn -= n;
             __syncwarp();       // the slots just read may be refilled
@@ -422,131 +405,93 @@ __global__ void __launch_bounds__(STREAM_THREADS, 2) compress_filter_kernel(Comp
                 }
             }
             const int c = ti * TILE_CHUNKS + warp;
-            const bool work = !dead && valid && !skip && c < a.nch;
+            const bool work = !dead && valid && !full_region && c < a.nch;
+            const unsigned char* chunk = stage_mem + s * TILE_BYTES + warp * (CHUNK * (int)sizeof(T));
             ChunkRegs<T> regs;
-            if (work) load_staged(regs, stage_mem + s * TILE_BYTES + warp * (CHUNK * (int)sizeof(T)), c * CHUNK, a.V, lane);
-            __syncwarp();
-            if (lane == 0 && !dead) mbar_arrive(&empty[s]);
-
             ChunkScan<T> sc;
             if (work) {
+                load_staged(regs, chunk, c * CHUNK, a.V, lane);
                 sc.scan(regs);
                 if (sc.lane_max != sc.lane_max) cs.nan = 1;
             }
             if (ti == 0 && valid) {
-                // first tile (every warp holds a full chunk): bound from the maxima of groups of g
-                // elements, counted in the histogram for the scan and taken back afterwards
+                // first tile (every warp holds a full chunk): each warp's own bound, then the minimum
                 if (work) {
-                    count_group_maxima(regs, g, hist, 1u);
+                    const unsigned k16 = first_tile_key(regs, g, need);
                     const float wm = warp_max(sc.lane_max);      // NaN lanes are ignored here
-                    if (lane == 0 && wm == wm) atomicMax(&cs.top_key, orderable(wm));
+                    if (lane == 0) {
+                        atomicMin(&cs.thr0_key, k16 << 16);
+                        if (STATS && wm == wm) atomicMax(&cs.top_key, orderable(wm));
+                    }
                 }
                 workers_sync();
-                if (warp == 0) refresh_threshold(hist, cs, k_eff, lane);
+                if (lane == 0) atomicMax(&cs.thr_key, *(volatile unsigned*)&cs.thr0_key);
                 if (STATS) ref_off = __fmul_rn(from_orderable(*(volatile unsigned*)&cs.top_key), c32);
-                workers_sync();
-                if (work) count_group_maxima(regs, g, hist, 0xffffffffu);
-            } else if (work) {
-                const unsigned lk = orderable(sc.lane_max);      // NaN maps above every number: harmless
-                if (sc.lane_max == sc.lane_max && lk > *(volatile unsigned*)&cs.top_key) atomicMax(&cs.top_key, lk);
+                __syncwarp();
             }
             if (work) {
                 if (STATS) acc += lane_exp_sum2(regs, c32, ref_off);
-                const uint32_t thr2 = ChunkScan<T>::pack_thr(*(volatile float*)&cs.thr);
-                const int v0 = c * CHUNK;
-#pragma unroll
+                const unsigned hits = sc.hit_mask(thr_of_key(*(volatile unsigned*)&cs.thr_key));
+                const int v0 = c * CHUNK + lane * VEC;
+                // warp 0 empties its ring before it refreshes the bound (after tiles 1, 2, 4, 8, ...)
+                const bool refresh_due = warp == 0 && ((ti + 1) & ti) == 0;
+                const int batch = refresh_due ? 1 : 32;
+#pragma unroll 1
                 for (int j = 0; j < NVEC; ++j) {
-                    const bool hit = sc.hit(j, thr2);
+                    const bool hit = (hits >> j) & 1u;
                     const unsigned m = __ballot_sync(0xffffffffu, hit);
-                    if (m) {
-                        if (hit) {
-                            const int slot = (qhead + qn + __popc(m & lt_mask)) & (CS_QCAP - 1);
-                            qvec[slot] = vec_words(regs, j);
-                            qidx[slot] = v0 + j * (32 * VEC) + lane * VEC;
-                        }
-                        qn += __popc(m);
-                        __syncwarp();
-                        if (qn >= 32) drain(32);
+                    if (m == 0u) continue;
+                    if (hit) {
+                        const int slot = (qhead + qn + __popc(m & lt_mask)) & (CS_QCAP - 1);
+                        qvec[slot] = reinterpret_cast<const uint4*>(chunk)[j * 32 + lane];
+                        qidx[slot] = v0 + j * (32 * VEC);
                     }
+                    qn += __popc(m);
+                    __syncwarp();
+                    if (qn >= batch) drain(min(qn, 32));
+                }
+                if (refresh_due) refresh_threshold(hist, cs, k_eff, lane);
+                if (wcount > CS_REGION_SOFT) {
+                    // region nearly full: bring the bound up to date and drop what fell below it
+                    refresh_threshold(hist, cs, k_eff, lane);
+                    __syncwarp();
+                    wcount = compact_region(region, wcount, *(volatile unsigned*)&cs.thr_key, lane);
+                    if (wcount > CS_REGION_SOFT) full_region = true;    // ties or a coarse bin too full
                 }
             }
-            const bool last = ti + 1 == tiles_per_row;
-            const bool refresh_due = last || ((ti + 1) & ti) == 0;     // after tiles 1, 2, 4, 8, ...
-            if (refresh_due && qn > 0) drain(qn);      // the histogram must be complete for a refresh
-
-            // ---- tile boundary ----------------------------------------------------------------
-            // One barrier that also ORs every warp's view of "the buffer needs attention".  The
-            // counters only grow while warps push, and the last warp to arrive sees their final
-            // values, so the OR is the same decision for everybody.
-            const bool attention = workers_sync_or(*(volatile int*)&cs.count > CS_SOFT ||
-                                                   *(volatile int*)&cs.overflow != 0 ||
-                                                   *(volatile int*)&cs.abort != 0);
-            if (attention) {
-                if (qn > 0) drain(qn);
-                workers_sync();                     // all pushes are in
-                int n = *(volatile int*)&cs.count;
-                const bool ovf = *(volatile int*)&cs.overflow != 0;
-                if (*(volatile int*)&cs.abort) dead = true;
-                workers_sync();                     // everybody has read the counters
-                if (valid && !skip) {
-                    if (ovf) {
-                        skip = true;
-                    } else {
-                        if (warp == 0) refresh_threshold(hist, cs, k_eff, lane);
-                        workers_sync();
-                        if (n > CS_SOFT && !last) {
-                            n = compact_candidates(cand, n, cand, CS_CAND_CAP, cs);
-                            if (n > CS_SOFT) {
-                                // ties or a coarse bin too full: exact selection of the k best so far
-                                const u64 kth = keep_top_k<LOGIT16>(cand, reinterpret_cast<u64*>(qmem), n, k_eff, sh);
-                                n = k_eff;
-                                if (tid == 0) {
-                                    const float tl = key_logit(kth);
-                                    if (tl > cs.thr) {
-                                        cs.thr = tl;
-                                        cs.thr_bin = coarse_bin(tl);
-                                    }
-                                }
-                            }
-                            if (tid == 0) cs.count = n;
-                            workers_sync();
-                        }
-                    }
-                }
-            } else if (refresh_due && valid && !skip) {
-                if (warp == 0) refresh_threshold(hist, cs, k_eff, lane);
-                workers_sync();
-            }
+            __syncwarp();
+            if (lane == 0 && !dead) mbar_arrive(&empty[s]);     // the stage is free again
         }
 
         // ---- row end: survivors and row statistics to global scratch -----------------------------
+        while (qn > 0 && !full_region && !dead) drain(min(qn, 32));
+        if (lane == 0 && full_region) cs.overflow = 1;
         if (STATS) {
             const double sw = (double)warp_sum(acc);
             if (lane == 0) cs.wsum[warp] = sw;
         }
         workers_sync();
-        int flags = 0;
-        int m = 0;
-        if (dead || *(volatile int*)&cs.abort) {
-            flags = CSF_ABORT;
-        } else if (!valid) {
-            flags = CSF_TEMPERATURE;
-        } else if (skip || *(volatile int*)&cs.overflow) {
-            flags = CSF_REDO;
-        } else {
+        const bool row_ok = valid && !*(volatile int*)&cs.overflow && !*(volatile int*)&cs.abort;
+        if (row_ok && warp == 0) refresh_threshold(hist, cs, k_eff, lane);
+        workers_sync();
+        if (row_ok) {
+            // every warp filters its own region and appends to the row's scratch area
             u64* dst = a.surv_keys + (long long)row * surv_cap;
-            const int n = cs.count;
-            m = compact_candidates(cand, n, dst, surv_cap, cs);
-            if (m > surv_cap) {
-                // too many ties at the bound for the scratch area: exact selection here
-                m = compact_candidates(cand, n, cand, CS_CAND_CAP, cs);
-                keep_top_k<LOGIT16>(cand, reinterpret_cast<u64*>(qmem), m, k_eff, sh);
-                for (int x = tid; x < k_eff; x += THREADS) dst[x] = cand[x];
-                m = k_eff;
-            }
-            if (cs.nan || m < k_eff) flags = CSF_LOGIT;
+            const int n = compact_region(region, wcount, *(volatile unsigned*)&cs.thr_key, lane);
+            int base = 0;
+            if (lane == 0 && n) base = atomicAdd(&cs.m, n);
+            base = __shfl_sync(0xffffffffu, base, 0);
+            for (int x = lane; x < n; x += 32)
+                if (base + x < surv_cap) dst[base + x] = region[x];
         }
+        workers_sync();
         if (tid == 0) {
+            int flags = 0;
+            const int m = cs.m;
+            if (cs.abort) flags = CSF_ABORT;
+            else if (!valid) flags = CSF_TEMPERATURE;
+            else if (cs.overflow || m > surv_cap) flags = CSF_REDO;      // too many candidates or ties at the bound
+            else if (cs.nan || m < k_eff) flags = CSF_LOGIT;
             double zs = 0.0;
             if (STATS)
                 for (int w = 0; w < WARPS; ++w) zs += cs.wsum[w];
@@ -560,18 +505,15 @@ __global__ void __launch_bounds__(STREAM_THREADS, 2) compress_filter_kernel(Comp
             meta.pad = 0.f;
             meta.z_stream = zs;
             a.surv_meta[row] = meta;
-        }
-        workers_sync();
-        // reset the row state
-        for (int x = tid; x < CS_BINS + CS_SUPER; x += THREADS) hist[x] = 0u;
-        if (tid == 0) {
-            cs.thr = -CUDART_INF_F;
-            cs.thr_bin = 0;
+            // reset the row state
+            cs.thr_key = 0u;
+            cs.thr0_key = 0xffffffffu;
             cs.top_key = 0u;
-            cs.count = 0;
             cs.overflow = 0;
             cs.nan = 0;
+            cs.m = 0;
         }
+        for (int x = tid; x < CS_BINS + CS_SUPER; x += THREADS) hist[x] = 0u;
         workers_sync();
     }
 }

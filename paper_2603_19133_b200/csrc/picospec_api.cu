@@ -135,7 +135,13 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
         cudaError_t ea = ensure_kernel_attrs(ctx->device);
         if (ea != cudaSuccess) return ea;
         const int tiles_per_row = (a.nch + TILE_CHUNKS - 1) / TILE_CHUNKS;
-        const int per_sm = CsGeom<T>::SMEM_BYTES > 110 * 1024 ? 1 : 2;
+        int per_sm = 1;     // resident CTAs per SM for this kernel's registers and shared memory
+        cudaError_t eo = stats ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_filter_kernel<T, true>,
+                                                                             STREAM_THREADS, CsGeom<T>::SMEM_BYTES)
+                               : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_filter_kernel<T, false>,
+                                                                             STREAM_THREADS, CsGeom<T>::SMEM_BYTES);
+        if (eo != cudaSuccess) return eo;
+        if (per_sm < 1) per_sm = 1;
         const int g = rows < ctx->num_sms * per_sm ? rows : ctx->num_sms * per_sm;
         {
             ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_STREAM, 1, s);

@@ -9,7 +9,7 @@
 namespace picospec {
 
 constexpr unsigned ST_INTERNAL = 8u;          // a bounded wait ran out (mirrors picospec.h)
-constexpr uint32_t WAIT_SPINS = 1u << 22;     // polls before a wait gives up (of the order of a second)
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after two seconds
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -36,13 +36,31 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// false: the limit ran out
+// the same with a suspend-time hint (ns): the thread may sleep in hardware instead of polling
+__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// false: the time limit ran out
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    for (uint32_t i = 0; i < WAIT_SPINS; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (i >= 32) __nanosleep(i < 4096 ? 32 : 256);
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try_wait_hint(bar, parity, 20000u)) return true;
+        if ((i & 7u) == 0u && global_ns() - t0 > WAIT_LIMIT_NS) return false;
     }
-    return false;
 }
 
 __device__ __forceinline__ uint64_t l2_evict_first_policy() {

@@ -211,20 +211,20 @@ template <typename T> __device__ __forceinline__ float lane_exp_sum(const ChunkR
     return (a0 + a1) + (a2 + a3);
 }
 
-// Double-precision weight of one logit in the definition's own terms: exp(l/T - row_max/T).
+// Double-precision weight of one logit: exp(l * (1/T) - row_max * (1/T)) (the definition's
+// exp(l/T - max/T) with the division replaced by one multiplication: 2^-53 relative per term).
 // The fp32 streaming pass sums 2^(l*c32 - off) with c32 = fp32(log2 e / T) and
 // off = fp32(row_max * c32); stream_sum_scale() is the exact factor 2^(off - row_max*c32) that
 // brings such a sum onto the scale of these weights (what remains is the bounded error GUARD_Z).
-// PRECISE divides by T as the definition does; the fast variant multiplies by 1/T.
+// The fast path and the double-precision re-evaluation use the same weights; they differ in
+// where the normaliser comes from.
 template <bool PRECISE> struct Weight {
     double t, m;
     __device__ __forceinline__ void init(float T, float row_max) {
-        t = PRECISE ? (double)T : 1.0 / (double)T;
-        m = PRECISE ? (double)row_max / (double)T : (double)row_max * t;
+        t = 1.0 / (double)T;
+        m = (double)row_max * t;
     }
-    __device__ __forceinline__ double operator()(float l) const {
-        return PRECISE ? exp((double)l / t - m) : exp((double)l * t - m);
-    }
+    __device__ __forceinline__ double operator()(float l) const { return exp((double)l * t - m); }
 };
 __device__ __forceinline__ double stream_sum_scale(float row_max, float c32) {
     return exp2((double)__fmul_rn(row_max, c32) - (double)row_max * (double)c32);

@@ -159,11 +159,18 @@ __device__ u64 keep_top_k(u64* cand, u64* keep, int count, int k, CompressShared
     return kth;
 }
 
-// Descending bitonic sort of keys[0..n2), n2 a power of two.
+// Descending bitonic sort of keys[0..n2), n2 a power of two, by the 256 workers.  Thread t takes the
+// compare-exchange pairs t, t + 256, ...; with a stride of at most 32 the 32 pairs of a warp
+// stay inside one aligned block of 64 keys that no other warp touches in that stage, so those stages
+// only need a warp-level sync; a CTA barrier separates them from the stages with longer strides.
 __device__ void bitonic_sort_desc(u64* keys, int n2) {
+    bool cross = true;      // the previous stage (or the caller's writes) crossed warp blocks
     for (int size = 2; size <= n2; size <<= 1) {
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            workers_sync();
+            const bool local = stride <= 32;
+            if (!local || cross) workers_sync();
+            else __syncwarp();
+            cross = !local;
             for (int i = threadIdx.x; i < (n2 >> 1); i += THREADS) {
                 const int pos = 2 * i - (i & (stride - 1));
                 const int j = pos + stride;

@@ -171,18 +171,25 @@ __device__ __forceinline__ void pair_keys(const ChunkRegs<float>& r, unsigned (&
     for (int k = 0; k < 16; ++k) key[k] = orderable(fmaxf(r.f[2 * k], r.f[2 * k + 1])) >> 16;
 }
 
-// Warp-wide bisection: the largest 16-bit key t such that at least `need` of the warp's G*32 group
-// keys are >= t (the need-th largest key).  G in {4, 8, 16} keys per lane.
+// Warp-wide search, two bits per step: the largest 16-bit key t such that at least `need` of the
+// warp's G*32 group keys are >= t (the need-th largest key).  G in {4, 8, 16} keys per lane.
 template <int G>
 __device__ __forceinline__ unsigned warp_kth_key(const unsigned (&key)[16], int need) {
     unsigned prefix = 0;
 #pragma unroll 1
-    for (int bit = 15; bit >= 0; --bit) {
-        const unsigned trial = prefix | (1u << bit);
-        int c = 0;
+    for (int bit = 14; bit >= 0; bit -= 2) {
+        const unsigned t1 = prefix | (1u << bit), t2 = prefix | (2u << bit), t3 = prefix | (3u << bit);
+        int c1 = 0, c2 = 0, c3 = 0;
 #pragma unroll
-        for (int x = 0; x < G; ++x) c += key[x] >= trial ? 1 : 0;
-        if (__reduce_add_sync(0xffffffffu, c) >= need) prefix = trial;
+        for (int x = 0; x < G; ++x) {
+            c1 += key[x] >= t1 ? 1 : 0;
+            c2 += key[x] >= t2 ? 1 : 0;
+            c3 += key[x] >= t3 ? 1 : 0;
+        }
+        c1 = __reduce_add_sync(0xffffffffu, c1);
+        c2 = __reduce_add_sync(0xffffffffu, c2);
+        c3 = __reduce_add_sync(0xffffffffu, c3);
+        prefix = c3 >= need ? t3 : c2 >= need ? t2 : c1 >= need ? t1 : prefix;
     }
     return prefix;
 }
@@ -264,6 +271,74 @@ __device__ __forceinline__ int compact_region(u64* region, int n, unsigned thr_k
     return out;
 }
 
+__device__ __forceinline__ uint4 vec_words(const ChunkRegs<__nv_bfloat16>& r, int j) {
+    return make_uint4(r.w[4 * j], r.w[4 * j + 1], r.w[4 * j + 2], r.w[4 * j + 3]);
+}
+__device__ __forceinline__ uint4 vec_words(const ChunkRegs<float>& r, int j) {
+    return make_uint4(__float_as_uint(r.f[4 * j]), __float_as_uint(r.f[4 * j + 1]), __float_as_uint(r.f[4 * j + 2]),
+                      __float_as_uint(r.f[4 * j + 3]));
+}
+
+// Per-warp filter state kept in registers.
+struct WarpQ {
+    int qhead, qn;      // ring of parked vectors
+    int wcount;         // candidates in this warp's region
+    int full;           // the region ran out of room (the row goes to the redo list)
+};
+
+// Tests up to 32 parked vectors, one element position per step with every lane on its own vector,
+// and appends the survivors to the warp's region.  Not inlined: it is called from several places of
+// the hot loop, which has to stay small.  Offsets are bytes into the kernel's dynamic shared memory.
+template <typename T>
+__device__ __noinline__ WarpQ drain_parked(WarpQ st, int n, int qvec_off, int qidx_off, int region_off, int hist_off,
+                                           unsigned thr_key, int V) {
+    extern __shared__ __align__(1024) unsigned char dyn[];
+    constexpr int VEC = ChunkRegs<T>::VEC;
+    const int lane = threadIdx.x & 31;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    const uint4* qvec = reinterpret_cast<const uint4*>(dyn + qvec_off);
+    const int* qidx = reinterpret_cast<const int*>(dyn + qidx_off);
+    u64* region = reinterpret_cast<u64*>(dyn + region_off);
+    unsigned* hist = reinterpret_cast<unsigned*>(dyn + hist_off);
+    const int slot = (st.qhead + lane) & (CS_QCAP - 1);
+    uint4 q = make_uint4(0, 0, 0, 0);
+    int vb = V;
+    __syncwarp();       // the other lanes' parked vectors are visible
+    if (lane < n) {
+        q = qvec[slot];
+        vb = qidx[slot];
+    }
+    const bool active = vb < V;
+    const float thr = thr_of_key(thr_key);
+    const int before = st.wcount;
+    int wcount = st.wcount;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+        const float l = vec_elem(q, e, (const T*)nullptr) + 0.0f;     // -0 becomes +0
+        const bool p = active && l >= thr;
+        const unsigned m = __ballot_sync(0xffffffffu, p);
+        const int pos = wcount + __popc(m & lt_mask);
+        if (p && pos < CS_REGION) {
+            const uint32_t bits = __float_as_uint(l);
+            const uint32_t okey = bits ^ ((uint32_t)((int32_t)bits >> 31) | 0x80000000u);
+            region[pos] = ((u64)okey << 32) | (u64)(~(uint32_t)(vb + e));
+        }
+        wcount += __popc(m);
+    }
+    if (wcount > CS_REGION) {
+        st.full = 1;
+        wcount = CS_REGION;
+    }
+    __syncwarp();
+    // count the new entries in the histogram
+    for (int x = before + lane; x < wcount; x += 32) hist_add(hist, (int)(region[x] >> (32 + CS_BIN_SHIFT)));
+    st.wcount = wcount;
+    st.qhead = (st.qhead + n) & (CS_QCAP - 1);
+    st.qn -= n;
+    __syncwarp();       // the slots just read may be refilled
+    return st;
+}
+
 template <typename T, bool STATS>
 __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_filter_kernel(CompressArgs a, int tiles_per_row) {
     extern __shared__ __align__(1024) unsigned char dyn[];
@@ -339,6 +414,10 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
     int* qidx = reinterpret_cast<int*>(qmem + WARPS * CS_QCAP * 16) + warp * CS_QCAP;
     u64* region = cand + warp * CS_REGION;
     const unsigned lt_mask = (1u << lane) - 1u;
+    const int qvec_off = (int)(reinterpret_cast<unsigned char*>(qvec) - dyn);
+    const int qidx_off = (int)(reinterpret_cast<unsigned char*>(qidx) - dyn);
+    const int region_off = (int)(reinterpret_cast<unsigned char*>(region) - dyn);
+    const int hist_off = (int)(reinterpret_cast<unsigned char*>(hist) - dyn);
     // first-tile bound: groups of g elements, at least 4 k groups in the tile
     int g = VEC;
     while (g > 2 && (TILE_CHUNKS * CHUNK) / g < 4 * k_eff) g >>= 1;
@@ -352,47 +431,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
         const bool valid = temp_ok(Tb);
         const float c32 = temp_scale(Tb);
         float ref_off = 0.f, acc = 0.f;
-        int qhead = 0, qn = 0;      // ring of parked vectors
-        int wcount = 0;             // candidates in this warp's region
-        bool full_region = false;   // the region ran out of room (row goes to the redo list)
-
-        // Tests up to 32 parked vectors, one element position per step with every lane on its own
-        // vector, and appends the survivors to the warp's region.
-        auto drain = [&](int n) {
-            const int slot = (qhead + lane) & (CS_QCAP - 1);
-            uint4 q = make_uint4(0, 0, 0, 0);
-            int vb = a.V;
-            if (lane < n) {
-                q = qvec[slot];
-                vb = qidx[slot];
-            }
-            const bool active = vb < a.V;
-            const float thr = thr_of_key(*(volatile unsigned*)&cs.thr_key);
-            const int before = wcount;
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) {
-                const float l = vec_elem(q, e, (const T*)nullptr) + 0.0f;     // -0 becomes +0
-                const bool p = active && l >= thr;
-                const unsigned m = __ballot_sync(0xffffffffu, p);
-                const int pos = wcount + __popc(m & lt_mask);
-                if (p && pos < CS_REGION) {
-                    const uint32_t bits = __float_as_uint(l);
-                    const uint32_t okey = bits ^ ((uint32_t)((int32_t)bits >> 31) | 0x80000000u);
-                    region[pos] = ((u64)okey << 32) | (u64)(~(uint32_t)(vb + e));
-                }
-                wcount += __popc(m);
-            }
-            if (wcount > CS_REGION) {
-                full_region = true;
-                wcount = CS_REGION;
-            }
-            __syncwarp();
-            // count the new entries in the histogram
-            for (int x = before + lane; x < wcount; x += 32) hist_add(hist, (int)(region[x] >> (32 + CS_BIN_SHIFT)));
-            qhead = (qhead + n) & (CS_QCAP - 1);
-            qn -= n;
-            __syncwarp();       // the slots just read may be refilled
-        };
+        WarpQ st = {0, 0, 0, 0};
 
         for (int ti = 0; ti < tiles_per_row; ++ti, ++i) {
             const int s = (int)(i % STAGES);
@@ -405,12 +444,13 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
                 }
             }
             const int c = ti * TILE_CHUNKS + warp;
-            const bool work = !dead && valid && !full_region && c < a.nch;
-            const unsigned char* chunk = stage_mem + s * TILE_BYTES + warp * (CHUNK * (int)sizeof(T));
+            const bool work = !dead && valid && !st.full && c < a.nch;
             ChunkRegs<T> regs;
+            if (work) load_staged(regs, stage_mem + s * TILE_BYTES + warp * (CHUNK * (int)sizeof(T)), c * CHUNK, a.V, lane);
+            __syncwarp();
+            if (lane == 0 && !dead) mbar_arrive(&empty[s]);     // the chunk is in registers: the stage is free
             ChunkScan<T> sc;
             if (work) {
-                load_staged(regs, chunk, c * CHUNK, a.V, lane);
                 sc.scan(regs);
                 if (sc.lane_max != sc.lane_max) cs.nan = 1;
             }
@@ -430,42 +470,43 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
                 __syncwarp();
             }
             if (work) {
+                const unsigned thr_key = *(volatile unsigned*)&cs.thr_key;
+                const unsigned hits = sc.hit_mask(thr_of_key(thr_key));
+                unsigned mj[NVEC];
+#pragma unroll
+                for (int j = 0; j < NVEC; ++j) mj[j] = __ballot_sync(0xffffffffu, (hits >> j) & 1u);
                 if (STATS) acc += lane_exp_sum2(regs, c32, ref_off);
-                const unsigned hits = sc.hit_mask(thr_of_key(*(volatile unsigned*)&cs.thr_key));
                 const int v0 = c * CHUNK + lane * VEC;
-                // warp 0 empties its ring before it refreshes the bound (after tiles 1, 2, 4, 8, ...)
-                const bool refresh_due = warp == 0 && ((ti + 1) & ti) == 0;
-                const int batch = refresh_due ? 1 : 32;
-#pragma unroll 1
+#pragma unroll
                 for (int j = 0; j < NVEC; ++j) {
-                    const bool hit = (hits >> j) & 1u;
-                    const unsigned m = __ballot_sync(0xffffffffu, hit);
-                    if (m == 0u) continue;
-                    if (hit) {
-                        const int slot = (qhead + qn + __popc(m & lt_mask)) & (CS_QCAP - 1);
-                        qvec[slot] = reinterpret_cast<const uint4*>(chunk)[j * 32 + lane];
+                    if (mj[j] == 0u) continue;
+                    if (st.qn >= 32) st = drain_parked<T>(st, 32, qvec_off, qidx_off, region_off, hist_off, thr_key, a.V);
+                    if ((hits >> j) & 1u) {
+                        const int slot = (st.qhead + st.qn + __popc(mj[j] & lt_mask)) & (CS_QCAP - 1);
+                        qvec[slot] = vec_words(regs, j);
                         qidx[slot] = v0 + j * (32 * VEC);
                     }
-                    qn += __popc(m);
-                    __syncwarp();
-                    if (qn >= batch) drain(min(qn, 32));
+                    st.qn += __popc(mj[j]);
                 }
-                if (refresh_due) refresh_threshold(hist, cs, k_eff, lane);
-                if (wcount > CS_REGION_SOFT) {
+                __syncwarp();
+                if (st.qn >= 32) st = drain_parked<T>(st, 32, qvec_off, qidx_off, region_off, hist_off, thr_key, a.V);
+                // the bound is refreshed after tiles 1, 2, 4, 8, ..., each time by another warp (vectors
+                // still parked in the rings are not counted yet, which only makes it a little lower)
+                if (((ti + 1) & ti) == 0 && warp == ((31 - __clz(ti + 1)) & (WARPS - 1))) refresh_threshold(hist, cs, k_eff, lane);
+                if (st.wcount > CS_REGION_SOFT) {
                     // region nearly full: bring the bound up to date and drop what fell below it
                     refresh_threshold(hist, cs, k_eff, lane);
                     __syncwarp();
-                    wcount = compact_region(region, wcount, *(volatile unsigned*)&cs.thr_key, lane);
-                    if (wcount > CS_REGION_SOFT) full_region = true;    // ties or a coarse bin too full
+                    st.wcount = compact_region(region, st.wcount, *(volatile unsigned*)&cs.thr_key, lane);
+                    if (st.wcount > CS_REGION_SOFT) st.full = 1;    // ties or a coarse bin too full
                 }
             }
-            __syncwarp();
-            if (lane == 0 && !dead) mbar_arrive(&empty[s]);     // the stage is free again
         }
 
         // ---- row end: survivors and row statistics to global scratch -----------------------------
-        while (qn > 0 && !full_region && !dead) drain(min(qn, 32));
-        if (lane == 0 && full_region) cs.overflow = 1;
+        while (st.qn > 0 && !st.full && !dead)
+            st = drain_parked<T>(st, min(st.qn, 32), qvec_off, qidx_off, region_off, hist_off, *(volatile unsigned*)&cs.thr_key, a.V);
+        if (lane == 0 && st.full) cs.overflow = 1;
         if (STATS) {
             const double sw = (double)warp_sum(acc);
             if (lane == 0) cs.wsum[warp] = sw;
@@ -477,7 +518,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
         if (row_ok) {
             // every warp filters its own region and appends to the row's scratch area
             u64* dst = a.surv_keys + (long long)row * surv_cap;
-            const int n = compact_region(region, wcount, *(volatile unsigned*)&cs.thr_key, lane);
+            const int n = compact_region(region, st.wcount, *(volatile unsigned*)&cs.thr_key, lane);
             int base = 0;
             if (lane == 0 && n) base = atomicAdd(&cs.m, n);
             base = __shfl_sync(0xffffffffu, base, 0);

@@ -37,14 +37,26 @@ __global__ void __launch_bounds__(THREADS) precise_chunk_sums_kernel(PreciseArgs
         const int src_row = a.pos ? e * a.seq_rows + a.pos[e] : e * a.expand + ri;
         const int b = src_row / a.seq_rows;
         const T* row = reinterpret_cast<const T*>(a.logits) + (long long)src_row * a.row_stride;
-        const double Td = (double)a.temperature[b];
-        const double m = (double)a.row_max[src_row] / Td;
-        double s = 0.0;
+        // x = l * (1/T) instead of l / T: one rounding of 2^-53 more per term, far below every
+        // threshold this pass decides; four independent sums keep the exp pipeline busy
+        const double rT = 1.0 / (double)a.temperature[b];
+        const double m = (double)a.row_max[src_row] * rT;
         const int v0 = c * CHUNK;
-        for (int k = lane; k < CHUNK; k += 32) {
+        double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+#pragma unroll 2
+        for (int k = lane; k < CHUNK; k += 128) {
             const int v = v0 + k;
-            if (v < a.V) s += exp((double)load_logit(row, v) / Td - m);
+            float l0 = -CUDART_INF_F, l1 = -CUDART_INF_F, l2 = -CUDART_INF_F, l3 = -CUDART_INF_F;
+            if (v < a.V) l0 = load_logit(row, v);
+            if (v + 32 < a.V) l1 = load_logit(row, v + 32);
+            if (v + 64 < a.V) l2 = load_logit(row, v + 64);
+            if (v + 96 < a.V) l3 = load_logit(row, v + 96);
+            s0 += exp((double)l0 * rT - m);
+            s1 += exp((double)l1 * rT - m);
+            s2 += exp((double)l2 * rT - m);
+            s3 += exp((double)l3 * rT - m);
         }
+        double s = (s0 + s1) + (s2 + s3);
         s = warp_sum(s);
         if (lane == 0) a.dsum[(long long)src_row * a.nch + c] = s;
     }

@@ -9,6 +9,9 @@
 namespace picospec {
 
 constexpr unsigned ST_INTERNAL = 8u;          // a bounded wait ran out (mirrors picospec.h)
+#ifndef PICOSPEC_WAIT_HINT_NS
+#define PICOSPEC_WAIT_HINT_NS 20000u      // suspend-time hint of one mbarrier.try_wait
+#endif
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after two seconds
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -58,7 +61,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (uint32_t i = 1;; ++i) {
-        if (mbar_try_wait_hint(bar, parity, 20000u)) return true;
+        if (mbar_try_wait_hint(bar, parity, PICOSPEC_WAIT_HINT_NS)) return true;
         if ((i & 7u) == 0u && global_ns() - t0 > WAIT_LIMIT_NS) return false;
     }
 }

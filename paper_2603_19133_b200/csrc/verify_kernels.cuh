@@ -347,16 +347,31 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 if (!range_bad) {
                     const int* idx = a.q_idx + (long long)ri * a.k_max;
                     const float* prob = a.q_prob + (long long)ri * a.k_max;
-                    for (int k = lane; k < n; k += 32) {
-                        const int v = idx[k];
-                        if (v < 0 || v >= a.V) {
-                            range_bad = true;
-                            continue;
+                    // eight entries per lane at a time: all index loads, then all logit gathers
+                    for (int k0 = 0; k0 < n; k0 += 256) {
+                        int vv[8];
+                        float qq[8], ll[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const int k = k0 + u * 32 + lane;
+                            vv[u] = k < n ? idx[k] : -2;
+                            qq[u] = k < n ? prob[k] : 0.f;
                         }
-                        const double qk = (double)prob[k];
-                        const double pk = wt(load_logit(row, v)) / Z;
-                        smin += fmin(pk, qk);
-                        if (v == x && k < kx) kx = k;
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const bool ok = vv[u] >= 0 && vv[u] < a.V;
+                            if (vv[u] != -2 && !ok) range_bad = true;
+                            ll[u] = ok ? load_logit(row, vv[u]) : -CUDART_INF_F;
+                        }
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const int k = k0 + u * 32 + lane;
+                            if (vv[u] >= 0 && vv[u] < a.V) {
+                                const double pk = wt(ll[u]) / Z;
+                                smin += fmin(pk, (double)qq[u]);
+                                if (vv[u] == x && k < kx) kx = k;
+                            }
+                        }
                     }
                 }
                 range_bad = __any_sync(0xffffffffu, range_bad);
@@ -444,14 +459,26 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 __syncthreads();
                 if (use_resid) {
                     bool rb = false;
-                    for (int k = tid; k < n; k += THREADS) {
-                        const int v = idx[k];
-                        if (v < 0 || v >= a.V) {
-                            rb = true;
-                            continue;
+                    {
+                        // n <= 1024: at most four entries per thread, loads first
+                        int vv[4];
+                        float qq[4], ll[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int k = tid + u * THREADS;
+                            vv[u] = k < n ? idx[k] : -2;
+                            qq[u] = k < n ? prob[k] : 0.f;
                         }
-                        const double pk = wt(load_logit(row, v)) / Z;
-                        atomicAdd(&cm[v / CHUNK], -fmin(pk, (double)prob[k]));
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const bool ok = vv[u] >= 0 && vv[u] < a.V;
+                            if (vv[u] != -2 && !ok) rb = true;
+                            ll[u] = ok ? load_logit(row, vv[u]) : -CUDART_INF_F;
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (vv[u] >= 0 && vv[u] < a.V)
+                                atomicAdd(&cm[vv[u] / CHUNK], -fmin(wt(ll[u]) / Z, (double)qq[u]));
                     }
                     if (rb) atomicOr(&sh.bad, (int)ST_RANGE);
                 }

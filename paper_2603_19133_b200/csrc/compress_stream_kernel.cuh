@@ -279,6 +279,15 @@ __device__ __forceinline__ uint4 vec_words(const ChunkRegs<float>& r, int j) {
                       __float_as_uint(r.f[4 * j + 3]));
 }
 
+// Region nearly full: bring the bound up to date and drop what fell below it (one warp; out of line).
+__device__ __noinline__ int maintain_region(int wcount, int region_off, int hist_off, CsShared* cs, int k_eff) {
+    extern __shared__ __align__(1024) unsigned char dyn[];
+    const int lane = threadIdx.x & 31;
+    refresh_threshold(reinterpret_cast<const unsigned*>(dyn + hist_off), *cs, k_eff, lane);
+    __syncwarp();
+    return compact_region(reinterpret_cast<u64*>(dyn + region_off), wcount, *(volatile unsigned*)&cs->thr_key, lane);
+}
+
 // Per-warp filter state kept in registers.
 struct WarpQ {
     int qhead, qn;      // ring of parked vectors
@@ -480,7 +489,10 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
 #pragma unroll
                 for (int j = 0; j < NVEC; ++j) {
                     if (mj[j] == 0u) continue;
-                    if (st.qn >= 32) st = drain_parked<T>(st, 32, qvec_off, qidx_off, region_off, hist_off, thr_key, a.V);
+                    if (st.qn >= 32) {
+                        if (st.wcount > CS_REGION_SOFT) st.wcount = maintain_region(st.wcount, region_off, hist_off, &cs, k_eff);
+                        st = drain_parked<T>(st, 32, qvec_off, qidx_off, region_off, hist_off, *(volatile unsigned*)&cs.thr_key, a.V);
+                    }
                     if ((hits >> j) & 1u) {
                         const int slot = (st.qhead + st.qn + __popc(mj[j] & lt_mask)) & (CS_QCAP - 1);
                         qvec[slot] = vec_words(regs, j);
@@ -488,16 +500,15 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
                     }
                     st.qn += __popc(mj[j]);
                 }
-                __syncwarp();
-                if (st.qn >= 32) st = drain_parked<T>(st, 32, qvec_off, qidx_off, region_off, hist_off, thr_key, a.V);
+                if (st.qn >= 32) {
+                    if (st.wcount > CS_REGION_SOFT) st.wcount = maintain_region(st.wcount, region_off, hist_off, &cs, k_eff);
+                    st = drain_parked<T>(st, 32, qvec_off, qidx_off, region_off, hist_off, *(volatile unsigned*)&cs.thr_key, a.V);
+                }
                 // the bound is refreshed after tiles 1, 2, 4, 8, ..., each time by another warp (vectors
                 // still parked in the rings are not counted yet, which only makes it a little lower)
                 if (((ti + 1) & ti) == 0 && warp == ((31 - __clz(ti + 1)) & (WARPS - 1))) refresh_threshold(hist, cs, k_eff, lane);
                 if (st.wcount > CS_REGION_SOFT) {
-                    // region nearly full: bring the bound up to date and drop what fell below it
-                    refresh_threshold(hist, cs, k_eff, lane);
-                    __syncwarp();
-                    st.wcount = compact_region(region, st.wcount, *(volatile unsigned*)&cs.thr_key, lane);
+                    st.wcount = maintain_region(st.wcount, region_off, hist_off, &cs, k_eff);
                     if (st.wcount > CS_REGION_SOFT) st.full = 1;    // ties or a coarse bin too full
                 }
             }

@@ -40,6 +40,12 @@ __device__ __forceinline__ float warp_max(float v) {
     for (int d = 16; d > 0; d >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, d));
     return v;
 }
+// maximum over the warp in one instruction; NaN inputs are ignored (all NaN gives NaN)
+__device__ __forceinline__ float warp_max_redux(float v) {
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
+}
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
@@ -153,6 +159,18 @@ template <> struct ChunkRegs<__nv_bfloat16> {
         uint32_t mm = *reinterpret_cast<uint32_t*>(&m);
         return fmaxf(__uint_as_float(mm << 16), __uint_as_float(mm & 0xffff0000u));
     }
+    // maximum of the lane's 32 values, NaN ignored
+    __device__ __forceinline__ float lane_max_plain() const {
+        __nv_bfloat162 m[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            m[k] = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&w[2 * k]), *reinterpret_cast<const __nv_bfloat162*>(&w[2 * k + 1]));
+#pragma unroll
+        for (int k = 0; k < 4; ++k) m[k] = __hmax2(m[2 * k], m[2 * k + 1]);
+        const __nv_bfloat162 a = __hmax2(__hmax2(m[0], m[1]), __hmax2(m[2], m[3]));
+        const uint32_t mm = *reinterpret_cast<const uint32_t*>(&a);
+        return fmaxf(__uint_as_float(mm << 16), __uint_as_float(mm & 0xffff0000u));
+    }
     // NaN-propagating maximum of the lane's 32 values
     __device__ __forceinline__ float lane_max() const {
         __nv_bfloat162 m = *reinterpret_cast<const __nv_bfloat162*>(&w[0]);
@@ -185,6 +203,12 @@ template <> struct ChunkRegs<float> {
     static __device__ __forceinline__ int offset(int k, int lane) { return (k >> 2) * 128 + lane * 4 + (k & 3); }
     __device__ __forceinline__ float vec_max(int j) const {
         return fmaxf(fmaxf(f[4 * j], f[4 * j + 1]), fmaxf(f[4 * j + 2], f[4 * j + 3]));
+    }
+    __device__ __forceinline__ float lane_max_plain() const {
+        float m[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) m[k] = fmaxf(fmaxf(f[4 * k], f[4 * k + 1]), fmaxf(f[4 * k + 2], f[4 * k + 3]));
+        return fmaxf(fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])), fmaxf(fmaxf(m[4], m[5]), fmaxf(m[6], m[7])));
     }
     __device__ __forceinline__ float lane_max() const {
         float m = f[0];

@@ -5,11 +5,12 @@
 // shared memory by bulk async copies; the producer lane runs ahead into the next row) and keeps
 // every element that can still be among the k largest:
 //   - the CTA holds a running lower bound `thr` on the k-th largest logit of the row;
-//   - per chunk a lane compares the maximum of each 16-byte vector it holds with thr; vectors
-//     that reach it are parked in a per-warp ring in shared memory, and whenever 32 are parked the
-//     warp tests their elements with all lanes busy (one element position per step, positions by
-//     ballot) and appends the survivors (64-bit keys: logit, then lower index first) to the warp's
-//     own region of the candidate buffer: no atomics with a return value, no CTA barrier;
+//   - per chunk a lane compares its 32 values with thr (packed compares for bf16) into a 32-bit
+//     mask; the warp then takes one set bit per lane per step, ranks the lanes by ballot and
+//     appends the values (64-bit keys: logit, then lower index first; the value is re-read from the
+//     staged tile) to the warp's own region of the candidate buffer: no atomics with a return
+//     value, no CTA barrier.  About 15 of the 1024 values of a chunk pass, so this is two or three
+//     steps per chunk;
 //   - every stored candidate is counted in a two-level histogram over the top 12 bits of the
 //     orderable logit; thr is the lower edge of the highest bin whose suffix count reaches k, so
 //     it is a valid bound whenever it is computed, by any warp, from whatever has been counted so
@@ -34,23 +35,13 @@
 
 namespace picospec {
 
-// Tunables (overridable at build time).
-#ifndef PICOSPEC_CS_CAND_CAP
-#define PICOSPEC_CS_CAND_CAP 4096
-#endif
-#ifndef PICOSPEC_CS_STAGES_BF16
-#define PICOSPEC_CS_STAGES_BF16 3
-#endif
-#ifndef PICOSPEC_CS_CTAS
-#define PICOSPEC_CS_CTAS 2
-#endif
-constexpr int CS_CAND_CAP = PICOSPEC_CS_CAND_CAP;          // candidate keys held in shared memory
-constexpr int CS_REGION = CS_CAND_CAP / WARPS;             // each worker warp appends to its own region
-constexpr int CS_REGION_SOFT = CS_REGION - CS_REGION / 4;  // a region this full is compacted against thr
+// Two shapes of the filter kernel: rows with k <= 256 need few live candidates, so a small
+// candidate buffer and two stages leave room for three CTAs per SM; larger k takes the big buffer.
+constexpr int CS_CAP_SMALL = 2048, CS_CAP_LARGE = 4096;    // candidate keys held in shared memory
+constexpr int CS_K_SMALL = 256;                            // largest k served by the small shape
 constexpr int CS_BIN_SHIFT = 20;
 constexpr int CS_BINS = 4096;        // histogram bins: top 12 bits of the orderable logit
 constexpr int CS_SUPER = CS_BINS / 32;
-constexpr int CS_QCAP = 64;          // per-warp ring of parked vectors
 
 // row flags written by the filter kernel
 constexpr int CSF_TEMPERATURE = 1, CSF_LOGIT = 2, CSF_REDO = 4, CSF_ABORT = 8;
@@ -63,14 +54,16 @@ struct CsRowMeta {
     double z_stream;  // sum of 2^(l * c32 - ref_off) over the row (top-p only)
 };
 
-template <typename T> struct CsCfg;
-template <> struct CsCfg<__nv_bfloat16> { static constexpr int STAGES = PICOSPEC_CS_STAGES_BF16; };   // x 16 KB
-template <> struct CsCfg<float> { static constexpr int STAGES = 2; };                                 // x 32 KB
-template <typename T> struct CsGeom {
+// SMALL: CAP 2048, bf16 2 stages x 16 KB (3 CTAs / SM); LARGE: CAP 4096, bf16 3 stages (2 CTAs / SM).
+// fp32 tiles are 32 KB: 2 stages in both shapes.
+template <typename T, bool SMALL> struct CsGeom {
+    static constexpr int CAP = SMALL ? CS_CAP_SMALL : CS_CAP_LARGE;
+    static constexpr int REGION = CAP / WARPS;             // each worker warp appends to its own region
+    static constexpr int STAGES = sizeof(T) == 2 ? (SMALL ? 2 : 3) : 2;
+    static constexpr int CTAS = (sizeof(T) == 2 && SMALL) ? 3 : 2;
     static constexpr int TILE_BYTES = TILE_CHUNKS * CHUNK * (int)sizeof(T);
-    static constexpr int STAGE_BYTES = CsCfg<T>::STAGES * TILE_BYTES;
-    static constexpr int QUEUE_BYTES = WARPS * CS_QCAP * 20;
-    static constexpr int SMEM_BYTES = STAGE_BYTES + CS_CAND_CAP * 8 + (CS_BINS + CS_SUPER) * 4 + QUEUE_BYTES;
+    static constexpr int STAGE_BYTES = STAGES * TILE_BYTES;
+    static constexpr int SMEM_BYTES = STAGE_BYTES + CAP * 8 + (CS_BINS + CS_SUPER) * 4;
 };
 
 // capacity of a row's scratch area (keys) for a sparse-row capacity k_max
@@ -94,73 +87,44 @@ __device__ __forceinline__ float thr_of_key(unsigned key) {
 
 // ---- per-dtype pieces --------------------------------------------------------------------------
 
-// element e of a parked vector
-__device__ __forceinline__ float vec_elem(const uint4& q, int e, const __nv_bfloat16*) {
-    const uint32_t w = e < 4 ? (e < 2 ? q.x : q.y) : (e < 6 ? q.z : q.w);
-    return (e & 1) ? __uint_as_float(w & 0xffff0000u) : __uint_as_float(w << 16);
+// 32-bit mask of the lane's values that are >= thr (NaN never passes).
+//   bf16: bit k = low half of word k, bit 16 + k = high half of word k.  The packed threshold is
+//         the smallest bf16 >= thr for every threshold this kernel produces (a bf16 value itself,
+//         or the lower edge of a histogram bin: positive edges are bf16 values, negative edges
+//         have all low bits set, so dropping them rounds towards zero, i.e. up).
+//   fp32: bit k = value k.
+__device__ __forceinline__ unsigned pass_mask(const ChunkRegs<__nv_bfloat16>& r, float thr) {
+    const uint32_t h = __float_as_uint(thr) >> 16;
+    const uint32_t t2 = h | (h << 16);
+    const __nv_bfloat162 t = *reinterpret_cast<const __nv_bfloat162*>(&t2);
+    unsigned mask = 0;
+#pragma unroll
+    for (int k = 0; k < 16; ++k)
+        mask |= __hge2_mask(*reinterpret_cast<const __nv_bfloat162*>(&r.w[k]), t) & (0x00010001u << k);
+    return mask;
 }
-__device__ __forceinline__ float vec_elem(const uint4& q, int e, const float*) {
-    return __uint_as_float(e < 2 ? (e == 0 ? q.x : q.y) : (e == 2 ? q.z : q.w));
+__device__ __forceinline__ unsigned pass_mask(const ChunkRegs<float>& r, float thr) {
+    unsigned mask = 0;
+#pragma unroll
+    for (int k = 0; k < 32; ++k) mask |= (r.f[k] >= thr ? 1u : 0u) << k;
+    return mask;
 }
-
-// Per-lane view of a chunk for the filter: a bit per vector that may hold an element >= thr (a
-// superset: the element test decides) and the lane's maximum (NaN if the lane holds a NaN).
-template <typename T> struct ChunkScan;
-template <> struct ChunkScan<__nv_bfloat16> {
-    __nv_bfloat162 vmax[4];      // per vector: (max of even elements, max of odd elements)
-    float lane_max;
-    __device__ __forceinline__ void scan(const ChunkRegs<__nv_bfloat16>& r) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            __nv_bfloat162 m = *reinterpret_cast<const __nv_bfloat162*>(&r.w[4 * j]);
-#pragma unroll
-            for (int k = 1; k < 4; ++k) m = __hmax2_nan(m, *reinterpret_cast<const __nv_bfloat162*>(&r.w[4 * j + k]));
-            vmax[j] = m;
-        }
-        __nv_bfloat162 a = __hmax2_nan(__hmax2_nan(vmax[0], vmax[1]), __hmax2_nan(vmax[2], vmax[3]));
-        const uint32_t aa = *reinterpret_cast<uint32_t*>(&a);
-        const uint32_t sw = __byte_perm(aa, aa, 0x1032);
-        a = __hmax2_nan(a, *reinterpret_cast<const __nv_bfloat162*>(&sw));
-        lane_max = __uint_as_float(*reinterpret_cast<uint32_t*>(&a) << 16);
-    }
-    // thr as a packed pair: the smallest bf16 >= thr when thr is negative or a bf16 itself (every
-    // threshold this kernel produces); otherwise a slightly lower value, which only adds vectors.
-    // A NaN maximum counts as a hit; the element test drops it.
-    __device__ __forceinline__ unsigned hit_mask(float thr) const {
-        const uint32_t h = __float_as_uint(thr) >> 16;
-        const uint32_t t2 = h | (h << 16);
-        const __nv_bfloat162 t = *reinterpret_cast<const __nv_bfloat162*>(&t2);
-        unsigned m = 0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) m |= (__hblt2(vmax[j], t) ? 0u : 1u) << j;     // not (both halves < thr)
-        return m;
-    }
-};
-template <> struct ChunkScan<float> {
-    float vmax[8];
-    float lane_max;
-    __device__ __forceinline__ void scan(const ChunkRegs<float>& r) {
-        bool nan = false;
-        float lm = -CUDART_INF_F;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            vmax[j] = fmaxf(fmaxf(r.f[4 * j], r.f[4 * j + 1]), fmaxf(r.f[4 * j + 2], r.f[4 * j + 3]));
-            nan |= (r.f[4 * j] != r.f[4 * j]) | (r.f[4 * j + 1] != r.f[4 * j + 1]) | (r.f[4 * j + 2] != r.f[4 * j + 2]) |
-                   (r.f[4 * j + 3] != r.f[4 * j + 3]);
-            lm = fmaxf(lm, vmax[j]);
-        }
-        lane_max = nan ? CUDART_NAN_F : lm;
-    }
-    __device__ __forceinline__ unsigned hit_mask(float thr) const {
-        unsigned m = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) m |= (vmax[j] >= thr ? 1u : 0u) << j;
-        return m;
-    }
-};
+// offset inside the chunk (in elements) of the value behind mask bit b of a lane
+__device__ __forceinline__ int bit_offset(int b, int lane, const __nv_bfloat16*) {
+    const int k = b & 15;
+    return (k >> 2) * 256 + lane * 8 + (k & 3) * 2 + (b >> 4);
+}
+__device__ __forceinline__ int bit_offset(int b, int lane, const float*) { return (b >> 2) * 128 + lane * 4 + (b & 3); }
+// value at an element offset of a staged chunk
+__device__ __forceinline__ float staged_value(const unsigned char* chunk, int off, const __nv_bfloat16*) {
+    return __uint_as_float((uint32_t)reinterpret_cast<const unsigned short*>(chunk)[off] << 16);
+}
+__device__ __forceinline__ float staged_value(const unsigned char* chunk, int off, const float*) {
+    return reinterpret_cast<const float*>(chunk)[off];
+}
 
 // 16-bit orderable keys of the maxima of groups of 2 consecutive elements of the lane's chunk
-// (NaN is ignored here; the lane maximum reports it).
+// (NaN is ignored here).
 __device__ __forceinline__ void pair_keys(const ChunkRegs<__nv_bfloat16>& r, unsigned (&key)[16]) {
 #pragma unroll
     for (int k = 0; k < 16; ++k)
@@ -194,9 +158,10 @@ __device__ __forceinline__ unsigned warp_kth_key(const unsigned (&key)[16], int 
     return prefix;
 }
 
-// First-tile bound of one warp: group size g (elements) in {2, 4, 8 (bf16 only)}.
+// First-tile bound of one warp: group size g (elements) in {2, 4, 8 (bf16 only)}.  Out of line: it
+// runs once per row.
 template <typename T>
-__device__ __forceinline__ unsigned first_tile_key(const ChunkRegs<T>& regs, int g, int need) {
+__device__ __noinline__ unsigned first_tile_key(const ChunkRegs<T>& regs, int g, int need) {
     unsigned key[16];
     pair_keys(regs, key);
     if (g == 2) return warp_kth_key<16>(key, need);
@@ -271,14 +236,11 @@ __device__ __forceinline__ int compact_region(u64* region, int n, unsigned thr_k
     return out;
 }
 
-__device__ __forceinline__ uint4 vec_words(const ChunkRegs<__nv_bfloat16>& r, int j) {
-    return make_uint4(r.w[4 * j], r.w[4 * j + 1], r.w[4 * j + 2], r.w[4 * j + 3]);
+// Refresh the bound (one warp; out of line).
+__device__ __noinline__ void refresh_bound(int hist_off, CsShared* cs, int k_eff) {
+    extern __shared__ __align__(1024) unsigned char dyn[];
+    refresh_threshold(reinterpret_cast<const unsigned*>(dyn + hist_off), *cs, k_eff, threadIdx.x & 31);
 }
-__device__ __forceinline__ uint4 vec_words(const ChunkRegs<float>& r, int j) {
-    return make_uint4(__float_as_uint(r.f[4 * j]), __float_as_uint(r.f[4 * j + 1]), __float_as_uint(r.f[4 * j + 2]),
-                      __float_as_uint(r.f[4 * j + 3]));
-}
-
 // Region nearly full: bring the bound up to date and drop what fell below it (one warp; out of line).
 __device__ __noinline__ int maintain_region(int wcount, int region_off, int hist_off, CsShared* cs, int k_eff) {
     extern __shared__ __align__(1024) unsigned char dyn[];
@@ -288,76 +250,17 @@ __device__ __noinline__ int maintain_region(int wcount, int region_off, int hist
     return compact_region(reinterpret_cast<u64*>(dyn + region_off), wcount, *(volatile unsigned*)&cs->thr_key, lane);
 }
 
-// Per-warp filter state kept in registers.
-struct WarpQ {
-    int qhead, qn;      // ring of parked vectors
-    int wcount;         // candidates in this warp's region
-    int full;           // the region ran out of room (the row goes to the redo list)
-};
-
-// Tests up to 32 parked vectors, one element position per step with every lane on its own vector,
-// and appends the survivors to the warp's region.  Not inlined: it is called from several places of
-// the hot loop, which has to stay small.  Offsets are bytes into the kernel's dynamic shared memory.
-template <typename T>
-__device__ __noinline__ WarpQ drain_parked(WarpQ st, int n, int qvec_off, int qidx_off, int region_off, int hist_off,
-                                           unsigned thr_key, int V) {
+template <typename T, bool STATS, bool SMALL>
+__global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compress_filter_kernel(CompressArgs a, int tiles_per_row) {
     extern __shared__ __align__(1024) unsigned char dyn[];
+    typedef CsGeom<T, SMALL> Geom;
+    constexpr int STAGES = Geom::STAGES;
+    constexpr int TILE_BYTES = Geom::TILE_BYTES;
+    constexpr int CS_CAND_CAP = Geom::CAP, CS_REGION = Geom::REGION;
     constexpr int VEC = ChunkRegs<T>::VEC;
-    const int lane = threadIdx.x & 31;
-    const unsigned lt_mask = (1u << lane) - 1u;
-    const uint4* qvec = reinterpret_cast<const uint4*>(dyn + qvec_off);
-    const int* qidx = reinterpret_cast<const int*>(dyn + qidx_off);
-    u64* region = reinterpret_cast<u64*>(dyn + region_off);
-    unsigned* hist = reinterpret_cast<unsigned*>(dyn + hist_off);
-    const int slot = (st.qhead + lane) & (CS_QCAP - 1);
-    uint4 q = make_uint4(0, 0, 0, 0);
-    int vb = V;
-    __syncwarp();       // the other lanes' parked vectors are visible
-    if (lane < n) {
-        q = qvec[slot];
-        vb = qidx[slot];
-    }
-    const bool active = vb < V;
-    const float thr = thr_of_key(thr_key);
-    const int before = st.wcount;
-    int wcount = st.wcount;
-#pragma unroll
-    for (int e = 0; e < VEC; ++e) {
-        const float l = vec_elem(q, e, (const T*)nullptr) + 0.0f;     // -0 becomes +0
-        const bool p = active && l >= thr;
-        const unsigned m = __ballot_sync(0xffffffffu, p);
-        const int pos = wcount + __popc(m & lt_mask);
-        if (p && pos < CS_REGION) {
-            const uint32_t bits = __float_as_uint(l);
-            const uint32_t okey = bits ^ ((uint32_t)((int32_t)bits >> 31) | 0x80000000u);
-            region[pos] = ((u64)okey << 32) | (u64)(~(uint32_t)(vb + e));
-        }
-        wcount += __popc(m);
-    }
-    if (wcount > CS_REGION) {
-        st.full = 1;
-        wcount = CS_REGION;
-    }
-    __syncwarp();
-    // count the new entries in the histogram
-    for (int x = before + lane; x < wcount; x += 32) hist_add(hist, (int)(region[x] >> (32 + CS_BIN_SHIFT)));
-    st.wcount = wcount;
-    st.qhead = (st.qhead + n) & (CS_QCAP - 1);
-    st.qn -= n;
-    __syncwarp();       // the slots just read may be refilled
-    return st;
-}
-
-template <typename T, bool STATS>
-__global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_filter_kernel(CompressArgs a, int tiles_per_row) {
-    extern __shared__ __align__(1024) unsigned char dyn[];
-    constexpr int STAGES = CsCfg<T>::STAGES;
-    constexpr int TILE_BYTES = CsGeom<T>::TILE_BYTES;
-    constexpr int VEC = ChunkRegs<T>::VEC, NVEC = ChunkRegs<T>::NVEC;
     unsigned char* stage_mem = dyn;
-    u64* cand = reinterpret_cast<u64*>(dyn + CsGeom<T>::STAGE_BYTES);
+    u64* cand = reinterpret_cast<u64*>(dyn + Geom::STAGE_BYTES);
     unsigned* hist = reinterpret_cast<unsigned*>(cand + CS_CAND_CAP);          // bins, then super-bins
-    unsigned char* qmem = reinterpret_cast<unsigned char*>(hist + CS_BINS + CS_SUPER);
     __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES];
     __shared__ CsShared cs;
 
@@ -419,12 +322,8 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
     }
 
     // ---- workers ------------------------------------------------------------------------------
-    uint4* qvec = reinterpret_cast<uint4*>(qmem) + warp * CS_QCAP;
-    int* qidx = reinterpret_cast<int*>(qmem + WARPS * CS_QCAP * 16) + warp * CS_QCAP;
     u64* region = cand + warp * CS_REGION;
     const unsigned lt_mask = (1u << lane) - 1u;
-    const int qvec_off = (int)(reinterpret_cast<unsigned char*>(qvec) - dyn);
-    const int qidx_off = (int)(reinterpret_cast<unsigned char*>(qidx) - dyn);
     const int region_off = (int)(reinterpret_cast<unsigned char*>(region) - dyn);
     const int hist_off = (int)(reinterpret_cast<unsigned char*>(hist) - dyn);
     // first-tile bound: groups of g elements, at least 4 k groups in the tile
@@ -440,7 +339,8 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
         const bool valid = temp_ok(Tb);
         const float c32 = temp_scale(Tb);
         float ref_off = 0.f, acc = 0.f;
-        WarpQ st = {0, 0, 0, 0};
+        int wcount = 0;             // candidates in this warp's region
+        bool full_region = false;   // the region ran out of room (the row goes to the redo list)
 
         for (int ti = 0; ti < tiles_per_row; ++ti, ++i) {
             const int s = (int)(i % STAGES);
@@ -453,21 +353,23 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
                 }
             }
             const int c = ti * TILE_CHUNKS + warp;
-            const bool work = !dead && valid && !st.full && c < a.nch;
+            const bool work = !dead && valid && !full_region && c < a.nch;
+            const unsigned char* chunk = stage_mem + s * TILE_BYTES + warp * (CHUNK * (int)sizeof(T));
             ChunkRegs<T> regs;
-            if (work) load_staged(regs, stage_mem + s * TILE_BYTES + warp * (CHUNK * (int)sizeof(T)), c * CHUNK, a.V, lane);
-            __syncwarp();
-            if (lane == 0 && !dead) mbar_arrive(&empty[s]);     // the chunk is in registers: the stage is free
-            ChunkScan<T> sc;
             if (work) {
-                sc.scan(regs);
-                if (sc.lane_max != sc.lane_max) cs.nan = 1;
+                load_staged(regs, chunk, c * CHUNK, a.V, lane);
+                if (!STATS) {
+                    // without the exp-sum (which turns NaN by itself) a NaN has to be looked for
+                    const float lm = regs.lane_max();
+                    if (lm != lm) cs.nan = 1;
+                }
             }
             if (ti == 0 && valid) {
                 // first tile (every warp holds a full chunk): each warp's own bound, then the minimum
                 if (work) {
                     const unsigned k16 = first_tile_key(regs, g, need);
-                    const float wm = warp_max(sc.lane_max);      // NaN lanes are ignored here
+                    float wm = 0.f;
+                    if (STATS) wm = warp_max_redux(regs.lane_max_plain());
                     if (lane == 0) {
                         atomicMin(&cs.thr0_key, k16 << 16);
                         if (STATS && wm == wm) atomicMax(&cs.top_key, orderable(wm));
@@ -480,44 +382,56 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
             }
             if (work) {
                 const unsigned thr_key = *(volatile unsigned*)&cs.thr_key;
-                const unsigned hits = sc.hit_mask(thr_of_key(thr_key));
-                unsigned mj[NVEC];
-#pragma unroll
-                for (int j = 0; j < NVEC; ++j) mj[j] = __ballot_sync(0xffffffffu, (hits >> j) & 1u);
+                unsigned mask = pass_mask(regs, thr_of_key(thr_key));
+                if (thr_key < 0x00800000u) {
+                    // no finite bound (rows of -inf): everything would pass, padding included
+                    full_region = true;
+                    mask = 0u;
+                }
                 if (STATS) acc += lane_exp_sum2(regs, c32, ref_off);
-                const int v0 = c * CHUNK + lane * VEC;
-#pragma unroll
-                for (int j = 0; j < NVEC; ++j) {
-                    if (mj[j] == 0u) continue;
-                    if (st.qn >= 32) {
-                        if (st.wcount > CS_REGION_SOFT) st.wcount = maintain_region(st.wcount, region_off, hist_off, &cs, k_eff);
-                        st = drain_parked<T>(st, 32, qvec_off, qidx_off, region_off, hist_off, *(volatile unsigned*)&cs.thr_key, a.V);
+                const int total = __reduce_add_sync(0xffffffffu, __popc(mask));     // what this chunk adds
+                if (wcount + total > CS_REGION) {
+                    // no room: bring the bound up to date and drop what fell below it
+                    wcount = maintain_region(wcount, region_off, hist_off, &cs, k_eff);
+                    if (wcount + total > CS_REGION) {     // ties, a coarse bin too full, or a very loose bound
+                        full_region = true;
+                        mask = 0u;
                     }
-                    if ((hits >> j) & 1u) {
-                        const int slot = (st.qhead + st.qn + __popc(mj[j] & lt_mask)) & (CS_QCAP - 1);
-                        qvec[slot] = vec_words(regs, j);
-                        qidx[slot] = v0 + j * (32 * VEC);
+                }
+                // one set bit per lane per step; lanes are ranked by ballot
+                const int before = wcount;
+                const int vchunk = c * CHUNK;
+                for (;;) {
+                    const unsigned m = __ballot_sync(0xffffffffu, mask != 0u);
+                    if (m == 0u) break;
+                    if (mask != 0u) {
+                        const int bit = __ffs(mask) - 1;
+                        mask &= mask - 1u;
+                        const int off = bit_offset(bit, lane, (const T*)nullptr);
+                        const int pos = wcount + __popc(m & lt_mask);
+                        {
+                            const uint32_t bits = __float_as_uint(staged_value(chunk, off, (const T*)nullptr) + 0.0f);   // -0 becomes +0
+                            const uint32_t okey = bits ^ ((uint32_t)((int32_t)bits >> 31) | 0x80000000u);
+                            region[pos] = ((u64)okey << 32) | (u64)(~(uint32_t)(vchunk + off));
+                        }
                     }
-                    st.qn += __popc(mj[j]);
+                    wcount += __popc(m);
                 }
-                if (st.qn >= 32) {
-                    if (st.wcount > CS_REGION_SOFT) st.wcount = maintain_region(st.wcount, region_off, hist_off, &cs, k_eff);
-                    st = drain_parked<T>(st, 32, qvec_off, qidx_off, region_off, hist_off, *(volatile unsigned*)&cs.thr_key, a.V);
-                }
-                // the bound is refreshed after tiles 1, 2, 4, 8, ..., each time by another warp (vectors
-                // still parked in the rings are not counted yet, which only makes it a little lower)
-                if (((ti + 1) & ti) == 0 && warp == ((31 - __clz(ti + 1)) & (WARPS - 1))) refresh_threshold(hist, cs, k_eff, lane);
-                if (st.wcount > CS_REGION_SOFT) {
-                    st.wcount = maintain_region(st.wcount, region_off, hist_off, &cs, k_eff);
-                    if (st.wcount > CS_REGION_SOFT) st.full = 1;    // ties or a coarse bin too full
+                __syncwarp();
+                // count the new entries in the histogram
+                for (int x = before + lane; x < wcount; x += 32) hist_add(hist, (int)(region[x] >> (32 + CS_BIN_SHIFT)));
+                // the bound is refreshed after tiles 1, 2, 4, 8, ..., each time by another warp
+                if (((ti + 1) & ti) == 0 && warp == ((31 - __clz(ti + 1)) & (WARPS - 1))) {
+                    __syncwarp();
+                    refresh_bound(hist_off, &cs, k_eff);
                 }
             }
+            __syncwarp();
+            if (lane == 0 && !dead) mbar_arrive(&empty[s]);     // the stage is free again
         }
 
         // ---- row end: survivors and row statistics to global scratch -----------------------------
-        while (st.qn > 0 && !st.full && !dead)
-            st = drain_parked<T>(st, min(st.qn, 32), qvec_off, qidx_off, region_off, hist_off, *(volatile unsigned*)&cs.thr_key, a.V);
-        if (lane == 0 && st.full) cs.overflow = 1;
+        if (lane == 0 && full_region) cs.overflow = 1;
         if (STATS) {
             const double sw = (double)warp_sum(acc);
             if (lane == 0) cs.wsum[warp] = sw;
@@ -529,7 +443,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
         if (row_ok) {
             // every warp filters its own region and appends to the row's scratch area
             u64* dst = a.surv_keys + (long long)row * surv_cap;
-            const int n = compact_region(region, st.wcount, *(volatile unsigned*)&cs.thr_key, lane);
+            const int n = compact_region(region, wcount, *(volatile unsigned*)&cs.thr_key, lane);
             int base = 0;
             if (lane == 0 && n) base = atomicAdd(&cs.m, n);
             base = __shfl_sync(0xffffffffu, base, 0);
@@ -543,7 +457,8 @@ __global__ void __launch_bounds__(STREAM_THREADS, PICOSPEC_CS_CTAS) compress_fil
             if (cs.abort) flags = CSF_ABORT;
             else if (!valid) flags = CSF_TEMPERATURE;
             else if (cs.overflow || m > surv_cap) flags = CSF_REDO;      // too many candidates or ties at the bound
-            else if (cs.nan || m < k_eff) flags = CSF_LOGIT;
+            else if (cs.nan) flags = CSF_LOGIT;
+            else if (m < k_eff) flags = CSF_REDO;                        // cannot happen with a valid bound; be safe
             double zs = 0.0;
             if (STATS)
                 for (int w = 0; w < WARPS; ++w) zs += cs.wsum[w];

@@ -89,6 +89,21 @@ template <typename T> void set_compress_attrs() {
     cudaFuncSetAttribute(compress_kernel<T, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, COMPRESS_SMEM);
 }
 
+template <typename T> cudaError_t set_filter_attrs() {
+    cudaError_t e = cudaFuncSetAttribute(compress_filter_kernel<T, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         CsGeom<T, true>::SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(compress_filter_kernel<T, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 CsGeom<T, true>::SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(compress_filter_kernel<T, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 CsGeom<T, false>::SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(compress_filter_kernel<T, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 CsGeom<T, false>::SMEM_BYTES);
+    return e;
+}
+
 // Opt-in shared-memory sizes of the staged kernels: once per device and process.
 cudaError_t ensure_kernel_attrs(int device) {
     static std::mutex mu;
@@ -102,18 +117,8 @@ cudaError_t ensure_kernel_attrs(int device) {
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(chunk_stats_bulk_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  TileGeom<float>::SMEM_BYTES);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(compress_filter_kernel<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 CsGeom<__nv_bfloat16>::SMEM_BYTES);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(compress_filter_kernel<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 CsGeom<__nv_bfloat16>::SMEM_BYTES);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(compress_filter_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 CsGeom<float>::SMEM_BYTES);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(compress_filter_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 CsGeom<float>::SMEM_BYTES);
+    if (e == cudaSuccess) e = set_filter_attrs<__nv_bfloat16>();
+    if (e == cudaSuccess) e = set_filter_attrs<float>();
     if (e == cudaSuccess) done[device] = true;
     return e;
 }
@@ -135,18 +140,21 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
         cudaError_t ea = ensure_kernel_attrs(ctx->device);
         if (ea != cudaSuccess) return ea;
         const int tiles_per_row = (a.nch + TILE_CHUNKS - 1) / TILE_CHUNKS;
+        int k_eff = a.top_k > 0 ? a.top_k : a.k_max;
+        if (k_eff > a.k_max) k_eff = a.k_max;
+        const bool small = k_eff <= CS_K_SMALL;
+        void (*kern)(CompressArgs, int) =
+            small ? (stats ? compress_filter_kernel<T, true, true> : compress_filter_kernel<T, false, true>)
+                  : (stats ? compress_filter_kernel<T, true, false> : compress_filter_kernel<T, false, false>);
+        const int smem = small ? CsGeom<T, true>::SMEM_BYTES : CsGeom<T, false>::SMEM_BYTES;
         int per_sm = 1;     // resident CTAs per SM for this kernel's registers and shared memory
-        cudaError_t eo = stats ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_filter_kernel<T, true>,
-                                                                             STREAM_THREADS, CsGeom<T>::SMEM_BYTES)
-                               : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_filter_kernel<T, false>,
-                                                                             STREAM_THREADS, CsGeom<T>::SMEM_BYTES);
+        cudaError_t eo = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, STREAM_THREADS, smem);
         if (eo != cudaSuccess) return eo;
         if (per_sm < 1) per_sm = 1;
         const int g = rows < ctx->num_sms * per_sm ? rows : ctx->num_sms * per_sm;
         {
             ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_STREAM, 1, s);
-            if (stats) compress_filter_kernel<T, true><<<g, STREAM_THREADS, CsGeom<T>::SMEM_BYTES, s>>>(a, tiles_per_row);
-            else compress_filter_kernel<T, false><<<g, STREAM_THREADS, CsGeom<T>::SMEM_BYTES, s>>>(a, tiles_per_row);
+            kern<<<g, STREAM_THREADS, smem, s>>>(a, tiles_per_row);
         }
         cudaError_t e0 = cudaGetLastError();
         if (e0 != cudaSuccess) return e0;

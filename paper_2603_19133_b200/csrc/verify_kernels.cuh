@@ -218,13 +218,11 @@ __global__ void __launch_bounds__(STREAM_THREADS, StreamCfg<T>::CTAS_PER_SM) chu
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty[s]);
         if (work) {
-            const float lm = regs.lane_max();
-            const float cm = warp_max(lm);
-            const float off = __fmul_rn(cm, d.c32);
-            float sum = 0.f;
-            if (cm > -CUDART_INF_F) sum = lane_exp_sum2(regs, d.c32, off);
-            if (lm != lm) sum = CUDART_NAN_F;     // NaN in the chunk: the finish kernel reports it
-            sum = warp_sum(sum);
+            // chunk maximum with NaN ignored; a NaN (or +inf) logit turns the exp-sum into NaN by
+            // itself, which the finish kernel reports; a chunk of -inf only sums to zero
+            const float cm = warp_max_redux(regs.lane_max_plain());
+            const float off = cm > -CUDART_INF_F ? __fmul_rn(cm, d.c32) : 0.f;
+            const float sum = warp_sum(lane_exp_sum2(regs, d.c32, off));
             if (lane == 0) a.stats[(long long)d.src_row * a.nch + c] = make_float2(cm, sum);
         }
     }

@@ -5,7 +5,8 @@ One "step" is one pass of the whole path over one batch of synthetic input: draf
 compression (picospec_compress, with the draft-token draw) followed by target-side verification
 with the fused residual / bonus sample (picospec_verify).  The headline metric is verified
 draft positions per second (B * gamma per step); the roofline entry is the achieved HBM
-bandwidth of the verify streaming kernel.
+bandwidth of the dominant kernel (the one with the longest average launch of the step: the
+compress filter pass or the verify streaming pass; the other one is listed under "kernels").
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config4] [--impl ours|reference]
 
@@ -35,8 +36,9 @@ import gen  # noqa: E402
 METRIC = "verified_draft_positions_per_sec"
 UNIT = "positions/s"
 
-# DRAM traffic of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum per launch)
-# from the ncu captures summarised under profiles/; None until a capture exists for the workload.
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/, keyed by (workload, kernel); absent until a capture of the current
+# kernel exists.  Captured at B = 64 and scaled to the full batch by the rows processed.
 NCU_TRAFFIC_BYTES = {}
 
 
@@ -65,7 +67,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "25",
                  "-i", str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -140,7 +142,14 @@ def run_reference(args):
     import oracle
     w = gen.WORKLOADS[args.workload]
     cores = oracle.cores()
-    sample_B = min(w.B, args.ref_sample)
+    # size the per-step sample so that steps + warm-up end within about two minutes: calibrate on
+    # a few sequences first (sequences are independent, so the cost is linear in their number)
+    cal_B = min(w.B, 4)
+    wc, ic = oracle_sample(w, 4241, cal_B)
+    per_seq = oracle_step_time(wc, ic, cores) / cal_B
+    budget_s = 100.0
+    sample_B = int(budget_s / (max(args.steps + min(args.warmup, 1), 1) * per_seq))
+    sample_B = max(1, min(w.B, args.ref_sample, sample_B))
     ws, inp = oracle_sample(w, 4242, sample_B)
     for _ in range(min(args.warmup, 1)):
         oracle_step_time(ws, inp, cores)
@@ -152,7 +161,10 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * t / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "V": w.V, "B": ws.B, "gamma": w.G, "logits": w.dtype, "k_max": w.k_max},
+        "config": {"workload": w.name, "V": w.V, "B_per_gpu": w.B, "gamma": w.G, "logits": w.dtype,
+                   "top_k": w.top_k, "top_p": w.top_p, "k_max": w.k_max,
+                   "step": "oracle compress + oracle verify (with sample) on a bounded sample of the batch",
+                   "sample_sequences_per_step": ws.B},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -349,7 +361,16 @@ def run_ours(args):
                                   f"all {cores} host threads (OpenMP over rows)"}
 
     if rank == 0:
-        vs = main["verify_stream"]
+        peak = main["peak"]
+        kern = {
+            "compress_filter_kernel (picospec_compress streaming pass)": main["compress_stream"],
+            "chunk_stats_bulk_kernel (picospec_verify streaming pass)": main["verify_stream"],
+        }
+        for v in kern.values():
+            v["frac_of_peak"] = (v["GBps"] or 0) / peak
+            v["frac_of_8TBps_nominal"] = (v["GBps"] or 0) / 8000.0
+        dom_name = max(kern, key=lambda k: kern[k]["avg_us"])
+        dom = kern[dom_name]
         line = {
             "metric": METRIC, "value": main["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * main["seconds"] / args.steps, "higher_is_better": True,
@@ -360,14 +381,14 @@ def run_ours(args):
                        "l2": f"inputs larger than L2: {main['nsets']} input set(s) of "
                              f"{(w.B * (2 * w.G + 1)) * w.V * w.bytes_per_logit / 1e6:.0f} MB rotated",
                        "parallelism": f"dp{world} (sequences sharded, no collective)"},
-            "roofline": {"bound": "hbm", "kernel": "chunk_stats_kernel (picospec_verify streaming pass)",
-                         "achieved": vs["GBps"], "peak": main["peak"], "unit": "GB/s",
-                         "frac": (vs["GBps"] or 0) / main["peak"], "peak_kind": f"of {main['peak_kind']}",
-                         "frac_of_8TBps_nominal": (vs["GBps"] or 0) / 8000.0,
-                         "avg_launch_us": vs["avg_us"], "launches_timed": vs["launches"],
-                         "algorithmic_bytes_per_launch": vs["alg_bytes"],
-                         "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
-            "kernels": {"compress_stream": main["compress_stream"]},
+            "roofline": {"bound": "hbm", "kernel": dom_name,
+                         "achieved": dom["GBps"], "peak": peak, "unit": "GB/s",
+                         "frac": (dom["GBps"] or 0) / peak, "peak_kind": f"of {main['peak_kind']}",
+                         "frac_of_8TBps_nominal": (dom["GBps"] or 0) / 8000.0,
+                         "avg_launch_us": dom["avg_us"], "launches_timed": dom["launches"],
+                         "algorithmic_bytes_per_launch": dom["alg_bytes"],
+                         "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom_name.split(" ")[0]))},
+            "kernels": kern,
             "e2e": {k: main["e2e"][k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step")},
             "gpu_launches": main["launches_per_step"] * args.steps,
             "cpu_baseline": cpu_baseline,
@@ -387,8 +408,8 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config4", choices=sorted(gen.WORKLOADS))
     ap.add_argument("--ref-sample", type=int, default=64, help="sequences per step of the CPU oracle legs")

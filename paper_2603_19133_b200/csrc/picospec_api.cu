@@ -185,7 +185,7 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
     p.logits = a.logits; p.row_stride = a.row_stride; p.V = a.V; p.nch = a.nch;
     p.seq_rows = a.G; p.expand = 1; p.pos = nullptr; p.temperature = a.temperature;
     p.queue = a.queue; p.queue_count = a.queue_count; p.row_max = a.row_max; p.dsum = a.dsum;
-    precise_chunk_sums_kernel<T><<<ctx->num_sms * 2, THREADS, 0, s>>>(p);
+    precise_chunk_sums_kernel<T><<<ctx->num_sms * 6, THREADS, 0, s>>>(p);
     const int g2 = rows < ctx->num_sms ? rows : ctx->num_sms;
     compress_precise_kernel<T><<<g2, THREADS, MAX_K * 8, s>>>(a);
     return cudaGetLastError();
@@ -225,7 +225,7 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
     p.seq_rows = a.G + 1; p.expand = a.sample_only ? 1 : a.G + 1; p.pos = a.sample_only ? a.pos : nullptr;
     p.temperature = a.temperature; p.queue = a.queue; p.queue_count = a.queue_count;
     p.row_max = a.row_max; p.dsum = a.dsum;
-    precise_chunk_sums_kernel<T><<<ctx->num_sms * 2, THREADS, 0, s>>>(p);
+    precise_chunk_sums_kernel<T><<<ctx->num_sms * 6, THREADS, 0, s>>>(p);
     const int g2 = a.B < ctx->num_sms ? a.B : ctx->num_sms;
     verify_finish_kernel<T, true><<<g2, THREADS, dyn, s>>>(a);
     return cudaGetLastError();

@@ -39,7 +39,10 @@ UNIT = "positions/s"
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/, keyed by (workload, kernel); absent until a capture of the current
 # kernel exists.  Captured at B = 64 and scaled to the full batch by the rows processed.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    ("config4", "compress_filter_kernel"): 4 * (98564608 + 4149504),
+    ("config4", "chunk_stats_bulk_kernel"): 4 * (114932224 + 3787520),
+}
 
 
 def _peaks():

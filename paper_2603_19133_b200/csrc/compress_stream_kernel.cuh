@@ -158,10 +158,10 @@ __device__ __forceinline__ unsigned warp_kth_key(const unsigned (&key)[16], int 
     return prefix;
 }
 
-// First-tile bound of one warp: group size g (elements) in {2, 4, 8 (bf16 only)}.  Out of line: it
-// runs once per row.
+// First-tile bound of one warp: group size g (elements) in {2, 4, 8 (bf16 only)}.  (Inlined: an
+// out-of-line call would force the chunk registers through local memory in every tile.)
 template <typename T>
-__device__ __noinline__ unsigned first_tile_key(const ChunkRegs<T>& regs, int g, int need) {
+__device__ __forceinline__ unsigned first_tile_key(const ChunkRegs<T>& regs, int g, int need) {
     unsigned key[16];
     pair_keys(regs, key);
     if (g == 2) return warp_kth_key<16>(key, need);

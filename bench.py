@@ -390,7 +390,7 @@ def run_ours(args):
                          "frac_of_8TBps_nominal": (dom["GBps"] or 0) / 8000.0,
                          "avg_launch_us": dom["avg_us"], "launches_timed": dom["launches"],
                          "algorithmic_bytes_per_launch": dom["alg_bytes"],
-                         "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom_name.split(" ")[0]))},
+                         "traffic": None if args.batch > 0 else NCU_TRAFFIC_BYTES.get((w.name, dom_name.split(" ")[0]))},
             "kernels": kern,
             "e2e": {k: main["e2e"][k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step")},
             "gpu_launches": main["launches_per_step"] * args.steps,

@@ -42,6 +42,11 @@ constexpr int CS_K_SMALL = 256;                            // largest k served b
 constexpr int CS_BIN_SHIFT = 20;
 constexpr int CS_BINS = 4096;        // histogram bins: top 12 bits of the orderable logit
 constexpr int CS_SUPER = CS_BINS / 32;
+// Bin counts are 16 bits wide, two per word (super-bin counts are 32-bit).  A count can only wrap
+// on rows that push tens of thousands of values into one bin; a wrap makes a sum too small (a
+// lower, still valid bound) and its carry makes the neighbouring bin one too large, which can at
+// worst leave fewer than k survivors: such a row goes to the redo list.
+constexpr int CS_HIST_WORDS = CS_BINS / 2 + CS_SUPER;
 
 // row flags written by the filter kernel
 constexpr int CSF_TEMPERATURE = 1, CSF_LOGIT = 2, CSF_REDO = 4, CSF_ABORT = 8;
@@ -54,16 +59,16 @@ struct CsRowMeta {
     double z_stream;  // sum of 2^(l * c32 - ref_off) over the row (top-p only)
 };
 
-// SMALL: CAP 2048, bf16 2 stages x 16 KB (3 CTAs / SM); LARGE: CAP 4096, bf16 3 stages (2 CTAs / SM).
+// SMALL: CAP 2048, bf16 3 stages x 16 KB (72.5 KB: 3 CTAs / SM); LARGE: CAP 4096 (88.5 KB: 2 CTAs / SM).
 // fp32 tiles are 32 KB: 2 stages in both shapes.
 template <typename T, bool SMALL> struct CsGeom {
     static constexpr int CAP = SMALL ? CS_CAP_SMALL : CS_CAP_LARGE;
     static constexpr int REGION = CAP / WARPS;             // each worker warp appends to its own region
-    static constexpr int STAGES = sizeof(T) == 2 ? (SMALL ? 2 : 3) : 2;
+    static constexpr int STAGES = sizeof(T) == 2 ? 3 : 2;
     static constexpr int CTAS = (sizeof(T) == 2 && SMALL) ? 3 : 2;
     static constexpr int TILE_BYTES = TILE_CHUNKS * CHUNK * (int)sizeof(T);
     static constexpr int STAGE_BYTES = STAGES * TILE_BYTES;
-    static constexpr int SMEM_BYTES = STAGE_BYTES + CAP * 8 + (CS_BINS + CS_SUPER) * 4;
+    static constexpr int SMEM_BYTES = STAGE_BYTES + CAP * 8 + CS_HIST_WORDS * 4;
 };
 
 // capacity of a row's scratch area (keys) for a sparse-row capacity k_max
@@ -175,14 +180,14 @@ __device__ __forceinline__ unsigned first_tile_key(const ChunkRegs<T>& regs, int
 
 // two-level histogram update
 __device__ __forceinline__ void hist_add(unsigned* hist, int bin) {
-    atomicAdd(&hist[bin], 1u);
-    atomicAdd(&hist[CS_BINS + (bin >> 5)], 1u);
+    atomicAdd(&hist[bin >> 1], (bin & 1) ? 0x10000u : 1u);
+    atomicAdd(&hist[CS_BINS / 2 + (bin >> 5)], 1u);
 }
 
 // One warp: raise thr to the lower edge of the highest bin whose suffix count reaches k.
 __device__ __forceinline__ void refresh_threshold(const unsigned* hist, CsShared& cs, int k, int lane) {
     // level 1: lane l owns super-bins 4l .. 4l+3 (super-bin s covers bins 32 s .. 32 s + 31)
-    const uint4 sv = *reinterpret_cast<const uint4*>(&hist[CS_BINS + 4 * lane]);
+    const uint4 sv = *reinterpret_cast<const uint4*>(&hist[CS_BINS / 2 + 4 * lane]);
     const unsigned own = sv.x + sv.y + sv.z + sv.w;
     unsigned suf = own;             // inclusive suffix sum over lanes (higher lanes = higher bins)
 #pragma unroll
@@ -210,7 +215,7 @@ __device__ __forceinline__ void refresh_threshold(const unsigned* hist, CsShared
         }
     }
     // level 2: the 32 bins of super-bin s, lane l reads bin 32 s + l
-    unsigned bs = hist[32 * s + lane];
+    unsigned bs = (hist[16 * s + (lane >> 1)] >> ((lane & 1) * 16)) & 0xffffu;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
         const unsigned y = __shfl_down_sync(0xffffffffu, bs, d);
@@ -289,7 +294,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
         cs.abort = 0;
         cs.m = 0;
     }
-    for (int i = tid; i < CS_BINS + CS_SUPER; i += STREAM_THREADS) hist[i] = 0u;
+    for (int i = tid; i < CS_HIST_WORDS; i += STREAM_THREADS) hist[i] = 0u;
     __syncthreads();
 
     if (warp == WARPS) {
@@ -480,7 +485,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
             cs.nan = 0;
             cs.m = 0;
         }
-        for (int x = tid; x < CS_BINS + CS_SUPER; x += THREADS) hist[x] = 0u;
+        for (int x = tid; x < CS_HIST_WORDS; x += THREADS) hist[x] = 0u;
         workers_sync();
     }
 }

@@ -31,6 +31,7 @@ struct picospec_ctx {
     double* dsum;
     float* row_max;
     int* queue;
+    unsigned long long* need_rows;
     int* counters;  // [0] verify queue, [1],[2] compress queue (alternating), [3],[4] compress redo list (alternating)
     int* redo_rows; // rows the staged compress kernel hands to the direct kernel
     unsigned long long* surv_keys;  // staged compress: survivors per row
@@ -185,6 +186,7 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
     p.logits = a.logits; p.row_stride = a.row_stride; p.V = a.V; p.nch = a.nch;
     p.seq_rows = a.G; p.expand = 1; p.pos = nullptr; p.temperature = a.temperature;
     p.queue = a.queue; p.queue_count = a.queue_count; p.row_max = a.row_max; p.dsum = a.dsum;
+    p.need_rows = nullptr;
     precise_chunk_sums_kernel<T><<<ctx->num_sms * 6, THREADS, 0, s>>>(p);
     const int g2 = rows < ctx->num_sms ? rows : ctx->num_sms;
     compress_precise_kernel<T><<<g2, THREADS, MAX_K * 8, s>>>(a);
@@ -224,6 +226,7 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
     p.logits = a.logits; p.row_stride = a.row_stride; p.V = a.V; p.nch = a.nch;
     p.seq_rows = a.G + 1; p.expand = a.sample_only ? 1 : a.G + 1; p.pos = a.sample_only ? a.pos : nullptr;
     p.temperature = a.temperature; p.queue = a.queue; p.queue_count = a.queue_count;
+    p.need_rows = a.need_rows;
     p.row_max = a.row_max; p.dsum = a.dsum;
     precise_chunk_sums_kernel<T><<<ctx->num_sms * 6, THREADS, 0, s>>>(p);
     const int g2 = a.B < ctx->num_sms ? a.B : ctx->num_sms;
@@ -267,6 +270,7 @@ int picospec_create(picospec_ctx** out, int device, int max_batch, int max_gamma
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->dsum, rows * nch * sizeof(double));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->row_max, rows * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->queue, rows * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->need_rows, rows * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->counters, 8 * sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->redo_rows, rows * sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_keys, rows * (size_t)cs_survivor_cap(max_k) * sizeof(unsigned long long));
@@ -297,6 +301,7 @@ int picospec_destroy(picospec_ctx* ctx) {
     cudaFree(ctx->dsum);
     cudaFree(ctx->row_max);
     cudaFree(ctx->queue);
+    cudaFree(ctx->need_rows);
     cudaFree(ctx->counters);
     cudaFree(ctx->redo_rows);
     cudaFree(ctx->surv_keys);
@@ -426,6 +431,7 @@ static int verify_common(picospec_ctx* ctx, VerifyArgs& a, picospec_dtype dtype,
     if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
     a.nch = (a.V + CHUNK - 1) / CHUNK;
     a.stats = ctx->stats; a.row_max = ctx->row_max; a.dsum = ctx->dsum; a.queue = ctx->queue;
+    a.need_rows = ctx->need_rows;
     a.queue_count = ctx->counters; a.status = ctx->status; a.slow_rows = ctx->slow_rows;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     cudaError_t e;
@@ -492,6 +498,7 @@ struct StaticWorkspace {
     double dsum[STATIC_ROWS * STATIC_NCH];
     float row_max[STATIC_ROWS];
     int queue[STATIC_ROWS];
+    unsigned long long need_rows[STATIC_ROWS];
     // the words below must read zero when a call starts; one memset covers them
     int counters[4];
     unsigned status;
@@ -567,6 +574,7 @@ extern "C" int picospec_verify_static(const void* target_logits, picospec_dtype 
     a.accept_len = accept_len; a.p_draft = p_draft; a.resid_mass = resid_mass; a.borderline = borderline_count;
     a.token = token; a.mass = nullptr;
     a.stats = ws->stats; a.row_max = ws->row_max; a.dsum = ws->dsum; a.queue = ws->queue;
+    a.need_rows = ws->need_rows;
     a.queue_count = ws->counters; a.status = &ws->status; a.slow_rows = &ws->slow_rows;
     cudaError_t e;
     if (dtype == PICOSPEC_BF16)

@@ -17,6 +17,7 @@ struct PreciseArgs {
     const float* temperature;  // [B]
     const int* queue;
     const int* queue_count;
+    const unsigned long long* need_rows;   // optional [entries]: bit ri = row ri of the entry is wanted
     const float* row_max;      // [rows] exact row maxima from the fp32 pass
     double* dsum;              // [rows, nch]
 };
@@ -34,6 +35,7 @@ __global__ void __launch_bounds__(THREADS) precise_chunk_sums_kernel(PreciseArgs
         const long long t = item / a.nch;
         const int ri = (int)(t % a.expand);
         const int e = a.queue[(int)(t / a.expand)];
+        if (a.need_rows && !a.pos && ri < 64 && !((a.need_rows[e] >> ri) & 1ull)) continue;
         const int src_row = a.pos ? e * a.seq_rows + a.pos[e] : e * a.expand + ri;
         const int b = src_row / a.seq_rows;
         const T* row = reinterpret_cast<const T*>(a.logits) + (long long)src_row * a.row_stride;

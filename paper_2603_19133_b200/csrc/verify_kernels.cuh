@@ -31,6 +31,7 @@ struct VerifyArgs {
     float* row_max;            // [B*(G+1)]
     double* dsum;              // [B*(G+1), nch]: exact chunk sums of flagged sequences
     int* queue;                // [B] flagged sequences
+    unsigned long long* need_rows;  // [B] per flagged sequence: bit i = row i needs exact chunk sums
     int* queue_count;          // [1]
     unsigned* status;          // sticky status word
     unsigned long long* slow_rows;  // cumulative rows re-evaluated in double precision
@@ -245,12 +246,17 @@ struct FinishShared {
     float qloc[CHUNK];
 };
 
-template <typename T, bool PRECISE>
-__device__ __forceinline__ void row_stats(const VerifyArgs& a, int src_row, float c32, int lane, double& Z,
+// bit i of a sequence's row mask (rows beyond 63 always count as set)
+__device__ __forceinline__ bool row_needed(unsigned long long need, int i) { return i >= 64 || ((need >> i) & 1ull); }
+
+template <typename T>
+__device__ __forceinline__ void row_stats(const VerifyArgs& a, int src_row, float c32, int lane, bool exact, double& Z,
                                           double& Zraw, float& mx, bool& bad) {
-    // combine the chunk statistics of one row (called by a full warp)
+    // combine the chunk statistics of one row (called by a full warp): the exact double-precision
+    // chunk sums if they were recomputed for this row, else the fp32 streaming statistics
     bad = false;
-    if (PRECISE) {
+    Zraw = 0.0;
+    if (exact) {
         mx = a.row_max[src_row];
         double s = 0.0;
         for (int c = lane; c < a.nch; c += 32) s += a.dsum[(long long)src_row * a.nch + c];
@@ -292,6 +298,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
     const int nloop = PRECISE ? *a.queue_count : a.B;
     for (int slot = blockIdx.x; slot < nloop; slot += gridDim.x) {
         const int b = PRECISE ? a.queue[slot] : slot;
+        const unsigned long long need = PRECISE ? a.need_rows[b] : 0ull;   // rows with exact chunk sums
         const float Tb = a.temperature[b];
         const float c32 = temp_scale(Tb);
         const T* seq = reinterpret_cast<const T*>(a.logits) + (long long)b * G1 * a.row_stride;
@@ -316,7 +323,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 double Z, Zraw;
                 float mx;
                 bool bad;
-                row_stats<T, PRECISE>(a, b * G1 + i, c32, lane, Z, Zraw, mx, bad);
+                row_stats<T>(a, b * G1 + i, c32, lane, PRECISE && row_needed(need, i), Z, Zraw, mx, bad);
                 if (lane == 0) {
                     sh.Z[i] = Z;
                     sh.Zraw[i] = Zraw;
@@ -443,7 +450,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
             bool use_resid = n > 0;
             for (int pass = 0; pass < 2 && !st_bits; ++pass) {
                 // chunk masses (in units where the row sums to one)
-                if (PRECISE) {
+                if (PRECISE && row_needed(need, j)) {
                     for (int c = tid; c < a.nch; c += THREADS) cm[c] = a.dsum[(long long)(b * G1 + j) * a.nch + c] / Z;
                 } else {
                     const float2* st = a.stats + (long long)(b * G1 + j) * a.nch;
@@ -621,9 +628,31 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 if (PRECISE) {
                     if (nborder && a.borderline) atomicAdd(a.borderline, nborder);
                 } else if (flagged) {
+                    // Which rows need exact sums: an ambiguous accept test can move the first
+                    // rejection anywhere from its position on, so every row from there; an ambiguous
+                    // draw needs the sampled row only.
+                    unsigned long long nd = 0ull;
+                    int nrows = 0;
+                    if (a.sample_only) {
+                        nd = ~0ull;
+                        nrows = 1;
+                    } else {
+                        int first_amb = -1;
+                        const int last = alen < G ? alen : G - 1;
+                        for (int i = 0; i <= last && first_amb < 0; ++i)
+                            if (sh.amb[i]) first_amb = i;
+                        for (int i = 0; i < G1; ++i) {
+                            const bool nr = i >= 64 || (first_amb >= 0 && i >= first_amb) || (sh.flag && want_token && i == alen);
+                            if (nr) {
+                                if (i < 64) nd |= 1ull << i;
+                                ++nrows;
+                            }
+                        }
+                    }
+                    a.need_rows[b] = nd;
                     const int q = atomicAdd(a.queue_count, 1);
                     a.queue[q] = b;
-                    atomicAdd(a.slow_rows, (unsigned long long)(a.sample_only ? 1 : G1));
+                    atomicAdd(a.slow_rows, (unsigned long long)nrows);
                 }
             }
         }

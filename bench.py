@@ -256,6 +256,7 @@ def bench_workload(ps, w, args, rank, world, device, with_e2e, with_clocks):
             torch.cuda.synchronize()
 
     ctx.status(clear=True)
+    ctx.counters(clear=True)
     ctx.profile_enable(1)
     sampler = ClockSampler(torch.cuda.current_device()) if with_clocks else None
     if sampler:
@@ -266,6 +267,7 @@ def bench_workload(ps, w, args, rank, world, device, with_e2e, with_clocks):
     ms_vs, n_vs = ctx.profile_read(1)
     ms_cs, n_cs = ctx.profile_read(0)
     ctx.profile_enable(0)
+    _, redo = ctx.counters()
     st, slow = ctx.status(clear=True)
     if world > 1:
         tt = torch.tensor([t], device=device, dtype=torch.float64)
@@ -281,6 +283,7 @@ def bench_workload(ps, w, args, rank, world, device, with_e2e, with_clocks):
     res = {
         "seconds": t, "seconds_unbracketed": t_plain, "status": st,
         "slow_rows_per_step": slow / float(args.steps + args.warmup),
+        "redo_rows_per_step": redo / float(args.steps + args.warmup),
         "value": world * w.B * w.G * args.steps / t,
         "rows_streamed_per_sec": world * w.B * (2 * w.G + 1) * args.steps / t,
         "verify_stream": {"avg_us": vs_time * 1e6, "launches": n_vs, "alg_bytes": vbytes,
@@ -399,6 +402,7 @@ def run_ours(args):
             "ms_per_step_without_event_brackets": 1e3 * main["seconds_unbracketed"] / args.steps,
             "rows_streamed_per_sec": main["rows_streamed_per_sec"],
             "slow_path_rows_per_step": main["slow_rows_per_step"],
+            "compress_redo_rows_per_step": main["redo_rows_per_step"],
             "device_status": main["status"],
             "other_configs": others,
         }

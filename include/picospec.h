@@ -100,6 +100,14 @@ PICOSPEC_API int picospec_profile_read(picospec_ctx* ctx, int kind, float* total
 PICOSPEC_API int picospec_status(picospec_ctx* ctx, int* device_status_out, long long* slow_path_rows_out, int clear,
                     void* cuda_stream);
 
+/* Synchronise `cuda_stream`, then copy two cumulative work counters to HOST memory: out[0] = rows
+ * re-evaluated in double precision (the same number picospec_status reports), out[1] = draft rows
+ * that the staged compress kernel handed to the direct kernel because their candidates did not
+ * fit its buffer (heavy ties, adversarial order, no finite bound).  Both are performance
+ * diagnostics; results do not depend on them.  If `clear` is non-zero both are reset.  The paper
+ * has no counterpart. */
+PICOSPEC_API int picospec_counters(picospec_ctx* ctx, long long* out, int clear, void* cuda_stream);
+
 /* Half 1 -- draft-side sparse compression (Sec. 3.3, Eq. (4): keep the K most probable entries
  * with their vocabulary indices; this build applies it to the drafter's distribution, adds the
  * top-p cut and renormalises).

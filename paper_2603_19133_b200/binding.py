@@ -44,6 +44,8 @@ def lib() -> ctypes.CDLL:
                                                c_int, vp, vp, vp, vp]
         L.picospec_profile_enable.argtypes = [vp, c_int]
         L.picospec_profile_read.argtypes = [vp, c_int, ctypes.POINTER(c_f), ctypes.POINTER(c_int), vp]
+        L.picospec_counters.argtypes = [vp, ctypes.POINTER(c_ll), c_int, vp]
+        L.picospec_counters.restype = c_int
         L.picospec_verify_static.argtypes = [vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp, c_int,
                                              vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.picospec_verify_static.restype = c_int
@@ -160,6 +162,13 @@ class Context:
         if rc not in (OK, EDATA):
             raise PicospecError(rc, "picospec_status")
         return st.value, slow.value
+
+    def counters(self, clear: bool = False) -> Tuple[int, int]:
+        """Synchronise the current stream; return (rows re-evaluated in double precision, draft rows
+        the staged compress kernel handed to the direct kernel), both cumulative."""
+        out = (ctypes.c_longlong * 2)()
+        _check(lib().picospec_counters(self._h, out, int(clear), _stream()), "picospec_counters")
+        return int(out[0]), int(out[1])
 
     def profile_enable(self, level: int):
         """0 = off, 1 = time the two streaming kernels, 2 = time every kernel group."""

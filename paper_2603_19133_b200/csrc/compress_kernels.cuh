@@ -39,6 +39,7 @@ struct CompressArgs {
     int* redo_count;           // zero on entry of the staged kernel
     int* redo_count_next;      // cleared for the next call
     int use_redo_list;         // direct kernel: 1 = process redo_rows[0 .. *redo_count) only
+    unsigned long long* redo_total;   // cumulative number of rows handed over (reported by picospec_counters)
     // staged path: survivors of the filter kernel, [B*G, cs_survivor_cap(k_max)] keys + one record per row
     unsigned long long* surv_keys;
     CsRowMeta* surv_meta;

@@ -469,7 +469,10 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
                 for (int w = 0; w < WARPS; ++w) zs += cs.wsum[w];
             // a reference that later logits overflowed, or NaN / +inf data: the direct kernel sorts it out
             if (STATS && flags == 0 && !(zs > 0.0 && zs < CUDART_INF)) flags = CSF_REDO;
-            if (flags & CSF_REDO) a.redo_rows[atomicAdd(a.redo_count, 1)] = row;
+            if (flags & CSF_REDO) {
+                a.redo_rows[atomicAdd(a.redo_count, 1)] = row;
+                atomicAdd(a.redo_total, 1ull);
+            }
             CsRowMeta meta;
             meta.count = m;
             meta.flags = flags;

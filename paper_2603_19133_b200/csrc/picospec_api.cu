@@ -203,7 +203,7 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
     if (staged) {
         cudaError_t ea = ensure_kernel_attrs(ctx->device);
         if (ea != cudaSuccess) return ea;
-        const int tiles_per_row = (a.nch + TILE_CHUNKS - 1) / TILE_CHUNKS;
+        const int tiles_per_row = (a.nch + TileGeom<T>::CHUNKS - 1) / TileGeom<T>::CHUNKS;
         const long long tiles = (long long)(a.sample_only ? a.B : a.B * (a.G + 1)) * tiles_per_row;
         const int gcap = ctx->num_sms * StreamCfg<T>::CTAS_PER_SM;
         const int g = (int)(tiles < gcap ? tiles : gcap);
@@ -276,10 +276,10 @@ int picospec_create(picospec_ctx** out, int device, int max_batch, int max_gamma
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_keys, rows * (size_t)cs_survivor_cap(max_k) * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_meta, rows * sizeof(CsRowMeta));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->status, sizeof(unsigned));
-    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->slow_rows, sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->slow_rows, 2 * sizeof(unsigned long long));   // [0] slow rows, [1] redo rows
     if (e == cudaSuccess) e = cudaMemset(ctx->counters, 0, 8 * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(unsigned));
-    if (e == cudaSuccess) e = cudaMemset(ctx->slow_rows, 0, sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(ctx->slow_rows, 0, 2 * sizeof(unsigned long long));
     if (e == cudaSuccess) {
         set_compress_attrs<float>();
         set_compress_attrs<__nv_bfloat16>();
@@ -389,6 +389,20 @@ int picospec_status(picospec_ctx* ctx, int* device_status_out, long long* slow_p
     return st ? PICOSPEC_EDATA : PICOSPEC_OK;
 }
 
+int picospec_counters(picospec_ctx* ctx, long long* out, int clear, void* cuda_stream) {
+    if (!ctx || !out) return PICOSPEC_EINVAL;
+    DeviceGuard g(ctx->device);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    unsigned long long v[2] = {0, 0};
+    cudaError_t e = cudaMemcpyAsync(v, ctx->slow_rows, sizeof(v), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && clear) e = cudaMemsetAsync(ctx->slow_rows, 0, sizeof(v), s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    out[0] = (long long)v[0];
+    out[1] = (long long)v[1];
+    return PICOSPEC_OK;
+}
+
 int picospec_compress(picospec_ctx* ctx, const void* draft_logits, picospec_dtype dtype, int B, int G, int V,
                       long long row_stride_elems, const float* temperature, int top_k, float top_p, int k_max,
                       int* q_idx, float* q_prob, int* q_count, const float* u_draft, int* draft_tok,
@@ -413,6 +427,7 @@ int picospec_compress(picospec_ctx* ctx, const void* draft_logits, picospec_dtyp
     a.redo_count = ctx->counters + 2 + cur;           // [3] / [4]
     a.redo_count_next = ctx->counters + 2 + (3 - cur);
     a.use_redo_list = 0;
+    a.redo_total = ctx->slow_rows + 1;
     a.surv_keys = ctx->surv_keys;
     a.surv_meta = ctx->surv_meta;
     ctx->compress_calls++;

@@ -152,16 +152,23 @@ template <typename T> struct StreamCfg;
 #ifndef PICOSPEC_CTAS_PER_SM_F32
 #define PICOSPEC_CTAS_PER_SM_F32 2
 #endif
+#ifndef PICOSPEC_CPW_BF16
+#define PICOSPEC_CPW_BF16 1                      // chunks per worker warp and tile (statistics pass)
+#endif
 template <> struct StreamCfg<__nv_bfloat16> {
     static constexpr int STAGES = PICOSPEC_STAGES_BF16;
     static constexpr int CTAS_PER_SM = PICOSPEC_CTAS_PER_SM_BF16;
+    static constexpr int CPW = PICOSPEC_CPW_BF16;
 };
 template <> struct StreamCfg<float> {
     static constexpr int STAGES = PICOSPEC_STAGES_F32;
     static constexpr int CTAS_PER_SM = PICOSPEC_CTAS_PER_SM_F32;
+    static constexpr int CPW = 1;
 };
+// tiles of the statistics pass: CPW consecutive chunks per worker warp
 template <typename T> struct TileGeom {
-    static constexpr int TILE_BYTES = TILE_CHUNKS * CHUNK * (int)sizeof(T);
+    static constexpr int CHUNKS = TILE_CHUNKS * StreamCfg<T>::CPW;
+    static constexpr int TILE_BYTES = CHUNKS * CHUNK * (int)sizeof(T);
     static constexpr int SMEM_BYTES = StreamCfg<T>::STAGES * TILE_BYTES;
 };
 

@@ -140,6 +140,8 @@ __global__ void __launch_bounds__(STREAM_THREADS, StreamCfg<T>::CTAS_PER_SM) chu
                                                                              long long total_tiles) {
     extern __shared__ __align__(1024) unsigned char stage_mem[];
     constexpr int STAGES = StreamCfg<T>::STAGES;
+    constexpr int CPW = StreamCfg<T>::CPW;
+    constexpr int TCH = TileGeom<T>::CHUNKS;
     constexpr int TILE_BYTES = TileGeom<T>::TILE_BYTES;
     __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES];
     __shared__ TileDesc desc[STAGES];
@@ -186,11 +188,11 @@ __global__ void __launch_bounds__(STREAM_THREADS, StreamCfg<T>::CTAS_PER_SM) chu
             const float Tb = a.temperature[b];
             if (!temp_ok(Tb)) d.valid = 0;
             d.c32 = temp_scale(Tb);
-            d.c0 = tc * TILE_CHUNKS;
+            d.c0 = tc * TCH;
             desc[s] = d;
             if (d.valid) {
                 const int v0 = d.c0 * CHUNK;
-                const int v1 = min(a.V, v0 + TILE_CHUNKS * CHUNK);
+                const int v1 = min(a.V, v0 + TCH * CHUNK);
                 const uint32_t bytes = (uint32_t)(v1 - v0) * (uint32_t)sizeof(T);
                 const T* src = reinterpret_cast<const T*>(a.logits) + (long long)d.src_row * a.row_stride + v0;
                 mbar_arrive_expect_tx(&full[s], bytes);
@@ -212,19 +214,24 @@ __global__ void __launch_bounds__(STREAM_THREADS, StreamCfg<T>::CTAS_PER_SM) chu
             break;
         }
         const TileDesc d = desc[s];
-        const int c = d.c0 + warp;
-        const bool work = d.valid && c < a.nch;
-        ChunkRegs<T> regs;
-        if (work) load_staged(regs, stage_mem + s * TILE_BYTES + warp * (CHUNK * (int)sizeof(T)), c * CHUNK, a.V, lane);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[s]);
-        if (work) {
-            // chunk maximum with NaN ignored; a NaN (or +inf) logit turns the exp-sum into NaN by
-            // itself, which the finish kernel reports; a chunk of -inf only sums to zero
-            const float cm = warp_max_redux(regs.lane_max_plain());
-            const float off = cm > -CUDART_INF_F ? __fmul_rn(cm, d.c32) : 0.f;
-            const float sum = warp_sum(lane_exp_sum2(regs, d.c32, off));
-            if (lane == 0) a.stats[(long long)d.src_row * a.nch + c] = make_float2(cm, sum);
+#pragma unroll
+        for (int q = 0; q < CPW; ++q) {
+            const int c = d.c0 + warp * CPW + q;
+            const bool work = d.valid && c < a.nch;
+            ChunkRegs<T> regs;
+            if (work) load_staged(regs, stage_mem + s * TILE_BYTES + (warp * CPW + q) * (CHUNK * (int)sizeof(T)), c * CHUNK, a.V, lane);
+            if (q == CPW - 1) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[s]);     // the warp's chunks are in registers or done
+            }
+            if (work) {
+                // chunk maximum with NaN ignored; a NaN (or +inf) logit turns the exp-sum into NaN by
+                // itself, which the finish kernel reports; a chunk of -inf only sums to zero
+                const float cm = warp_max_redux(regs.lane_max_plain());
+                const float off = cm > -CUDART_INF_F ? __fmul_rn(cm, d.c32) : 0.f;
+                const float sum = warp_sum(lane_exp_sum2(regs, d.c32, off));
+                if (lane == 0) a.stats[(long long)d.src_row * a.nch + c] = make_float2(cm, sum);
+            }
         }
     }
 }

@@ -48,6 +48,7 @@ def run_both(ps, w, inputs, check_compress=True, nthreads=None, draft_tok_overri
     nthreads = nthreads or oracle.cores()
     B, G, V, K = w.B, w.G, w.V, w.k_max
     ctx = _ctx(ps, B, G, V, K)
+    ctx.counters(clear=True)
     dl, tl, T = inputs["draft_logits"], inputs["target_logits"], inputs["temperature"]
     sub = slice(None) if seq_subset is None else seq_subset
     # ---- oracle (on the sampled sequences) -------------------------------------------------
@@ -73,7 +74,9 @@ def run_both(ps, w, inputs, check_compress=True, nthreads=None, draft_tok_overri
         qi, qp, qc, tok = g_qi.clone(), g_qp.clone(), g_qc.clone(), g_tok.clone()
         qi[sub], qp[sub], qc[sub], tok[sub] = _cuda(o_qi), _cuda(o_qp), _cuda(o_qc), _cuda(o_tok)
     g = ctx.verify(tl, T, tok, qi, qp, qc, inputs["u_accept"], inputs["u_resample"])
+    _, redo = ctx.counters()
     st, slow = ctx.status(clear=True)
+    ctx.counters(clear=True)
     assert np.array_equal(_np(g["accept_len"][sub]), o["accept_len"]), "accept_len"
     assert np.array_equal(_np(g["token"][sub]), o["token"]), "token"
     if seq_subset is None:
@@ -84,7 +87,7 @@ def run_both(ps, w, inputs, check_compress=True, nthreads=None, draft_tok_overri
     bad = ~ok
     if bad.any():
         assert np.all(_np(g["p_draft"][sub])[bad] == -1) and np.all(_np(g["resid_mass"][sub])[bad] == -1)
-    return {"status": st, "slow_rows": slow, "oracle": o, "gpu": g}
+    return {"status": st, "slow_rows": slow, "redo_rows": redo, "oracle": o, "gpu": g}
 
 
 # ---------------------------------------------------------------------------------------------
@@ -97,6 +100,7 @@ def test_config_full_size(ps, name):
     inputs = gen.make_inputs(w, seed=1000 * int(name[-1]), device="cuda")
     r = run_both(ps, w, inputs)
     assert r["status"] == 0
+    assert r["redo_rows"] == 0          # the staged compress kernel keeps every row of the benchmark shapes
 
 
 def test_config4_full_size_launch_sampled_sequences(ps):
@@ -363,3 +367,88 @@ def test_near_threshold_uniforms_are_decided_exactly(ps):
     r = run_both(ps, w, inputs, check_compress=False)
     assert r["slow_rows"] > 0
     assert r["oracle"]["borderline_count"] > 0
+
+
+# ---------------------------------------------------------------------------------------------
+# staged kernels (16-byte aligned rows of at least one 8192-entry tile): ragged tiles, both
+# candidate-buffer shapes, and rows that overflow the filter's buffer and are redone by the
+# direct kernel
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("V,B,G,K,dtype,top_k,top_p", [
+    (8192, 3, 2, 64, "bf16", 64, 1.0),        # exactly one tile
+    (8200, 3, 2, 64, "bf16", 0, 0.9),         # one entry-vector into the second tile
+    (16392, 2, 3, 256, "bf16", 256, 1.0),     # last tile holds a single ragged chunk
+    (40960, 2, 2, 300, "bf16", 300, 1.0),     # k > 256: large candidate buffer
+    (65536, 2, 1, 1024, "bf16", 0, 0.9999),   # widest rows, top-p that never cuts
+    (12292, 2, 2, 32, "f32", 32, 1.0),        # fp32 tiles, ragged
+    (20000, 2, 2, 700, "f32", 0, 0.95),       # fp32, large buffer, top-p
+])
+def test_staged_shapes(ps, V, B, G, K, dtype, top_k, top_p):
+    w = gen.Workload("t", V=V, B=B, G=G, dtype=dtype, s=1.1, sigma_d=1.5, corr=0.8, sigma_t=1.0,
+                     T=None, top_k=top_k, top_p=top_p, k_max=K)
+    inputs = gen.make_inputs(w, seed=3 * V + K, device="cuda")
+    r = run_both(ps, w, inputs)
+    assert r["status"] == 0
+
+
+def _custom_inputs(dl, tl, seed):
+    B, G, V = dl.shape
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    return {"draft_logits": dl, "target_logits": tl, "temperature": torch.full((B,), 0.9, device="cuda"),
+            "u_draft": torch.rand((B, G), generator=g, device="cuda"),
+            "u_accept": torch.rand((B, G), generator=g, device="cuda"),
+            "u_resample": torch.rand((B, 2), generator=g, device="cuda")}
+
+
+@pytest.mark.parametrize("top_p", [1.0, 0.9])
+def test_staged_rows_that_overflow_the_filter_are_redone(ps, top_p):
+    # rows built to defeat a running threshold: all equal, heavy ties, ascending (every new value is
+    # a new maximum), descending, and mostly -inf; the oracle's order (logit desc, index asc) must
+    # come out of the redo path exactly
+    V, B, G, K = 24576, 5, 2, 48
+    base = torch.randn((G, V), device="cuda")
+    dl = torch.empty((B, G, V), dtype=torch.bfloat16, device="cuda")
+    dl[0] = 1.25
+    dl[1] = torch.randint(-2, 3, (G, V), device="cuda").to(torch.bfloat16)
+    dl[2] = (torch.arange(V, device="cuda").float() * 1e-3 - 5.0).expand(G, V).to(torch.bfloat16)
+    dl[3] = (5.0 - torch.arange(V, device="cuda").float() * 1e-3).expand(G, V).to(torch.bfloat16)
+    dl[4] = float("-inf")
+    dl[4, :, ::997] = base[:, ::997].to(torch.bfloat16)
+    tl = (0.5 * torch.randn((B, G + 1, V), device="cuda")).to(torch.bfloat16)
+    w = gen.Workload("t", V=V, B=B, G=G, dtype="bf16", s=0, sigma_d=0, corr=0, sigma_t=0, T=0.9,
+                     top_k=(K if top_p >= 1.0 else 0), top_p=top_p, k_max=K)
+    r = run_both(ps, w, _custom_inputs(dl, tl, 11))
+    assert r["status"] == 0
+    assert r["redo_rows"] >= 4 * G          # all equal, ties, ascending, mostly -inf: handed over
+
+
+def test_staged_bad_data_is_reported(ps):
+    # NaN and +inf inside rows that take the staged kernels (with and without the exp-sum)
+    V, B, G, K = 16384, 4, 1, 16
+    for top_p in (1.0, 0.9):
+        w = gen.Workload("t", V=V, B=B, G=G, dtype="bf16", s=1.1, sigma_d=1.5, corr=0.8, sigma_t=1.0, T=1.0,
+                         top_k=(K if top_p >= 1.0 else 0), top_p=top_p, k_max=K)
+        inputs = gen.make_inputs(w, seed=31, device="cuda")
+        inputs["draft_logits"][1, 0, 12345] = float("nan")
+        inputs["draft_logits"][2, 0, 8191] = float("inf")
+        inputs["target_logits"][3, 1, 9000] = float("nan")
+        ctx = _ctx(ps, B, G, V, K)
+        o_qi, o_qp, o_qc, o_tok = oracle.compress(_np(inputs["draft_logits"]), _np(inputs["temperature"]), w.top_k,
+                                                  top_p, K, _np(inputs["u_draft"]))
+        g_qi, g_qp, g_qc, g_tok = ctx.compress(inputs["draft_logits"], inputs["temperature"], w.top_k, top_p, K,
+                                               inputs["u_draft"])
+        st, _ = ctx.status(clear=True)
+        assert st == 2
+        assert np.array_equal(_np(g_qc), o_qc) and np.array_equal(_np(g_qi), o_qi) and np.array_equal(_np(g_tok), o_tok)
+        assert _np(g_qc)[1, 0] == -1 and _np(g_qc)[2, 0] == -1 and _np(g_qc)[0, 0] > 0
+        tok = np.where(o_tok < 0, 0, o_tok).astype(np.int32)
+        o = oracle.verify(_np(inputs["target_logits"]), _np(inputs["temperature"]), tok, o_qi, o_qp, o_qc,
+                          _np(inputs["u_accept"]), _np(inputs["u_resample"]))
+        g = ctx.verify(inputs["target_logits"], inputs["temperature"], _cuda(tok), g_qi, g_qp, g_qc,
+                       inputs["u_accept"], inputs["u_resample"])
+        st, _ = ctx.status(clear=True)
+        assert st & 2
+        assert np.array_equal(_np(g["accept_len"]), o["accept_len"])
+        assert np.array_equal(_np(g["token"]), o["token"])
+        assert o["accept_len"][3] == -1 and o["accept_len"][0] >= 0

@@ -14,8 +14,8 @@
 //   - every stored candidate is counted in a two-level histogram over the top 12 bits of the
 //     orderable logit; thr is the lower edge of the highest bin whose suffix count reaches k, so
 //     it is a valid bound whenever it is computed, by any warp, from whatever has been counted so
-//     far.  Warp 0 refreshes it after tiles 1, 2, 4, 8, ...; a warp whose region fills refreshes
-//     it and drops its candidates below it;
+//     far.  The warps take turns refreshing it, once per tile; a warp whose region fills
+//     refreshes it and drops its candidates below it;
 //   - the first tile of a row gets its bound without the histogram: every warp finds, by a
 //     16-step bisection over its own chunk, a value that at least ceil(k/8) of its small groups
 //     of elements reach with their maximum; the smallest of the eight values is reached by at
@@ -425,8 +425,9 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
                 __syncwarp();
                 // count the new entries in the histogram
                 for (int x = before + lane; x < wcount; x += 32) hist_add(hist, (int)(region[x] >> (32 + CS_BIN_SHIFT)));
-                // the bound is refreshed after tiles 1, 2, 4, 8, ..., each time by another warp
-                if (((ti + 1) & ti) == 0 && warp == ((31 - __clz(ti + 1)) & (WARPS - 1))) {
+                // the bound is refreshed after every tile, each time by another warp (the others'
+                // latest values may not be counted yet, which only makes it a little lower)
+                if (warp == (ti & (WARPS - 1))) {
                     __syncwarp();
                     refresh_bound(hist_off, &cs, k_eff);
                 }

@@ -354,8 +354,14 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 wt.init(Tb, sh.mx[i]);
                 const double Z = sh.Z[i];
                 double smin = 0.0;
-                float qx = 0.f;
+                float qx = 0.f, qx_mine = 0.f;
                 int kx = 0x7fffffff;
+                // issued early: the logit of the draft token and its uniform (lane 0 uses them last)
+                float lx = -CUDART_INF_F, ux = 0.f;
+                if (!range_bad && lane == 0) {
+                    lx = load_logit(row, x);
+                    ux = a.u_accept[ri];
+                }
                 if (!range_bad) {
                     const int* idx = a.q_idx + (long long)ri * a.k_max;
                     const float* prob = a.q_prob + (long long)ri * a.k_max;
@@ -381,7 +387,10 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                             if (vv[u] >= 0 && vv[u] < a.V) {
                                 const double pk = wt(ll[u]) / Z;
                                 smin += fmin(pk, (double)qq[u]);
-                                if (vv[u] == x && k < kx) kx = k;
+                                if (vv[u] == x && k < kx) {
+                                    kx = k;
+                                    qx_mine = qq[u];
+                                }
                             }
                         }
                     }
@@ -390,13 +399,15 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 smin = warp_sum(smin);
 #pragma unroll
                 for (int d = 16; d > 0; d >>= 1) kx = min(kx, __shfl_xor_sync(0xffffffffu, kx, d));
+                // the stored probability of the first entry that names the draft token sits in lane kx % 32
+                qx = __shfl_sync(0xffffffffu, qx_mine, kx & 31);
+                if (kx == 0x7fffffff) qx = 0.f;
                 if (lane == 0) {
                     if (range_bad) {
                         atomicOr(&sh.bad, (int)ST_RANGE);
                     } else {
-                        if (kx != 0x7fffffff) qx = a.q_prob[(long long)ri * a.k_max + kx];
-                        const double px = wt(load_logit(row, x)) / Z;
-                        const double u = (double)a.u_accept[ri];
+                        const double px = wt(lx) / Z;
+                        const double u = (double)ux;
                         int acc = 1, amb = 0, bord = 0;
                         if (qx > 0.f) {
                             const double ratio = px / (double)qx;

@@ -40,7 +40,8 @@ def _load():
     if _lib is None:
         # a test that plants a mistake points this at its own build of a modified copy
         _lib = ctypes.CDLL(os.environ.get("PICOSPEC_ORACLE_LIB") or build())
-        for name in ("pso_compress", "pso_verify", "pso_residual_sample", "pso_softmax"):
+        for name in ("pso_compress", "pso_verify", "pso_residual_sample", "pso_softmax", "pso_target_topk",
+                     "pso_edge_resample"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -149,6 +150,49 @@ def residual_sample(target_logits, temperature, pos, q_idx, q_prob, q_count, u_r
                                      ctypes.c_long(chunk), ctypes.c_int(nthreads))
     if rc != 0:
         raise ValueError(f"pso_residual_sample failed: {rc}")
+    return token, mass
+
+
+def target_topk(target_logits, temperature, pos, k: int, nthreads: int = 1):
+    """The paper's downlink payload (Eq. 4): target_logits fp32 [B, R, V], row pos[b] of each
+    sequence -> (p_idx [B,k] i32, p_prob [B,k] f32 raw probabilities, p_count [B] i32)."""
+    l = _f32(target_logits)
+    B, R, V = _rows(l)
+    T = _f32(temperature)
+    ps = _i32(pos)
+    assert T.shape == (B,) and ps.shape == (B,)
+    p_idx = np.empty((B, k), np.int32)
+    p_prob = np.empty((B, k), np.float32)
+    p_count = np.empty((B,), np.int32)
+    rc = _load().pso_target_topk(_p(l), ctypes.c_long(B), ctypes.c_long(R), ctypes.c_long(V), ctypes.c_long(V),
+                                 _p(T), _p(ps), ctypes.c_int(k), _p(p_idx), _p(p_prob), _p(p_count),
+                                 ctypes.c_int(nthreads))
+    if rc != 0:
+        raise ValueError(f"pso_target_topk failed: {rc}")
+    return p_idx, p_prob, p_count
+
+
+def edge_resample(draft_logits, temperature, pos, p_idx, p_prob, p_count, u, nthreads: int = 1):
+    """The paper's edge-side correction: draft_logits fp32 [B, R, V] (the drafter's own rows), row
+    pos[b]; the transmitted components (p_idx, p_prob, p_count); one uniform per sequence ->
+    (token [B] i32, mass [B] f64)."""
+    l = _f32(draft_logits)
+    B, R, V = _rows(l)
+    T = _f32(temperature)
+    ps = _i32(pos)
+    pi = _i32(p_idx)
+    pp = _f32(p_prob)
+    pc = _i32(p_count)
+    uu = _f32(u)
+    k = pi.shape[-1]
+    assert pi.shape == (B, k) and pp.shape == (B, k) and pc.shape == (B,) and uu.shape == (B,) and ps.shape == (B,)
+    token = np.empty((B,), np.int32)
+    mass = np.empty((B,), np.float64)
+    rc = _load().pso_edge_resample(_p(l), ctypes.c_long(B), ctypes.c_long(R), ctypes.c_long(V), ctypes.c_long(V),
+                                   _p(T), _p(ps), _p(pi), _p(pp), _p(pc), ctypes.c_int(k), _p(uu), _p(token),
+                                   _p(mass), ctypes.c_int(nthreads))
+    if rc != 0:
+        raise ValueError(f"pso_edge_resample failed: {rc}")
     return token, mass
 
 

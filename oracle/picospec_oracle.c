@@ -23,6 +23,10 @@
  * Where the paper is silent the reading is stated next to the code (top-p,
  * renormalisation, tie-break, temperature, bonus row, two-level inverse CDF).
  *
+ *   - Sec. 3.3 read literally (pso_target_topk, pso_edge_resample): the verifier sends the K
+ *     largest components of the TARGET distribution at the rejected position, unnormalised,
+ *     and the edge resamples from norm(max(0, P~ - Q)) against its own dense row.
+ *
  * Pins (tests/test_oracle_pins.py): library top-k + softmax closed form, sum-to-one
  * and support invariants, q~ = p special case, brute-force output law on tiny
  * vocabularies, residual-mass identity, K = 1 textbook reduction, payload sizes
@@ -460,6 +464,142 @@ int pso_residual_sample(const float *target_logits, long B, long G, long V, long
         }
         free(w);
         free(qd);
+        free(r);
+    }
+    return err ? PSO_ENOMEM : PSO_OK;
+}
+
+/* ---- the paper's own direction (Sec. 3.3): Top-K of the target row on the verifier, ---------
+ * ---- resampling against the drafter's dense row on the edge ------------------------------- */
+
+/* Eq. (4): P_sent = the K components of the target distribution P_j with the highest
+ * probabilities, with their vocabulary indices.  The probabilities are sent as they are (the
+ * paper does not renormalise them).  Row j = pos[b] of sequence b's `rows_per_seq` rows.
+ * Order and tie-break as everywhere: logit descending, index ascending.
+ * p_count[b] = min(k, V), or -1 (ids -1, probabilities 0) for an unusable row / position. */
+int pso_target_topk(const float *target_logits, long B, long rows_per_seq, long V, long row_stride,
+                    const float *temperature, const int *pos, int k, int *p_idx, float *p_prob,
+                    int *p_count, int nthreads) {
+    if (!target_logits || !temperature || !pos || !p_idx || !p_prob || !p_count) return PSO_EINVAL;
+    if (B < 0 || rows_per_seq <= 0 || V <= 0 || k <= 0 || row_stride < V) return PSO_EINVAL;
+    if (nthreads < 1) nthreads = 1;
+    int err = 0;
+#pragma omp parallel num_threads(nthreads)
+    {
+        double *w = (double *)malloc((size_t)V * sizeof(double));
+        pso_key *keys = (pso_key *)malloc((size_t)V * sizeof(pso_key));
+        if (!w || !keys) {
+#pragma omp atomic write
+            err = 1;
+        }
+#pragma omp barrier
+        if (!err) {
+#pragma omp for schedule(dynamic, 1)
+            for (long b = 0; b < B; ++b) {
+                int *idx = p_idx + b * k;
+                float *prob = p_prob + b * k;
+                for (int j = 0; j < k; ++j) {
+                    idx[j] = -1;
+                    prob[j] = 0.0f;
+                }
+                p_count[b] = -1;
+                long j = pos[b];
+                double T = (double)temperature[b], Z;
+                if (j < 0 || j >= rows_per_seq || !pso_temperature_ok(T)) continue;
+                const float *l = target_logits + (b * rows_per_seq + j) * row_stride;
+                if (pso_softmax_row(l, V, T, w, &Z)) continue;
+                for (long v = 0; v < V; ++v) {
+                    keys[v].l = l[v];
+                    keys[v].v = (int)v;
+                }
+                qsort(keys, (size_t)V, sizeof(pso_key), pso_key_cmp);
+                long n = k < V ? k : V;
+                for (long t = 0; t < n; ++t) {
+                    idx[t] = keys[t].v;
+                    prob[t] = (float)(w[keys[t].v] / Z);
+                }
+                p_count[b] = (int)n;
+            }
+        }
+        free(w);
+        free(keys);
+    }
+    return err ? PSO_ENOMEM : PSO_OK;
+}
+
+/* Sec. 3.3: "the edge then autonomously performs local resampling using the logic
+ * norm(max(0, P_j(x) - Q_j(x)))".  The edge holds its own dense distribution Q_j = softmax of
+ * its logits at the rejected position j = pos[b], and the K transmitted components of P_j; a
+ * component that was not transmitted counts as zero, so only the K transmitted indices can carry
+ * positive weight (reading: the paper does not say what the edge assumes about the rest):
+ *   r_t = max(0, p_prob[t] - Q_j(p_idx[t])),  R = sum_t r_t  (stored order)
+ *   token = p_idx[first t with sum_{t' <= t} r_t' > u * R], else the last t with r_t > 0
+ * If R = 0 (Q_j covers every transmitted component) the draw is from the transmitted components
+ * themselves, r_t = p_prob[t] (reading; the paper is silent).  mass[b] = R of the weights drawn from.
+ * Unusable input (temperature, position, count or index out of range, NaN / +inf logits):
+ * token = -1, mass = -1. */
+int pso_edge_resample(const float *draft_logits, long B, long rows_per_seq, long V, long row_stride,
+                      const float *temperature, const int *pos, const int *p_idx, const float *p_prob,
+                      const int *p_count, int k, const float *u, int *token, double *mass, int nthreads) {
+    if (!draft_logits || !temperature || !pos || !p_idx || !p_prob || !p_count || !u || !token) return PSO_EINVAL;
+    if (B < 0 || rows_per_seq <= 0 || V <= 0 || k <= 0 || row_stride < V) return PSO_EINVAL;
+    if (nthreads < 1) nthreads = 1;
+    int err = 0;
+#pragma omp parallel num_threads(nthreads)
+    {
+        double *w = (double *)malloc((size_t)V * sizeof(double));
+        double *r = (double *)malloc((size_t)k * sizeof(double));
+        if (!w || !r) {
+#pragma omp atomic write
+            err = 1;
+        }
+#pragma omp barrier
+        if (!err) {
+#pragma omp for schedule(dynamic, 1)
+            for (long b = 0; b < B; ++b) {
+                token[b] = -1;
+                if (mass) mass[b] = -1.0;
+                long j = pos[b];
+                int n = p_count[b];
+                double T = (double)temperature[b], Z;
+                if (j < 0 || j >= rows_per_seq || n <= 0 || n > k || !pso_temperature_ok(T)) continue;
+                const int *idx = p_idx + b * k;
+                const float *prob = p_prob + b * k;
+                int bad = 0;
+                for (int t = 0; t < n; ++t)
+                    if (idx[t] < 0 || idx[t] >= V) bad = 1;
+                if (bad) continue;
+                const float *l = draft_logits + (b * rows_per_seq + j) * row_stride;
+                if (pso_softmax_row(l, V, T, w, &Z)) continue;
+                double R = 0.0;
+                for (int t = 0; t < n; ++t) {
+                    double d = (double)prob[t] - w[idx[t]] / Z;
+                    r[t] = d > 0.0 ? d : 0.0;
+                    R += r[t];
+                }
+                if (!(R > 0.0)) {
+                    R = 0.0;
+                    for (int t = 0; t < n; ++t) {
+                        r[t] = (double)prob[t];
+                        R += r[t];
+                    }
+                }
+                double thr = (double)u[b] * R, cum = 0.0;
+                int pick = -1, last = -1;
+                for (int t = 0; t < n; ++t) {
+                    if (r[t] > 0.0) last = t;
+                    cum += r[t];
+                    if (cum > thr) {
+                        pick = t;
+                        break;
+                    }
+                }
+                if (pick < 0) pick = last;
+                token[b] = pick >= 0 ? idx[pick] : -1;
+                if (mass) mass[b] = R;
+            }
+        }
+        free(w);
         free(r);
     }
     return err ? PSO_ENOMEM : PSO_OK;

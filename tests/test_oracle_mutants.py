@@ -37,6 +37,15 @@ MUTANTS = [
     ("sample_wrong_row", "long t = pso_sample_row(rows + a * row_stride,", "long t = pso_sample_row(rows + 0 * row_stride,"),
     ("px_wrong_index", "double px = w[x] / Z;", "double px = w[(x + 1) % V] / Z;"),
     ("draw_nonstrict", "if (cum > thr) return idx[j];", "if (cum >= thr * 1.3) return idx[j];"),
+    ("topk_renormalised", "prob[t] = (float)(w[keys[t].v] / Z);", "prob[t] = (float)(w[keys[t].v] / Z * 1.5);"),
+    ("topk_wrong_row", "const float *l = target_logits + (b * rows_per_seq + j) * row_stride;",
+     "const float *l = target_logits + (b * rows_per_seq + 0) * row_stride;"),
+    ("edge_residual_sign", "double d = (double)prob[t] - w[idx[t]] / Z;", "double d = w[idx[t]] / Z - (double)prob[t];"),
+    ("edge_ignores_q", "double d = (double)prob[t] - w[idx[t]] / Z;", "double d = (double)prob[t];"),
+    ("edge_wrong_row", "const float *l = draft_logits + (b * rows_per_seq + j) * row_stride;",
+     "const float *l = draft_logits + (b * rows_per_seq + 0) * row_stride;"),
+    ("edge_nonstrict", "if (cum > thr) {\n                        pick = t;", "if (cum >= thr * 1.2) {\n                        pick = t;"),
+    ("edge_no_fallback", "if (!(R > 0.0)) {\n                    R = 0.0;", "if (0) {\n                    R = 0.0;"),
 ]
 
 PINS = os.path.join(os.path.dirname(os.path.abspath(__file__)), "test_oracle_pins.py")

@@ -436,3 +436,163 @@ def test_invalid_inputs_are_flagged_not_sampled():
     for b in (1, 2, 3):           # bad count / +inf logit / zero temperature
         assert r["accept_len"][b] == -1 and r["token"][b] == -1
         assert np.all(r["p_draft"][b] == -1) and np.all(r["resid_mass"][b] == -1)
+
+
+# ---------------------------------------------------------------------------------------------
+# The paper's own direction (Sec. 3.3): Top-K of the target row on the verifier (Eq. 4),
+# resampling against the drafter's dense row on the edge
+# ---------------------------------------------------------------------------------------------
+
+def test_target_topk_is_library_softmax_at_the_k_largest_logits():
+    # Eq. (4): the K components with the highest probabilities and their indices, unnormalised
+    rng = _rng(101)
+    B, R, V, K = 5, 3, 97, 7
+    l = rng.normal(size=(B, R, V)).astype(np.float32) * 2
+    l[2, 1, 10] = l[2, 1, 3] = l[2, 1, 50] = 40.0         # ties: lower index first
+    T = rng.uniform(0.5, 1.5, size=B).astype(np.float32)
+    pos = np.array([0, 2, 1, 1, 0], np.int32)
+    pi, pp, pc = oracle.target_topk(l, T, pos, K)
+    for b in range(B):
+        row = l[b, pos[b]].astype(np.float64)
+        p = sp_softmax(row / np.float64(T[b]))
+        order = np.lexsort((np.arange(V), -row))[:K]
+        assert list(pi[b]) == list(order) and pc[b] == K
+        np.testing.assert_allclose(pp[b], p[order], rtol=2e-7)
+        assert pp[b].sum() < 1.0
+    assert list(pi[2, :3]) == [3, 10, 50]
+    # K >= V: the whole distribution, summing to one
+    pi, pp, pc = oracle.target_topk(l, T, pos, V + 5)
+    assert np.all(pc == V) and np.all(pi[:, V:] == -1) and np.all(pp[:, V:] == 0)
+    np.testing.assert_allclose(pp.astype(np.float64).sum(1), 1.0, atol=1e-6)
+    # a position outside the sequence's rows and a bad temperature are flagged
+    T2 = T.copy()
+    T2[1] = -1.0
+    pi, pp, pc = oracle.target_topk(l, T2, np.array([0, 2, 3, 1, -1], np.int32), K)
+    assert list(pc) == [K, -1, -1, K, -1] and np.all(pi[1] == -1)
+
+
+def _edge_reference(draft_row, T, idx, prob, u):
+    """norm(max(0, P~ - Q)) over the transmitted components, flat inverse CDF, by library calls."""
+    q = sp_softmax(draft_row.astype(np.float64) / np.float64(T))
+    r = np.maximum(0.0, prob.astype(np.float64) - q[idx])
+    if not r.sum() > 0:
+        r = prob.astype(np.float64)
+    cum = np.cumsum(r)
+    t = int(np.searchsorted(cum, np.float64(u) * cum[-1], side="right"))      # first cum > u * R
+    if t >= len(r):
+        t = int(np.nonzero(r > 0)[0][-1])
+    return int(idx[t]), float(cum[-1])
+
+
+def test_edge_resample_is_the_formula_of_sec_3_3_over_the_transmitted_components():
+    rng = _rng(103)
+    B, R, V, K = 6, 2, 64, 9
+    lt = rng.normal(size=(B, R, V)).astype(np.float32) * 2
+    ld = (0.6 * lt + rng.normal(size=(B, R, V))).astype(np.float32)
+    T = rng.uniform(0.6, 1.3, size=B).astype(np.float32)
+    pos = rng.integers(0, R, size=B).astype(np.int32)
+    pi, pp, pc = oracle.target_topk(lt, T, pos, K)
+    for u in np.linspace(0.0, 0.999, 41, dtype=np.float32):
+        tok, mass = oracle.edge_resample(ld, T, pos, pi, pp, pc, np.full(B, u, np.float32))
+        for b in range(B):
+            t_ref, m_ref = _edge_reference(ld[b, pos[b]], T[b], pi[b], pp[b], u)
+            assert tok[b] == t_ref
+            assert abs(mass[b] - m_ref) <= 1e-12 * max(1.0, m_ref)
+            assert tok[b] in pi[b]                      # only transmitted components can be drawn
+
+
+def test_edge_resample_law_and_zero_weight_entries():
+    # the measure of u that maps to a component equals r_t / R; components with P~ <= Q are never drawn
+    rng = _rng(107)
+    V, K = 12, 12
+    lt = rng.normal(size=(1, 1, V)).astype(np.float32) * 1.5
+    ld = rng.normal(size=(1, 1, V)).astype(np.float32) * 1.5
+    T = np.ones(1, np.float32)
+    pos = np.zeros(1, np.int32)
+    pi, pp, pc = oracle.target_topk(lt, T, pos, K)
+    q = sp_softmax(ld[0, 0].astype(np.float64))
+    r = np.maximum(0.0, pp[0].astype(np.float64) - q[pi[0]])
+    N = 20000
+    counts = np.zeros(V)
+    us = ((np.arange(N) + 0.5) / N).astype(np.float32)
+    for u in us:
+        tok, _ = oracle.edge_resample(ld, T, pos, pi, pp, pc, np.array([u], np.float32))
+        counts[tok[0]] += 1
+    law = np.zeros(V)
+    law[pi[0]] = r / r.sum()
+    np.testing.assert_allclose(counts / N, law, atol=2.0 / N + 1e-6)
+    assert np.all(counts[pi[0][r == 0]] == 0)
+
+
+def test_edge_resample_falls_back_to_the_transmitted_components_when_q_covers_them():
+    V, K = 8, 3
+    ld = np.zeros((1, 1, V), np.float32)
+    ld[0, 0, :3] = 5.0                                   # Q puts ~1/3 on each of ids 0, 1, 2
+    T = np.ones(1, np.float32)
+    pos = np.zeros(1, np.int32)
+    pi = np.array([[0, 1, 2]], np.int32)
+    pp = np.array([[0.2, 0.1, 0.05]], np.float32)        # all below Q: residual identically zero
+    pc = np.array([3], np.int32)
+    seen = set()
+    for u in np.linspace(0.0, 0.999, 50, dtype=np.float32):
+        tok, mass = oracle.edge_resample(ld, T, pos, pi, pp, pc, np.array([u], np.float32))
+        seen.add(int(tok[0]))
+        assert abs(mass[0] - 0.35) < 1e-6
+    assert seen == {0, 1, 2}
+    tok, _ = oracle.edge_resample(ld, T, pos, pi, pp, pc, np.array([0.5], np.float32))
+    assert tok[0] == 0                                   # cum 0.2 > 0.5 * 0.35
+    tok, _ = oracle.edge_resample(ld, T, pos, pi, pp, pc, np.array([0.6], np.float32))
+    assert tok[0] == 1
+
+
+def test_scalar_uplink_plus_edge_resample_with_full_downlink_reproduces_the_target_law():
+    # Sec. 3.3 with K = V (nothing truncated): the drafter samples x ~ Q and sends q(x) only; the
+    # verifier accepts with min(1, p(x)/q(x)); on rejection the edge resamples from
+    # norm(max(0, P - Q)).  The output law must be P (Sec. 2.1).  Exact enumeration over x, the
+    # accept probability integrated analytically, the edge law measured on a uniform grid.
+    rng = _rng(109)
+    V = 10
+    lt = rng.normal(size=(1, 2, V)).astype(np.float32) * 1.5
+    ld = (0.5 * lt[:, :1] + rng.normal(size=(1, 1, V))).astype(np.float32)
+    T = np.array([0.9], np.float32)
+    p = sp_softmax(lt[0, 0].astype(np.float64) / np.float64(T[0]))
+    q = sp_softmax(ld[0, 0].astype(np.float64) / np.float64(T[0]))
+    # the verifier's accept test with the scalar q(x): K = 1 sparse rows holding (x, q(x))
+    acc_prob = np.zeros(V)
+    for x in range(V):
+        qi = np.array([[[x]]], np.int32)
+        qp = np.array([[[q[x]]]], np.float32)
+        qc = np.array([[1]], np.int32)
+        tok = np.array([[x]], np.int32)
+        us = np.linspace(0.0, 0.9999, 2001, dtype=np.float32)
+        acc = [oracle.verify(lt, T, tok, qi, qp, qc, np.array([[u]], np.float32))["accept_len"][0] for u in us]
+        acc_prob[x] = np.mean(acc)
+        assert abs(acc_prob[x] - min(1.0, p[x] / q[x])) < 2e-3
+    # the edge's law with everything transmitted
+    pos = np.zeros(1, np.int32)
+    pi, pp, pc = oracle.target_topk(lt, T, pos, V)
+    N = 20000
+    edge = np.zeros(V)
+    for u in ((np.arange(N) + 0.5) / N).astype(np.float32):
+        tok, _ = oracle.edge_resample(ld, T, pos, pi, pp, pc, np.array([u], np.float32))
+        edge[tok[0]] += 1.0 / N
+    out = q * np.minimum(1.0, p / q) + (1.0 - np.sum(np.minimum(p, q))) * edge
+    np.testing.assert_allclose(out, p, atol=5e-4)
+
+
+def test_edge_resample_flags_unusable_input():
+    rng = _rng(113)
+    B, R, V, K = 5, 2, 20, 4
+    lt = rng.normal(size=(B, R, V)).astype(np.float32)
+    ld = rng.normal(size=(B, R, V)).astype(np.float32)
+    T = np.ones(B, np.float32)
+    pos = np.zeros(B, np.int32)
+    pi, pp, pc = oracle.target_topk(lt, T, pos, K)
+    ld[1, 0, 7] = np.nan
+    pi[2, 1] = V
+    pc[3] = K + 1
+    pos2 = pos.copy()
+    pos2[4] = R
+    tok, mass = oracle.edge_resample(ld, T, pos2, pi, pp, pc, np.full(B, 0.5, np.float32))
+    assert tok[0] >= 0 and mass[0] > 0
+    assert list(tok[1:]) == [-1, -1, -1, -1] and np.all(mass[1:] == -1)

@@ -458,7 +458,7 @@ def test_target_topk_is_library_softmax_at_the_k_largest_logits():
         order = np.lexsort((np.arange(V), -row))[:K]
         assert list(pi[b]) == list(order) and pc[b] == K
         np.testing.assert_allclose(pp[b], p[order], rtol=2e-7)
-        assert pp[b].sum() < 1.0
+        assert pp[b].astype(np.float64).sum() <= 1.0 + 1e-6
     assert list(pi[2, :3]) == [3, 10, 50]
     # K >= V: the whole distribution, summing to one
     pi, pp, pc = oracle.target_topk(l, T, pos, V + 5)

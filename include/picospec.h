@@ -178,6 +178,48 @@ PICOSPEC_API int picospec_residual_sample(picospec_ctx* ctx, const void* target_
                              const int* q_idx, const float* q_prob, const int* q_count, int k_max,
                              const float* u_resample, int* token, float* mass, void* cuda_stream);
 
+/* The paper's own data flow, verifier side -- Sec. 3.3, Eq. (4): "the cloud extracts only the K
+ * components with the highest probabilities and their corresponding indices" of the target
+ * distribution at the rejected position, and sends them.
+ *
+ * For every sequence b, row j = pos[b] of target_logits [B, R, V] (R rows per sequence):
+ *   p      = softmax(logits / temperature[b])
+ *   order  = vocabulary sorted by (logit descending, index ascending)
+ *   p_idx[b,t] = order[t], p_prob[b,t] = p[order[t]] for t < n = min(k, V)  (NOT renormalised: the
+ *                paper sends the components as they are); -1 and 0 beyond n; p_count[b] = n
+ * A sequence with bad data (temperature, position outside [0, R), NaN / +inf logits) gets
+ * p_count = -1, p_idx = -1, p_prob = 0 and sets the status word.
+ * The usual verifier call before it is picospec_verify with one-entry sparse rows holding the
+ * drafted token and the scalar q(x) the edge sent (k_max = 1), without the fused sample.
+ *
+ * pos [B] int32 in [0, R); p_idx, p_prob [B, k]; p_count [B]; k <= the context's max_k, R - 1 <= its
+ * max_gamma. */
+PICOSPEC_API int picospec_target_topk(picospec_ctx* ctx, const void* target_logits, picospec_dtype dtype, int B, int R,
+                         int V, long long row_stride_elems, const float* temperature, const int* pos, int k,
+                         int* p_idx, float* p_prob, int* p_count, void* cuda_stream);
+
+/* The paper's own data flow, edge side -- Sec. 3.3: "the edge then autonomously performs local
+ * resampling using the logic norm(max(0, P_j(x) - Q_j(x)))".
+ *
+ * For every sequence b, with Q = softmax(draft_logits[b, pos[b], :] / temperature[b]) (the edge's own
+ * dense row) and the transmitted components (p_idx, p_prob, p_count) of the target distribution
+ * (a component that was not transmitted counts as zero, so only transmitted indices can be drawn):
+ *   r_t = max(0, p_prob[b,t] - Q(p_idx[b,t])),  R = sum_t r_t                      (stored order)
+ *   token[b] = p_idx[b, first t whose running sum of r exceeds u[b] * R]  (else the last t with r_t > 0)
+ *   if R = 0 (Q covers every transmitted component) the draw is from p_prob itself
+ *   mass[b] (optional) = the total of the weights drawn from
+ * Bad data (temperature, position, count or index out of range, NaN / +inf logits): token = -1,
+ * mass = -1, status word set.  Unlike picospec_residual_sample this is not an exact sampler of the
+ * true residual unless every component was transmitted (k >= V): it is the truncation the paper
+ * proposes.
+ *
+ * draft_logits [B, R, V]; pos [B] in [0, R); p_idx, p_prob [B, k]; p_count [B] in [1, k];
+ * u [B] fp32 in [0,1); token [B]; mass [B] fp32 or NULL. */
+PICOSPEC_API int picospec_edge_resample(picospec_ctx* ctx, const void* draft_logits, picospec_dtype dtype, int B, int R,
+                           int V, long long row_stride_elems, const float* temperature, const int* pos,
+                           const int* p_idx, const float* p_prob, const int* p_count, int k, const float* u,
+                           int* token, float* mass, void* cuda_stream);
+
 /* Verification without any allocation -- the paper has no counterpart; this entry point exists
  * for callers that cannot obtain device memory at all.  Two kinds of caller are meant: a plugin
  * inside a serving engine that has already claimed the whole of the GPU's memory for its own

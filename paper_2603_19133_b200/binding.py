@@ -44,6 +44,11 @@ def lib() -> ctypes.CDLL:
                                                c_int, vp, vp, vp, vp]
         L.picospec_profile_enable.argtypes = [vp, c_int]
         L.picospec_profile_read.argtypes = [vp, c_int, ctypes.POINTER(c_f), ctypes.POINTER(c_int), vp]
+        L.picospec_target_topk.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, c_int, vp, vp, vp, vp]
+        L.picospec_target_topk.restype = c_int
+        L.picospec_edge_resample.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp, c_int,
+                                             vp, vp, vp, vp]
+        L.picospec_edge_resample.restype = c_int
         L.picospec_counters.argtypes = [vp, ctypes.POINTER(c_ll), c_int, vp]
         L.picospec_counters.restype = c_int
         L.picospec_verify_static.argtypes = [vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp, c_int,
@@ -229,6 +234,34 @@ class Context:
             _ptr(out["borderline_count"], torch.int32, (1,)), _ptr(u_resample, torch.float32, (B, 2)),
             _ptr(out["token"], torch.int32, (B,)), _stream()), "picospec_verify")
         return out
+
+    # -- the paper's own data flow (Sec. 3.3) ---------------------------------------------------
+    def target_topk(self, target_logits: torch.Tensor, temperature: torch.Tensor, pos: torch.Tensor, k: int):
+        """picospec_target_topk.  Returns (p_idx [B,k] i32, p_prob [B,k] f32 unnormalised, p_count [B] i32)."""
+        p, dt, B, R, V, pitch = _logits(target_logits)
+        dev = target_logits.device
+        p_idx = torch.empty((B, k), dtype=torch.int32, device=dev)
+        p_prob = torch.empty((B, k), dtype=torch.float32, device=dev)
+        p_count = torch.empty((B,), dtype=torch.int32, device=dev)
+        _check(lib().picospec_target_topk(
+            self._h, p, dt, B, R, V, pitch, _ptr(temperature, torch.float32, (B,)), _ptr(pos, torch.int32, (B,)),
+            int(k), _ptr(p_idx), _ptr(p_prob), _ptr(p_count), _stream()), "picospec_target_topk")
+        return p_idx, p_prob, p_count
+
+    def edge_resample(self, draft_logits: torch.Tensor, temperature: torch.Tensor, pos: torch.Tensor,
+                      p_idx: torch.Tensor, p_prob: torch.Tensor, p_count: torch.Tensor, u: torch.Tensor,
+                      want_mass: bool = True):
+        """picospec_edge_resample.  Returns (token [B] i32, mass [B] f32 or None)."""
+        p, dt, B, R, V, pitch = _logits(draft_logits)
+        k = p_idx.shape[-1]
+        dev = draft_logits.device
+        token = torch.empty((B,), dtype=torch.int32, device=dev)
+        mass = torch.empty((B,), dtype=torch.float32, device=dev) if want_mass else None
+        _check(lib().picospec_edge_resample(
+            self._h, p, dt, B, R, V, pitch, _ptr(temperature, torch.float32, (B,)), _ptr(pos, torch.int32, (B,)),
+            _ptr(p_idx, torch.int32, (B, k)), _ptr(p_prob, torch.float32, (B, k)), _ptr(p_count, torch.int32, (B,)),
+            int(k), _ptr(u, torch.float32, (B,)), _ptr(token), _ptr(mass), _stream()), "picospec_edge_resample")
+        return token, mass
 
     # -- half 2b ---------------------------------------------------------------------
     def residual_sample(self, target_logits: torch.Tensor, temperature: torch.Tensor, pos: torch.Tensor,

@@ -40,10 +40,23 @@ struct CompressArgs {
     int* redo_count_next;      // cleared for the next call
     int use_redo_list;         // direct kernel: 1 = process redo_rows[0 .. *redo_count) only
     unsigned long long* redo_total;   // cumulative number of rows handed over (reported by picospec_counters)
+    // Top-K of selected rows (picospec_target_topk): output row r reads logits row
+    // r * seq_rows + row_pos[r]; probabilities are emitted as they are (divided by the row's
+    // normaliser, not by the mass of the kept entries)
+    const int* row_pos;        // or null: output row r reads logits row r
+    int seq_rows;
+    int raw_probs;
     // staged path: survivors of the filter kernel, [B*G, cs_survivor_cap(k_max)] keys + one record per row
     unsigned long long* surv_keys;
     CsRowMeta* surv_meta;
 };
+
+// logits row behind output row `row`, or -1 if its position is out of range
+__device__ __forceinline__ long long source_row(const CompressArgs& a, int row) {
+    if (!a.row_pos) return row;
+    const int j = a.row_pos[row];
+    return (j < 0 || j >= a.seq_rows) ? -1 : (long long)row * a.seq_rows + j;
+}
 
 // Monotone map float -> uint32 (larger float, larger key); -0 is folded onto +0 so that the two
 // zeros tie as they do under a floating-point comparison.
@@ -263,7 +276,7 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
         const int j = tid * 4 + e;
-        pf[e] = j < n ? (float)(w[e] / Wn) : 0.f;
+        pf[e] = j < n ? (float)(w[e] / (a.raw_probs ? Z : Wn)) : 0.f;
         ploc += (double)pf[e];
         pcum[e] = ploc;
     }
@@ -345,7 +358,13 @@ __global__ void __launch_bounds__(THREADS, 2) compress_kernel(CompressArgs a) {
             continue;
         }
         const float c32 = temp_scale(Tb);
-        const T* rowp = reinterpret_cast<const T*>(a.logits) + (long long)row * a.row_stride;
+        const long long srow = source_row(a, row);
+        if (srow < 0) {
+            emit_invalid_row(a, row);
+            if (tid == 0) atomicOr(a.status, ST_RANGE);
+            continue;
+        }
+        const T* rowp = reinterpret_cast<const T*>(a.logits) + srow * a.row_stride;
         if (tid == 0) {
             sh.count = 0;
             sh.thr = -CUDART_INF_F;

@@ -49,7 +49,7 @@ constexpr int CS_SUPER = CS_BINS / 32;
 constexpr int CS_HIST_WORDS = CS_BINS / 2 + CS_SUPER;
 
 // row flags written by the filter kernel
-constexpr int CSF_TEMPERATURE = 1, CSF_LOGIT = 2, CSF_REDO = 4, CSF_ABORT = 8;
+constexpr int CSF_TEMPERATURE = 1, CSF_LOGIT = 2, CSF_REDO = 4, CSF_ABORT = 8, CSF_RANGE = 16;
 
 struct CsRowMeta {
     int count;        // survivors written for the row
@@ -303,8 +303,9 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
         const uint64_t pol = l2_evict_first_policy();
         uint32_t i = 0;
         for (int row = blockIdx.x; row < rows; row += gridDim.x) {
-            const bool valid = temp_ok(a.temperature[row / a.G]);
-            const T* rowp = reinterpret_cast<const T*>(a.logits) + (long long)row * a.row_stride;
+            const long long srow = source_row(a, row);
+            const bool valid = temp_ok(a.temperature[row / a.G]) && srow >= 0;
+            const T* rowp = reinterpret_cast<const T*>(a.logits) + (srow < 0 ? 0 : srow) * a.row_stride;
             for (int ti = 0; ti < tiles_per_row; ++ti, ++i) {
                 const int s = (int)(i % STAGES);
                 const uint32_t round = i / STAGES;
@@ -341,7 +342,8 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
     for (int row = blockIdx.x; row < rows; row += gridDim.x) {
         const int b = row / a.G;
         const float Tb = a.temperature[b];
-        const bool valid = temp_ok(Tb);
+        const bool in_range = source_row(a, row) >= 0;
+        const bool valid = temp_ok(Tb) && in_range;
         const float c32 = temp_scale(Tb);
         float ref_off = 0.f, acc = 0.f;
         int wcount = 0;             // candidates in this warp's region
@@ -461,6 +463,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
             int flags = 0;
             const int m = cs.m;
             if (cs.abort) flags = CSF_ABORT;
+            else if (!in_range) flags = CSF_RANGE;
             else if (!valid) flags = CSF_TEMPERATURE;
             else if (cs.overflow || m > surv_cap) flags = CSF_REDO;      // too many candidates or ties at the bound
             else if (cs.nan) flags = CSF_LOGIT;
@@ -508,8 +511,8 @@ __global__ void __launch_bounds__(THREADS) compress_finish_kernel(CompressArgs a
     if (meta.flags & CSF_REDO) return;                 // the direct kernel writes this row
     if (meta.flags) {
         emit_invalid_row(a, row);
-        if (tid == 0 && (meta.flags & (CSF_TEMPERATURE | CSF_LOGIT)))
-            atomicOr(a.status, (meta.flags & CSF_TEMPERATURE) ? ST_TEMPERATURE : ST_LOGIT);
+        if (tid == 0 && (meta.flags & (CSF_TEMPERATURE | CSF_LOGIT | CSF_RANGE)))
+            atomicOr(a.status, (meta.flags & CSF_TEMPERATURE) ? ST_TEMPERATURE : (meta.flags & CSF_RANGE) ? ST_RANGE : ST_LOGIT);
         return;
     }
     const int m = meta.count;

@@ -11,6 +11,7 @@
 #include "compress_kernels.cuh"
 #include "compress_stream_kernel.cuh"
 #include "verify_kernels.cuh"
+#include "edge_kernels.cuh"
 
 using namespace picospec;
 
@@ -134,7 +135,7 @@ template <typename T>
 cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool aligned, cudaStream_t s) {
     const int rows = a.B * a.G;
     const int grid = rows < ctx->num_sms * 2 ? rows : ctx->num_sms * 2;
-    const bool stats = a.top_p < 1.0f;
+    const bool stats = a.top_p < 1.0f || a.raw_probs;     // raw probabilities need the normaliser too
     // staged kernel: 16-byte aligned rows of at least one full tile
     const bool staged = aligned && ((size_t)a.V * sizeof(T)) % 16 == 0 && a.V >= TILE_CHUNKS * CHUNK;
     if (staged) {
@@ -194,7 +195,7 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
 }
 
 template <typename T>
-cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, cudaStream_t s) {
+cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, cudaStream_t s, bool edge = false) {
     const long long items = (long long)(a.sample_only ? a.B : a.B * (a.G + 1)) * a.nch;
     long long want = (items + WARPS - 1) / WARPS;
     const int cap = ctx->num_sms * 4;
@@ -219,7 +220,8 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
     const size_t dyn = (size_t)a.nch * sizeof(double);
     {
         ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_FINISH, 2, s);
-        verify_finish_kernel<T, false><<<a.B, THREADS, dyn, s>>>(a);
+        if (edge) edge_finish_kernel<T, false><<<a.B, THREADS, 0, s>>>(a);
+        else verify_finish_kernel<T, false><<<a.B, THREADS, dyn, s>>>(a);
     }
     ProfScope ps3(ctx, PICOSPEC_PROF_VERIFY_PRECISE, 2, s);
     PreciseArgs p;
@@ -230,8 +232,26 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
     p.row_max = a.row_max; p.dsum = a.dsum;
     precise_chunk_sums_kernel<T><<<ctx->num_sms * 6, THREADS, 0, s>>>(p);
     const int g2 = a.B < ctx->num_sms ? a.B : ctx->num_sms;
-    verify_finish_kernel<T, true><<<g2, THREADS, dyn, s>>>(a);
+    if (edge) edge_finish_kernel<T, true><<<g2, THREADS, 0, s>>>(a);
+    else verify_finish_kernel<T, true><<<g2, THREADS, dyn, s>>>(a);
     return cudaGetLastError();
+}
+
+// workspace pointers and the alternating counters of one compress-type call
+void fill_compress_workspace(picospec_ctx* ctx, CompressArgs& a) {
+    a.row_max = ctx->row_max; a.dsum = ctx->dsum; a.queue = ctx->queue;
+    const int cur = 1 + (int)(ctx->compress_calls & 1ull);
+    a.queue_count = ctx->counters + cur;
+    a.queue_count_next = ctx->counters + (3 - cur);
+    a.redo_rows = ctx->redo_rows;
+    a.redo_count = ctx->counters + 2 + cur;           // [3] / [4]
+    a.redo_count_next = ctx->counters + 2 + (3 - cur);
+    a.use_redo_list = 0;
+    a.redo_total = ctx->slow_rows + 1;
+    a.surv_keys = ctx->surv_keys;
+    a.surv_meta = ctx->surv_meta;
+    ctx->compress_calls++;
+    a.status = ctx->status; a.slow_rows = ctx->slow_rows;
 }
 
 int check_common(const picospec_ctx* ctx, const void* logits, int dtype, int B, int G, int V, long long row_stride,
@@ -419,19 +439,8 @@ int picospec_compress(picospec_ctx* ctx, const void* draft_logits, picospec_dtyp
     a.B = B; a.G = G; a.V = V; a.nch = (V + CHUNK - 1) / CHUNK; a.k_max = k_max; a.top_k = top_k; a.top_p = top_p;
     a.temperature = temperature; a.q_idx = q_idx; a.q_prob = q_prob; a.q_count = q_count;
     a.u_draft = u_draft; a.draft_tok = draft_tok;
-    a.row_max = ctx->row_max; a.dsum = ctx->dsum; a.queue = ctx->queue;
-    const int cur = 1 + (int)(ctx->compress_calls & 1ull);
-    a.queue_count = ctx->counters + cur;
-    a.queue_count_next = ctx->counters + (3 - cur);
-    a.redo_rows = ctx->redo_rows;
-    a.redo_count = ctx->counters + 2 + cur;           // [3] / [4]
-    a.redo_count_next = ctx->counters + 2 + (3 - cur);
-    a.use_redo_list = 0;
-    a.redo_total = ctx->slow_rows + 1;
-    a.surv_keys = ctx->surv_keys;
-    a.surv_meta = ctx->surv_meta;
-    ctx->compress_calls++;
-    a.status = ctx->status; a.slow_rows = ctx->slow_rows;
+    a.row_pos = nullptr; a.seq_rows = 0; a.raw_probs = 0;
+    fill_compress_workspace(ctx, a);
     cudaStream_t s = (cudaStream_t)cuda_stream;
     cudaError_t e;
     if (dtype == PICOSPEC_BF16)
@@ -441,7 +450,7 @@ int picospec_compress(picospec_ctx* ctx, const void* draft_logits, picospec_dtyp
     return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
 }
 
-static int verify_common(picospec_ctx* ctx, VerifyArgs& a, picospec_dtype dtype, void* cuda_stream) {
+static int verify_common(picospec_ctx* ctx, VerifyArgs& a, picospec_dtype dtype, void* cuda_stream, bool edge = false) {
     DeviceGuard g(ctx->device);
     if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
     a.nch = (a.V + CHUNK - 1) / CHUNK;
@@ -451,9 +460,9 @@ static int verify_common(picospec_ctx* ctx, VerifyArgs& a, picospec_dtype dtype,
     cudaStream_t s = (cudaStream_t)cuda_stream;
     cudaError_t e;
     if (dtype == PICOSPEC_BF16)
-        e = launch_verify<__nv_bfloat16>(ctx, a, rows_aligned(a.logits, a.row_stride, 2), s);
+        e = launch_verify<__nv_bfloat16>(ctx, a, rows_aligned(a.logits, a.row_stride, 2), s, edge);
     else
-        e = launch_verify<float>(ctx, a, rows_aligned(a.logits, a.row_stride, 4), s);
+        e = launch_verify<float>(ctx, a, rows_aligned(a.logits, a.row_stride, 4), s, edge);
     return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
 }
 
@@ -496,6 +505,49 @@ int picospec_residual_sample(picospec_ctx* ctx, const void* target_logits, picos
     a.accept_len = nullptr; a.p_draft = nullptr; a.resid_mass = nullptr; a.borderline = nullptr;
     a.token = token; a.mass = mass;
     return verify_common(ctx, a, dtype, cuda_stream);
+}
+
+int picospec_target_topk(picospec_ctx* ctx, const void* target_logits, picospec_dtype dtype, int B, int R, int V,
+                         long long row_stride_elems, const float* temperature, const int* pos, int k, int* p_idx,
+                         float* p_prob, int* p_count, void* cuda_stream) {
+    int rc = check_common(ctx, target_logits, (int)dtype, B, R > 0 ? R - 1 : -1, V, row_stride_elems, temperature, k);
+    if (rc != PICOSPEC_OK) return rc;
+    if (!pos || !p_idx || !p_prob || !p_count) return PICOSPEC_EINVAL;
+    if (B == 0) return PICOSPEC_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
+    CompressArgs a;
+    a.logits = target_logits; a.row_stride = row_stride_elems;
+    a.B = B; a.G = 1; a.V = V; a.nch = (V + CHUNK - 1) / CHUNK; a.k_max = k; a.top_k = k; a.top_p = 1.0f;
+    a.temperature = temperature; a.q_idx = p_idx; a.q_prob = p_prob; a.q_count = p_count;
+    a.u_draft = nullptr; a.draft_tok = nullptr;
+    a.row_pos = pos; a.seq_rows = R; a.raw_probs = 1;
+    fill_compress_workspace(ctx, a);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e;
+    if (dtype == PICOSPEC_BF16)
+        e = launch_compress<__nv_bfloat16>(ctx, a, rows_aligned(target_logits, row_stride_elems, 2), s);
+    else
+        e = launch_compress<float>(ctx, a, rows_aligned(target_logits, row_stride_elems, 4), s);
+    return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
+}
+
+int picospec_edge_resample(picospec_ctx* ctx, const void* draft_logits, picospec_dtype dtype, int B, int R, int V,
+                           long long row_stride_elems, const float* temperature, const int* pos, const int* p_idx,
+                           const float* p_prob, const int* p_count, int k, const float* u, int* token, float* mass,
+                           void* cuda_stream) {
+    int rc = check_common(ctx, draft_logits, (int)dtype, B, R > 0 ? R - 1 : -1, V, row_stride_elems, temperature, k);
+    if (rc != PICOSPEC_OK) return rc;
+    if (!pos || !p_idx || !p_prob || !p_count || !u || !token) return PICOSPEC_EINVAL;
+    if (B == 0) return PICOSPEC_OK;
+    VerifyArgs a;
+    a.logits = draft_logits; a.row_stride = row_stride_elems;
+    a.B = B; a.G = R - 1; a.V = V; a.k_max = k; a.sample_only = 1;
+    a.temperature = temperature; a.draft_tok = nullptr; a.q_idx = p_idx; a.q_prob = p_prob; a.q_count = p_count;
+    a.u_accept = nullptr; a.pos = pos; a.u_resample = u;
+    a.accept_len = nullptr; a.p_draft = nullptr; a.resid_mass = nullptr; a.borderline = nullptr;
+    a.token = token; a.mass = mass;
+    return verify_common(ctx, a, dtype, cuda_stream, true);
 }
 
 }  // extern "C"

@@ -326,6 +326,43 @@ def bench_workload(ps, w, args, rank, world, device, with_e2e, with_clocks):
     return res
 
 
+def bench_paper_direction(ps, w, device, k, iters):
+    """The paper's own data flow (Sec. 3.3) on the same shape, timed per call with CUDA events:
+    picospec_target_topk (Top-K of the target row at one position per sequence, K = 10 as in the
+    paper's payload example) and picospec_edge_resample (against the dense draft row)."""
+    ctx = ps.Context(w.B, w.G, w.V, max(k, 1))
+    nsets = 3
+    sets = [gen.make_inputs(w, seed=7000 + i, device=device) for i in range(nsets)]
+    gpos = torch.Generator(device="cpu").manual_seed(7)
+    pos = torch.randint(0, w.G, (w.B,), generator=gpos, dtype=torch.int32).to(device)
+    out = {}
+
+    def timed(fn):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / iters
+
+    payload = [ctx.target_topk(s["target_logits"], s["temperature"], pos, k) for s in sets]
+    out["target_topk_us"] = timed(lambda i: ctx.target_topk(sets[i % nsets]["target_logits"], sets[i % nsets]["temperature"], pos, k))
+    u = [s["u_resample"][:, 0].contiguous() for s in sets]
+    out["edge_resample_us"] = timed(lambda i: ctx.edge_resample(sets[i % nsets]["draft_logits"], sets[i % nsets]["temperature"],
+                                                                pos, *payload[i % nsets], u[i % nsets], want_mass=False))
+    row_bytes = w.B * w.V * w.bytes_per_logit
+    out.update({"k": k, "rows_per_call": w.B, "row_bytes_per_call": row_bytes,
+                "target_topk_GBps": row_bytes / out["target_topk_us"] / 1e3,
+                "edge_resample_GBps": row_bytes / out["edge_resample_us"] / 1e3,
+                "status": ctx.status(clear=True)[0]})
+    ctx.close()
+    return out
+
+
 def run_ours(args):
     rank, local_rank, world = _dist_env()
     if not torch.cuda.is_available():
@@ -354,6 +391,10 @@ def run_ours(args):
                             "compress_stream_us": r["compress_stream"]["avg_us"],
                             "compress_stream_GBps": r["compress_stream"]["GBps"],
                             "input_sets_rotated": r["nsets"], "slow_rows_per_step": r["slow_rows_per_step"]}
+
+    paper_direction = None
+    if args.all_configs and world == 1:
+        paper_direction = bench_paper_direction(ps, w, device, k=10, iters=min(args.steps, 200))
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -405,6 +446,7 @@ def run_ours(args):
             "compress_redo_rows_per_step": main["redo_rows_per_step"],
             "device_status": main["status"],
             "other_configs": others,
+            "paper_direction": paper_direction,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

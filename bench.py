@@ -40,8 +40,8 @@ UNIT = "positions/s"
 # summarised under profiles/, keyed by (workload, kernel); absent until a capture of the current
 # kernel exists.  Captured at B = 64 and scaled to the full batch by the rows processed.
 NCU_TRAFFIC_BYTES = {
-    ("config4", "compress_filter_kernel"): 4 * (98564608 + 4149504),
-    ("config4", "chunk_stats_bulk_kernel"): 4 * (114932224 + 3787520),
+    ("config4", "compress_filter_kernel"): 4 * (98561536 + 3489280),
+    ("config4", "chunk_stats_bulk_kernel"): 4 * (114932224 + 3586304),
 }
 
 

@@ -121,11 +121,15 @@ def test_config5_sweep_points_reduced_batch(ps, V, k):
     assert r["status"] == 0
 
 
-def test_config5_full_batch_sampled(ps):
-    w = gen.sweep_workload(128256, 64, B=512)
-    inputs = gen.make_inputs(w, seed=5512, device="cuda")
-    r = run_both(ps, w, inputs, seq_subset=np.arange(3, 512, 32))
+@pytest.mark.parametrize("V,k", [(128256, 64), (32000, 8), (262144, 1024), (151936, 512)])
+def test_config5_full_batch_sampled(ps, V, k):
+    # the sweep's full batch (B = 512, gamma = 8) in one launch; the oracle checks a sample of sequences
+    w = gen.sweep_workload(V, k, B=512)
+    inputs = gen.make_inputs(w, seed=5512 + k, device="cuda")
+    r = run_both(ps, w, inputs, seq_subset=np.arange(3, 512, 64))
     assert r["status"] == 0
+    del inputs
+    torch.cuda.empty_cache()
 
 
 # ---------------------------------------------------------------------------------------------

@@ -41,7 +41,7 @@ def _load():
         # a test that plants a mistake points this at its own build of a modified copy
         _lib = ctypes.CDLL(os.environ.get("PICOSPEC_ORACLE_LIB") or build())
         for name in ("pso_compress", "pso_verify", "pso_residual_sample", "pso_softmax", "pso_target_topk",
-                     "pso_edge_resample"):
+                     "pso_edge_resample", "pso_verify_range"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -125,6 +125,43 @@ def verify(target_logits, temperature, draft_tok, q_idx, q_prob, q_count, u_acce
         raise ValueError(f"pso_verify failed: {rc}")
     return {"accept_len": accept_len, "p_draft": p_draft, "resid_mass": resid,
             "borderline_seq": border, "borderline_count": int(border.sum()), "token": token}
+
+
+def verify_range(target_logits, temperature, gamma, r0: int, r1: int, state_in, draft_tok, q_idx, q_prob,
+                 q_count, u_accept, u_resample, out=None, chunk: int = CHUNK, nthreads: int = 1):
+    """Incremental verification of the target rows [r0, r1).  `out` carries accept_len, token,
+    p_draft, resid_mass from earlier calls (decided sequences and untested positions keep their
+    values); returns the updated dict with state [B] i32 and borderline_count of this call."""
+    l = _f32(target_logits)
+    B, G1, V = _rows(l)
+    G = G1 - 1
+    T = _f32(temperature)
+    gm = None if gamma is None else _i32(gamma)
+    st = None if state_in is None else _i32(state_in)
+    tok_in = _i32(draft_tok).reshape(B, G)
+    qi = _i32(q_idx)
+    qp = _f32(q_prob)
+    qc = _i32(q_count).reshape(B, G)
+    k_max = qi.shape[-1] if qi.ndim == 3 and G > 0 else 1
+    ua = _f32(u_accept).reshape(B, G)
+    ur = _f32(u_resample)
+    assert ur.shape == (B, 2)
+    if out is None:
+        out = {"accept_len": np.full((B,), -2, np.int32), "token": np.full((B,), -2, np.int32),
+               "p_draft": np.full((B, G), np.nan, np.float64), "resid_mass": np.full((B, G), np.nan, np.float64)}
+    out = {k: np.ascontiguousarray(v).copy() for k, v in out.items() if k in ("accept_len", "token", "p_draft", "resid_mass")}
+    border = np.zeros((B,), np.int64)
+    state = np.empty((B,), np.int32)
+    rc = _load().pso_verify_range(_p(l), ctypes.c_long(B), ctypes.c_long(G), ctypes.c_long(V), ctypes.c_long(V),
+                                  _p(T), _p(gm), ctypes.c_long(r0), ctypes.c_long(r1), _p(st), _p(tok_in), _p(qi),
+                                  _p(qp), _p(qc), ctypes.c_int(k_max), _p(ua), _p(out["accept_len"]),
+                                  _p(out["p_draft"]), _p(out["resid_mass"]), _p(border), _p(ur), _p(out["token"]),
+                                  _p(state), ctypes.c_long(chunk), ctypes.c_int(nthreads))
+    if rc != 0:
+        raise ValueError(f"pso_verify_range failed: {rc}")
+    out["state"] = state
+    out["borderline_count"] = int(border.sum())
+    return out
 
 
 def residual_sample(target_logits, temperature, pos, q_idx, q_prob, q_count, u_resample,

@@ -469,6 +469,151 @@ int pso_residual_sample(const float *target_logits, long B, long G, long V, long
     return err ? PSO_ENOMEM : PSO_OK;
 }
 
+/* ---- prefix / incremental verification (Sec. 3.2 "Fast Verification": the verifier starts on a
+ * ---- known prefix before the edge has finished its segment; Sec. 3.3: segments can be cut short) */
+
+/* Verify the target rows [r0, r1) of every sequence that is still undecided, carrying the state
+ * from the calls on earlier rows.  gamma[b] (or G when gamma is NULL) is the number of drafted
+ * tokens of sequence b (latency-aware truncation makes it vary); its target rows are 0 .. gamma[b],
+ * the last one being the bonus row.
+ *   state_in[b] (NULL = all 1): 1 = every position before r0 was accepted, 0 = already decided
+ *   (such a sequence is skipped and none of its outputs is written).
+ * For an undecided sequence the positions i in [r0, min(r1, gamma)) are tested in order exactly as
+ * in pso_verify.  A rejection at i decides it: accept_len = i, token from the residual of row i.
+ * If all are accepted and the bonus row lies in the range (r0 <= gamma < r1): accept_len = gamma,
+ * token from p at row gamma.  Otherwise it stays undecided: accept_len = -2, token = -2,
+ * state_out = 1.  p_draft / resid_mass are written for the tested positions only.
+ * Unusable input inside the range (or gamma outside [0, G], or gamma < r0 for an undecided
+ * sequence): accept_len = -1, token = -1, state_out = 0, tested positions' p_draft / resid_mass -1.
+ * Rows outside the range are never read. */
+int pso_verify_range(const float *target_logits, long B, long G, long V, long row_stride,
+                     const float *temperature, const int *gamma, long r0, long r1,
+                     const int *state_in, const int *draft_tok, const int *q_idx,
+                     const float *q_prob, const int *q_count, int k_max, const float *u_accept,
+                     int *accept_len, double *p_draft, double *resid_mass, long long *borderline_seq,
+                     const float *u_resample, int *token, int *state_out, long chunk, int nthreads) {
+    if (!target_logits || !temperature || !accept_len || !p_draft || !resid_mass || !borderline_seq ||
+        !u_resample || !token || !state_out)
+        return PSO_EINVAL;
+    if (G > 0 && (!draft_tok || !q_idx || !q_prob || !q_count || !u_accept)) return PSO_EINVAL;
+    if (B < 0 || G < 0 || V <= 0 || k_max <= 0 || row_stride < V || chunk <= 0) return PSO_EINVAL;
+    if (r0 < 0 || r1 <= r0 || r1 > G + 1) return PSO_EINVAL;
+    if (nthreads < 1) nthreads = 1;
+    int err = 0;
+#pragma omp parallel num_threads(nthreads)
+    {
+        double *w = (double *)malloc((size_t)V * sizeof(double));
+        double *qd = (double *)calloc((size_t)V, sizeof(double));
+        double *r = (double *)malloc((size_t)V * sizeof(double));
+        if (!w || !qd || !r) {
+#pragma omp atomic write
+            err = 1;
+        }
+#pragma omp barrier
+        if (!err) {
+#pragma omp for schedule(dynamic, 1)
+            for (long b = 0; b < B; ++b) {
+                borderline_seq[b] = 0;
+                if (state_in && state_in[b] == 0) {
+                    state_out[b] = 0;
+                    continue;
+                }
+                double T = (double)temperature[b];
+                long g = gamma ? gamma[b] : G;
+                const float *rows = target_logits + b * (G + 1) * row_stride;
+                int ok = pso_temperature_ok(T) && g >= 0 && g <= G && g >= r0;
+                long hi = g < r1 ? g : r1; /* positions tested: [r0, hi) */
+                for (long i = r0; i < hi && ok; ++i) {
+                    long ri = b * G + i;
+                    if (draft_tok[ri] < 0 || draft_tok[ri] >= V) ok = 0;
+                    if (ok && !pso_sparse_row_ok(q_idx + ri * k_max, q_count[ri], k_max, V)) ok = 0;
+                }
+                long a = r0;
+                int still = 1;
+                long long nborder = 0;
+                for (long i = r0; i < hi && ok; ++i) {
+                    long ri = b * G + i;
+                    double Z;
+                    if (pso_softmax_row(rows + i * row_stride, V, T, w, &Z)) {
+                        ok = 0;
+                        break;
+                    }
+                    const int *idx = q_idx + ri * k_max;
+                    const float *prob = q_prob + ri * k_max;
+                    int n = q_count[ri];
+                    int x = draft_tok[ri];
+                    double qx = 0.0;
+                    for (int j = 0; j < n; ++j)
+                        if (idx[j] == x) {
+                            qx = (double)prob[j];
+                            break;
+                        }
+                    double px = w[x] / Z;
+                    double u = (double)u_accept[ri];
+                    int acc, border = 0;
+                    if (qx > 0.0) {
+                        double ratio = px / qx;
+                        double lim = ratio < 1.0 ? ratio : 1.0;
+                        acc = u < lim;
+                        border = fabs(ratio - u) <= 1e-6 * u;
+                    } else {
+                        acc = 1;
+                    }
+                    p_draft[ri] = px;
+                    resid_mass[ri] = pso_residual_weights(w, Z, V, idx, prob, n, qd, r);
+                    if (still) {
+                        nborder += border;
+                        if (acc)
+                            a += 1;
+                        else
+                            still = 0;
+                    }
+                }
+                int rejected = ok && a < hi;
+                int bonus = ok && !rejected && g < r1; /* all accepted and row g is in the range */
+                if (bonus) {
+                    double Z;
+                    if (pso_softmax_row(rows + g * row_stride, V, T, w, &Z)) ok = 0;
+                }
+                if (ok && (rejected || bonus)) {
+                    long ri = b * G + a;
+                    long t = pso_sample_row(rows + a * row_stride, V, T, rejected,
+                                            rejected ? q_idx + ri * k_max : NULL,
+                                            rejected ? q_prob + ri * k_max : NULL,
+                                            rejected ? q_count[ri] : 0, chunk,
+                                            (double)u_resample[2 * b], (double)u_resample[2 * b + 1],
+                                            w, qd, r, NULL);
+                    if (t == -2) {
+#pragma omp atomic write
+                        err = 1;
+                    }
+                    token[b] = (int)t;
+                    accept_len[b] = (int)a;
+                    state_out[b] = 0;
+                    borderline_seq[b] = nborder;
+                } else if (ok) {
+                    token[b] = -2;
+                    accept_len[b] = -2;
+                    state_out[b] = 1;
+                    borderline_seq[b] = nborder;
+                } else {
+                    token[b] = -1;
+                    accept_len[b] = -1;
+                    state_out[b] = 0;
+                    for (long i = r0; i < hi && i < G; ++i) {
+                        p_draft[b * G + i] = -1.0;
+                        resid_mass[b * G + i] = -1.0;
+                    }
+                }
+            }
+        }
+        free(w);
+        free(qd);
+        free(r);
+    }
+    return err ? PSO_ENOMEM : PSO_OK;
+}
+
 /* ---- the paper's own direction (Sec. 3.3): Top-K of the target row on the verifier, ---------
  * ---- resampling against the drafter's dense row on the edge ------------------------------- */
 

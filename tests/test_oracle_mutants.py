@@ -45,6 +45,11 @@ MUTANTS = [
     ("edge_wrong_row", "const float *l = draft_logits + (b * rows_per_seq + j) * row_stride;",
      "const float *l = draft_logits + (b * rows_per_seq + 0) * row_stride;"),
     ("edge_nonstrict", "if (cum > thr) {\n                        pick = t;", "if (cum >= thr * 1.2) {\n                        pick = t;"),
+    ("range_restarts_at_zero", "long a = r0;", "long a = 0;"),
+    ("range_bonus_before_its_row", "int bonus = ok && !rejected && g < r1;", "int bonus = ok && !rejected;"),
+    ("range_ignores_gamma", "long g = gamma ? gamma[b] : G;", "long g = G;"),
+    ("range_ignores_state", "if (state_in && state_in[b] == 0) {", "if (0) {"),
+    ("range_reads_later_rows", "long hi = g < r1 ? g : r1;", "long hi = g;"),
     ("edge_no_fallback", "if (!(R > 0.0)) {\n                    R = 0.0;", "if (0) {\n                    R = 0.0;"),
 ]
 

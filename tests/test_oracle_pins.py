@@ -596,3 +596,88 @@ def test_edge_resample_flags_unusable_input():
     tok, mass = oracle.edge_resample(ld, T, pos2, pi, pp, pc, np.full(B, 0.5, np.float32))
     assert tok[0] >= 0 and mass[0] > 0
     assert list(tok[1:]) == [-1, -1, -1, -1] and np.all(mass[1:] == -1)
+
+
+# ---------------------------------------------------------------------------------------------
+# Prefix / incremental verification (Sec. 3.2 Fast Verification; Sec. 3.3 truncated segments)
+# ---------------------------------------------------------------------------------------------
+
+def _range_case(seed, B=12, G=6, V=40, K=6):
+    rng = _rng(seed)
+    ld = rng.normal(size=(B, G, V)).astype(np.float32) * 2
+    lt = (0.8 * np.concatenate([ld, ld[:, :1]], axis=1) + rng.normal(size=(B, G + 1, V))).astype(np.float32)
+    T = rng.uniform(0.6, 1.2, size=B).astype(np.float32)
+    qi, qp, qc, tok = oracle.compress(ld, T, top_k=K, top_p=1.0, k_max=K, u_draft=rng.random((B, G)).astype(np.float32))
+    ua = rng.random((B, G)).astype(np.float32)
+    ur = rng.random((B, 2)).astype(np.float32)
+    return lt, T, tok, qi, qp, qc, ua, ur
+
+
+@pytest.mark.parametrize("cuts", [[0, 7], [0, 1, 2, 3, 4, 5, 6, 7], [0, 3, 7], [0, 2, 5, 6, 7], [0, 6, 7]])
+def test_verifying_in_row_ranges_equals_verifying_at_once(cuts):
+    # rows arrive in pieces; carrying the state through the calls must give what pso_verify gives
+    lt, T, tok, qi, qp, qc, ua, ur = _range_case(201)
+    B, G = tok.shape
+    full = oracle.verify(lt, T, tok, qi, qp, qc, ua, ur)
+    out, state, border = None, None, 0
+    decided_at = np.full(B, -1)
+    for r0, r1 in zip(cuts[:-1], cuts[1:]):
+        # rows at and beyond r1 have not arrived: poison them to show they are not read
+        seen = lt.copy()
+        seen[:, r1:] = np.nan
+        out = oracle.verify_range(seen, T, None, r0, r1, state, tok, qi, qp, qc, ua, ur, out=out)
+        state = out["state"]
+        border += out["borderline_count"]
+        undecided = state == 1
+        assert np.all(out["accept_len"][undecided] == -2) and np.all(out["token"][undecided] == -2)
+        decided_at[(decided_at < 0) & ~undecided] = r1
+    assert np.all(state == 0)
+    assert np.array_equal(out["accept_len"], full["accept_len"])
+    assert np.array_equal(out["token"], full["token"])
+    assert border == full["borderline_count"]
+    for b in range(B):
+        a = int(full["accept_len"][b])
+        assert decided_at[b] == min(r for r in cuts[1:] if r > a)   # decided by the first call that sees row a
+        n = min(int(decided_at[b]), G)                       # positions of the calls up to the decision
+        np.testing.assert_array_equal(out["p_draft"][b, :n], full["p_draft"][b, :n])
+        np.testing.assert_array_equal(out["resid_mass"][b, :n], full["resid_mass"][b, :n])
+        assert np.all(np.isnan(out["p_draft"][b, n:]))       # positions of later calls were never tested
+
+
+def test_truncated_segments_equal_verifying_the_shorter_sequence():
+    # gamma[b] < G: the sequence's rows are 0 .. gamma[b], row gamma[b] is its bonus row
+    lt, T, tok, qi, qp, qc, ua, ur = _range_case(203)
+    B, G = tok.shape
+    rng = _rng(5)
+    gamma = rng.integers(0, G + 1, size=B).astype(np.int32)
+    gamma[0], gamma[1] = 0, G
+    out = oracle.verify_range(lt, T, gamma, 0, G + 1, None, tok, qi, qp, qc, ua, ur)
+    assert np.all(out["state"] == 0)
+    for b in range(B):
+        g = int(gamma[b])
+        ref = oracle.verify(lt[b:b + 1, :g + 1], T[b:b + 1], tok[b:b + 1, :g], qi[b:b + 1, :g], qp[b:b + 1, :g],
+                            qc[b:b + 1, :g], ua[b:b + 1, :g], ur[b:b + 1])
+        assert out["accept_len"][b] == ref["accept_len"][0] and out["token"][b] == ref["token"][0]
+
+
+def test_range_call_skips_decided_sequences_and_flags_bad_input():
+    lt, T, tok, qi, qp, qc, ua, ur = _range_case(207)
+    B, G = tok.shape
+    state = np.ones(B, np.int32)
+    state[3] = 0
+    prev = {"accept_len": np.full(B, 77, np.int32), "token": np.full(B, 88, np.int32),
+            "p_draft": np.full((B, G), 0.5), "resid_mass": np.full((B, G), 0.25)}
+    lt2 = lt.copy()
+    lt2[4, 1, 7] = np.inf               # inside the range
+    lt2[5, 5, 7] = np.nan               # outside the range: not read
+    gamma = np.full(B, G, np.int32)
+    gamma[6] = G + 1                    # out of range
+    out = oracle.verify_range(lt2, T, gamma, 0, 3, state, tok, qi, qp, qc, ua, ur, out=prev)
+    assert out["accept_len"][3] == 77 and out["token"][3] == 88 and out["state"][3] == 0
+    assert np.all(out["p_draft"][3] == 0.5)
+    for b in (4, 6):
+        assert out["accept_len"][b] == -1 and out["token"][b] == -1 and out["state"][b] == 0
+    assert out["accept_len"][5] in (-2, 0, 1, 2)
+    # an undecided sequence whose bonus row lies before the range is a caller error
+    out = oracle.verify_range(lt, T, np.full(B, 1, np.int32), 3, 5, None, tok, qi, qp, qc, ua, ur)
+    assert np.all(out["accept_len"] == -1)

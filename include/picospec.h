@@ -160,6 +160,40 @@ PICOSPEC_API int picospec_verify(picospec_ctx* ctx, const void* target_logits, p
                     float* p_draft, float* resid_mass, int* borderline_count, const float* u_resample,
                     int* token, void* cuda_stream);
 
+/* Half 2a on rows as they arrive -- incremental verification (Sec. 3.2: the verifier works on a
+ * prefix of the segment while the drafter is still producing the rest; Sec. 3.3: latency-aware
+ * truncation makes the number of drafted tokens differ between sequences).
+ *
+ * One call handles the target rows [r0, r1) of every sequence that is still undecided and never
+ * reads a row outside that range; a chain of calls over consecutive ranges that together cover
+ * [0, G + 1), each passing the previous call's state_out as state_in, gives every sequence the
+ * accept_len and token picospec_verify gives it.
+ *   gamma[b] (NULL: G) = drafted tokens of sequence b, in [0, G]; its rows are 0 .. gamma[b], the
+ *                        last one the bonus row; rows beyond it are never read.
+ *   state_in[b] (NULL: all 1): 1 = every position before r0 was accepted; 0 = decided by an
+ *                        earlier call: the sequence is skipped, of its outputs only
+ *                        state_out[b] = 0 is written.
+ * For an undecided sequence the positions i in [r0, min(r1, gamma)) get the accept test of
+ * picospec_verify, with p_draft[b,i] and resid_mass[b,i] written for exactly those positions.
+ *   first rejection at i:                       accept_len = i, token from the residual of row i
+ *   all accepted and r0 <= gamma < r1:          accept_len = gamma, token from p at row gamma
+ *   otherwise (undecided):                      accept_len = -2, token = -2, state_out = 1
+ * Decided sequences get state_out = 0.  *borderline_count counts this call's deciding tests.
+ * Bad data inside the range, gamma[b] outside [0, G], or gamma[b] < r0 for an undecided
+ * sequence: accept_len = -1, token = -1, state_out = 0, the range's p_draft = resid_mass = -1,
+ * and the matching status bit.
+ *
+ * 0 <= r0 < r1 <= G + 1, else PICOSPEC_EINVAL.  gamma, state_in [B] int32 or NULL; state_out [B]
+ * int32; every other array as in picospec_verify.  state_in and state_out may be the same
+ * array.
+ */
+PICOSPEC_API int picospec_verify_range(picospec_ctx* ctx, const void* target_logits, picospec_dtype dtype, int B, int G,
+                          int V, long long row_stride_elems, const float* temperature, const int* gamma, int r0,
+                          int r1, const int* state_in, const int* draft_tok, const int* q_idx, const float* q_prob,
+                          const int* q_count, int k_max, const float* u_accept, int* accept_len, float* p_draft,
+                          float* resid_mass, int* borderline_count, const float* u_resample, int* token,
+                          int* state_out, void* cuda_stream);
+
 /* Half 2b -- local resampling (Sec. 3.3: the corrected token is drawn from
  * norm(max(0, P_j(x) - Q_j(x)))).
  *

@@ -49,6 +49,9 @@ def lib() -> ctypes.CDLL:
         L.picospec_edge_resample.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp, c_int,
                                              vp, vp, vp, vp]
         L.picospec_edge_resample.restype = c_int
+        L.picospec_verify_range.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, c_int, c_int, vp, vp,
+                                            vp, vp, vp, c_int, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.picospec_verify_range.restype = c_int
         L.picospec_counters.argtypes = [vp, ctypes.POINTER(c_ll), c_int, vp]
         L.picospec_counters.restype = c_int
         L.picospec_verify_static.argtypes = [vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp, c_int,
@@ -233,6 +236,38 @@ class Context:
             _ptr(out["p_draft"], torch.float32, (B, G)), _ptr(out["resid_mass"], torch.float32, (B, G)),
             _ptr(out["borderline_count"], torch.int32, (1,)), _ptr(u_resample, torch.float32, (B, 2)),
             _ptr(out["token"], torch.int32, (B,)), _stream()), "picospec_verify")
+        return out
+
+    def verify_range(self, target_logits: torch.Tensor, temperature: torch.Tensor, gamma: Optional[torch.Tensor],
+                     r0: int, r1: int, state_in: Optional[torch.Tensor], draft_tok: torch.Tensor,
+                     q_idx: torch.Tensor, q_prob: torch.Tensor, q_count: torch.Tensor, u_accept: torch.Tensor,
+                     u_resample: Optional[torch.Tensor] = None, out=None):
+        """picospec_verify_range on the target rows [r0, r1).  `out` is the dict of an earlier call
+        (its arrays are updated in place; state may alias state_in) or None.  Returns dict(accept_len,
+        p_draft, resid_mass, borderline_count, token or None, state [B] i32)."""
+        p, dt, B, G1, V, pitch = _logits(target_logits)
+        G = G1 - 1
+        k_max = q_idx.shape[-1]
+        dev = target_logits.device
+        if out is None:
+            out = {
+                "accept_len": torch.full((B,), -2, dtype=torch.int32, device=dev),
+                "p_draft": torch.full((B, G), float("nan"), dtype=torch.float32, device=dev),
+                "resid_mass": torch.full((B, G), float("nan"), dtype=torch.float32, device=dev),
+                "borderline_count": torch.empty((1,), dtype=torch.int32, device=dev),
+                "token": torch.full((B,), -2, dtype=torch.int32, device=dev) if u_resample is not None else None,
+                "state": torch.empty((B,), dtype=torch.int32, device=dev),
+            }
+        _check(lib().picospec_verify_range(
+            self._h, p, dt, B, G, V, pitch, _ptr(temperature, torch.float32, (B,)), _ptr(gamma, torch.int32, (B,)),
+            int(r0), int(r1), _ptr(state_in, torch.int32, (B,)),
+            _ptr(draft_tok, torch.int32, (B, G)), _ptr(q_idx, torch.int32, (B, G, k_max)),
+            _ptr(q_prob, torch.float32, (B, G, k_max)), _ptr(q_count, torch.int32, (B, G)), int(k_max),
+            _ptr(u_accept, torch.float32, (B, G)), _ptr(out["accept_len"], torch.int32, (B,)),
+            _ptr(out["p_draft"], torch.float32, (B, G)), _ptr(out["resid_mass"], torch.float32, (B, G)),
+            _ptr(out["borderline_count"], torch.int32, (1,)), _ptr(u_resample, torch.float32, (B, 2)),
+            _ptr(out["token"], torch.int32, (B,)), _ptr(out["state"], torch.int32, (B,)), _stream()),
+            "picospec_verify_range")
         return out
 
     # -- the paper's own data flow (Sec. 3.3) ---------------------------------------------------

@@ -196,7 +196,8 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
 
 template <typename T>
 cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, cudaStream_t s, bool edge = false) {
-    const long long items = (long long)(a.sample_only ? a.B : a.B * (a.G + 1)) * a.nch;
+    const int stream_rows = a.sample_only ? a.B : a.B * (a.r1 - a.r0);
+    const long long items = (long long)stream_rows * a.nch;
     long long want = (items + WARPS - 1) / WARPS;
     const int cap = ctx->num_sms * 4;
     const int grid = (int)(want < cap ? want : cap);
@@ -205,7 +206,7 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
         cudaError_t ea = ensure_kernel_attrs(ctx->device);
         if (ea != cudaSuccess) return ea;
         const int tiles_per_row = (a.nch + TileGeom<T>::CHUNKS - 1) / TileGeom<T>::CHUNKS;
-        const long long tiles = (long long)(a.sample_only ? a.B : a.B * (a.G + 1)) * tiles_per_row;
+        const long long tiles = (long long)stream_rows * tiles_per_row;
         const int gcap = ctx->num_sms * StreamCfg<T>::CTAS_PER_SM;
         const int g = (int)(tiles < gcap ? tiles : gcap);
         ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_STREAM, 1, s);
@@ -229,6 +230,9 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
     p.seq_rows = a.G + 1; p.expand = a.sample_only ? 1 : a.G + 1; p.pos = a.sample_only ? a.pos : nullptr;
     p.temperature = a.temperature; p.queue = a.queue; p.queue_count = a.queue_count;
     p.need_rows = a.need_rows;
+    if (!a.sample_only) {
+        p.r0 = a.r0; p.r1 = a.r1; p.gamma = a.gamma;
+    }
     p.row_max = a.row_max; p.dsum = a.dsum;
     precise_chunk_sums_kernel<T><<<ctx->num_sms * 6, THREADS, 0, s>>>(p);
     const int g2 = a.B < ctx->num_sms ? a.B : ctx->num_sms;
@@ -454,6 +458,7 @@ static int verify_common(picospec_ctx* ctx, VerifyArgs& a, picospec_dtype dtype,
     DeviceGuard g(ctx->device);
     if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
     a.nch = (a.V + CHUNK - 1) / CHUNK;
+    if (a.r1 < 0) a.r1 = a.G + 1;
     a.stats = ctx->stats; a.row_max = ctx->row_max; a.dsum = ctx->dsum; a.queue = ctx->queue;
     a.need_rows = ctx->need_rows;
     a.queue_count = ctx->counters; a.status = ctx->status; a.slow_rows = ctx->slow_rows;
@@ -481,6 +486,31 @@ int picospec_verify(picospec_ctx* ctx, const void* target_logits, picospec_dtype
     VerifyArgs a;
     a.logits = target_logits; a.row_stride = row_stride_elems;
     a.B = B; a.G = G; a.V = V; a.k_max = k_max; a.sample_only = 0;
+    a.temperature = temperature; a.draft_tok = draft_tok; a.q_idx = q_idx; a.q_prob = q_prob; a.q_count = q_count;
+    a.u_accept = u_accept; a.pos = nullptr; a.u_resample = u_resample;
+    a.accept_len = accept_len; a.p_draft = p_draft; a.resid_mass = resid_mass; a.borderline = borderline_count;
+    a.token = token; a.mass = nullptr;
+    return verify_common(ctx, a, dtype, cuda_stream);
+}
+
+int picospec_verify_range(picospec_ctx* ctx, const void* target_logits, picospec_dtype dtype, int B, int G, int V,
+                          long long row_stride_elems, const float* temperature, const int* gamma, int r0, int r1,
+                          const int* state_in, const int* draft_tok, const int* q_idx, const float* q_prob,
+                          const int* q_count, int k_max, const float* u_accept, int* accept_len, float* p_draft,
+                          float* resid_mass, int* borderline_count, const float* u_resample, int* token,
+                          int* state_out, void* cuda_stream) {
+    int rc = check_common(ctx, target_logits, (int)dtype, B, G, V, row_stride_elems, temperature, k_max);
+    if (rc != PICOSPEC_OK) return rc;
+    if (!accept_len || !borderline_count || !state_out) return PICOSPEC_EINVAL;
+    if (r0 < 0 || r1 <= r0 || r1 > G + 1) return PICOSPEC_EINVAL;
+    if (G > 0 && (!draft_tok || !q_idx || !q_prob || !q_count || !u_accept || !p_draft || !resid_mass))
+        return PICOSPEC_EINVAL;
+    if ((u_resample == nullptr) != (token == nullptr)) return PICOSPEC_EINVAL;
+    if (B == 0) return PICOSPEC_OK;
+    VerifyArgs a;
+    a.logits = target_logits; a.row_stride = row_stride_elems;
+    a.B = B; a.G = G; a.V = V; a.k_max = k_max; a.sample_only = 0;
+    a.r0 = r0; a.r1 = r1; a.gamma = gamma; a.state_in = state_in; a.state_out = state_out;
     a.temperature = temperature; a.draft_tok = draft_tok; a.q_idx = q_idx; a.q_prob = q_prob; a.q_count = q_count;
     a.u_accept = u_accept; a.pos = nullptr; a.u_resample = u_resample;
     a.accept_len = accept_len; a.p_draft = p_draft; a.resid_mass = resid_mass; a.borderline = borderline_count;
@@ -636,6 +666,7 @@ extern "C" int picospec_verify_static(const void* target_logits, picospec_dtype 
     a.logits = target_logits; a.row_stride = row_stride_elems;
     a.B = B; a.G = G; a.V = V; a.k_max = k_max; a.sample_only = 0;
     a.nch = (V + CHUNK - 1) / CHUNK;
+    a.r1 = G + 1;
     a.temperature = temperature; a.draft_tok = draft_tok; a.q_idx = q_idx; a.q_prob = q_prob; a.q_count = q_count;
     a.u_accept = u_accept; a.pos = nullptr; a.u_resample = u_resample;
     a.accept_len = accept_len; a.p_draft = p_draft; a.resid_mass = resid_mass; a.borderline = borderline_count;

@@ -18,6 +18,9 @@ struct PreciseArgs {
     const int* queue;
     const int* queue_count;
     const unsigned long long* need_rows;   // optional [entries]: bit ri = row ri of the entry is wanted
+    // optional row window of an entry: rows outside [r0, r1), or beyond gamma[entry], are never read
+    int r0 = 0, r1 = 0x7fffffff;
+    const int* gamma = nullptr;
     const float* row_max;      // [rows] exact row maxima from the fp32 pass
     double* dsum;              // [rows, nch]
 };
@@ -36,6 +39,7 @@ __global__ void __launch_bounds__(THREADS) precise_chunk_sums_kernel(PreciseArgs
         const int ri = (int)(t % a.expand);
         const int e = a.queue[(int)(t / a.expand)];
         if (a.need_rows && !a.pos && ri < 64 && !((a.need_rows[e] >> ri) & 1ull)) continue;
+        if (!a.pos && (ri < a.r0 || ri >= a.r1 || (a.gamma && ri > a.gamma[e]))) continue;
         const int src_row = a.pos ? e * a.seq_rows + a.pos[e] : e * a.expand + ri;
         const int b = src_row / a.seq_rows;
         const T* row = reinterpret_cast<const T*>(a.logits) + (long long)src_row * a.row_stride;

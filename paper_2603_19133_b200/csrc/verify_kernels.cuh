@@ -12,6 +12,12 @@ struct VerifyArgs {
     long long row_stride;      // elements
     int B, G, V, nch, k_max;
     int sample_only;           // 1: residual_sample entry point (row pos[b] only)
+    // incremental verification: only the target rows [r0, r1) are read, for sequences that are
+    // still undecided; the whole batch at once is r0 = 0, r1 = G + 1 with the pointers null
+    int r0 = 0, r1 = -1;
+    const int* gamma = nullptr;     // [B] drafted tokens per sequence (rows 0 .. gamma[b]); null: G
+    const int* state_in = nullptr;  // [B] 1 = undecided so far, 0 = decided earlier (skipped); null: all 1
+    int* state_out = nullptr;       // [B] or null
     const float* temperature;  // [B]
     const int* draft_tok;      // [B,G]
     const int* q_idx;          // [B,G,k_max]
@@ -49,6 +55,18 @@ template <typename T> struct ItemMeta {
     bool valid;
 };
 
+// Row r of the rows a verify call streams -> (sequence, row of the logits tensor); false: the row
+// is not read (sequence decided earlier, or the row lies beyond the sequence's bonus row).
+__device__ __forceinline__ bool streamed_row(const VerifyArgs& a, int r, int& b, int& src_row) {
+    const int nr = a.r1 - a.r0;
+    b = r / nr;
+    const int i = a.r0 + (r - b * nr);
+    src_row = b * (a.G + 1) + i;
+    if (a.state_in && a.state_in[b] == 0) return false;
+    if (a.gamma && i > a.gamma[b]) return false;
+    return true;
+}
+
 template <typename T> __device__ __forceinline__ ItemMeta<T> decode_item(const VerifyArgs& a, long long item) {
     ItemMeta<T> m;
     const int r = (int)(item / a.nch);
@@ -61,8 +79,7 @@ template <typename T> __device__ __forceinline__ ItemMeta<T> decode_item(const V
         if (j < 0 || j > a.G) m.valid = false;
         src_row = b * (a.G + 1) + (m.valid ? j : 0);
     } else {
-        b = r / (a.G + 1);
-        src_row = r;
+        if (!streamed_row(a, r, b, src_row)) m.valid = false;
     }
     const float Tb = a.temperature[b];
     if (!temp_ok(Tb)) m.valid = false;
@@ -95,7 +112,7 @@ __global__ void __launch_bounds__(THREADS, 4) chunk_stats_kernel(VerifyArgs a) {
         *a.queue_count = 0;
         if (a.borderline) *a.borderline = 0;
     }
-    const long long total = (long long)(a.sample_only ? a.B : a.B * (a.G + 1)) * a.nch;
+    const long long total = (long long)(a.sample_only ? a.B : a.B * (a.r1 - a.r0)) * a.nch;
     long long itA = gw;
     if (itA >= total) return;
     ChunkRegs<T> A, Bf;
@@ -132,7 +149,7 @@ struct TileDesc {
     int src_row;   // row of the logits tensor
     int c0;        // first chunk of the tile
     float c32;     // log2(e) / T of the row's sequence
-    int valid;     // 0: bad temperature or position, nothing was copied
+    int valid;     // 0: bad temperature or position, or a row that is not read: nothing was copied
 };
 
 template <typename T>
@@ -182,8 +199,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, StreamCfg<T>::CTAS_PER_SM) chu
                 if (j < 0 || j > a.G) d.valid = 0;
                 d.src_row = b * (a.G + 1) + (d.valid ? j : 0);
             } else {
-                b = r / (a.G + 1);
-                d.src_row = r;
+                if (!streamed_row(a, r, b, d.src_row)) d.valid = 0;
             }
             const float Tb = a.temperature[b];
             if (!temp_ok(Tb)) d.valid = 0;
@@ -306,11 +322,22 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
     for (int slot = blockIdx.x; slot < nloop; slot += gridDim.x) {
         const int b = PRECISE ? a.queue[slot] : slot;
         const unsigned long long need = PRECISE ? a.need_rows[b] : 0ull;   // rows with exact chunk sums
+        if (!a.sample_only && a.state_in && a.state_in[b] == 0) {
+            // decided by an earlier call: nothing of this sequence is read or written
+            if (tid == 0 && a.state_out) a.state_out[b] = 0;
+            continue;
+        }
         const float Tb = a.temperature[b];
         const float c32 = temp_scale(Tb);
         const T* seq = reinterpret_cast<const T*>(a.logits) + (long long)b * G1 * a.row_stride;
         unsigned st_bits = 0;
         if (!temp_ok(Tb)) st_bits |= ST_TEMPERATURE;
+        // rows lo .. row_hi-1 are read, positions lo .. hi-1 are tested; g is the bonus row
+        const int lo = a.sample_only ? 0 : a.r0;
+        const int g = (!a.sample_only && a.gamma) ? a.gamma[b] : G;
+        if (g < 0 || g > G || g < lo) st_bits |= ST_RANGE;
+        const int hi = a.sample_only ? G : min(g, a.r1);
+        const int row_hi = a.sample_only ? G1 : min(g + 1, a.r1);
         __syncthreads();
         if (tid == 0) {
             sh.bad = 0;
@@ -325,8 +352,8 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
             if (jpos < 0 || jpos > G) st_bits |= ST_RANGE;
         }
         if (!st_bits) {
-            for (int i = warp; i < G1; i += WARPS) {
-                if (a.sample_only && i != jpos) continue;
+            const int i_lo = a.sample_only ? jpos : lo, i_hi = a.sample_only ? jpos + 1 : row_hi;
+            for (int i = i_lo + warp; i < i_hi; i += WARPS) {
                 double Z, Zraw;
                 float mx;
                 bool bad;
@@ -344,7 +371,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
 
         // ---- 2. per draft position: p(x), q~(x), accept test, residual mass ----------------
         if (!st_bits && !sh.bad && !a.sample_only) {
-            for (int i = warp; i < G; i += WARPS) {
+            for (int i = lo + warp; i < hi; i += WARPS) {
                 const int ri = b * G + i;
                 const int x = a.draft_tok[ri];
                 const int n = a.q_count[ri];
@@ -433,12 +460,16 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
         st_bits |= (unsigned)sh.bad;
 
         // ---- 3. first-rejection scan -----------------------------------------------------
-        int alen = 0, nborder = 0;
-        bool flagged = false;
+        // A rejection inside the range decides the sequence; so does accepting every position
+        // when the bonus row g is in the range.  Otherwise it waits for the next rows.
+        int alen = lo, nborder = 0;
+        bool flagged = false, rejected = false, decided = true;
         if (!st_bits && !a.sample_only) {
-            while (alen < G && sh.acc[alen]) ++alen;
-            const int last = alen < G ? alen : G - 1;
-            for (int i = 0; i <= last; ++i) {
+            while (alen < hi && sh.acc[alen]) ++alen;
+            rejected = alen < hi;
+            decided = rejected || g < a.r1;
+            const int last = rejected ? alen : hi - 1;
+            for (int i = lo; i <= last; ++i) {
                 flagged |= sh.amb[i] != 0;
                 nborder += sh.bord[i];
             }
@@ -448,11 +479,11 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
         int token = -1;
         double Rtot = -1.0;
         const bool want_token = a.token != nullptr;
-        if (!st_bits && want_token) {
+        if (!st_bits && want_token && decided) {
             const int j = a.sample_only ? jpos : alen;
             const int rj = b * G + j;
             int n = 0;
-            if (j < G) {
+            if (a.sample_only ? j < G : rejected) {
                 n = a.q_count[rj];
                 if (n < 0 || n > a.k_max) {
                     n = 0;
@@ -632,16 +663,20 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 atomicOr(a.status, st_bits);
                 if (!a.sample_only) {
                     a.accept_len[b] = -1;
-                    for (int i = 0; i < G; ++i) {
+                    for (int i = lo; i < hi && i < G; ++i) {
                         a.p_draft[b * G + i] = -1.f;
                         a.resid_mass[b * G + i] = -1.f;
                     }
+                    if (a.state_out) a.state_out[b] = 0;
                 }
                 if (want_token) a.token[b] = -1;
                 if (a.mass) a.mass[b] = -1.f;
             } else {
-                if (!a.sample_only) a.accept_len[b] = alen;
-                if (want_token) a.token[b] = token;
+                if (!a.sample_only) {
+                    a.accept_len[b] = decided ? alen : -2;
+                    if (a.state_out) a.state_out[b] = decided ? 0 : 1;
+                }
+                if (want_token) a.token[b] = decided ? token : -2;
                 if (a.mass) a.mass[b] = (float)Rtot;
                 if (PRECISE) {
                     if (nborder && a.borderline) atomicAdd(a.borderline, nborder);
@@ -656,11 +691,12 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                         nrows = 1;
                     } else {
                         int first_amb = -1;
-                        const int last = alen < G ? alen : G - 1;
-                        for (int i = 0; i <= last && first_amb < 0; ++i)
+                        const int last = rejected ? alen : hi - 1;
+                        for (int i = lo; i <= last && first_amb < 0; ++i)
                             if (sh.amb[i]) first_amb = i;
-                        for (int i = 0; i < G1; ++i) {
-                            const bool nr = i >= 64 || (first_amb >= 0 && i >= first_amb) || (sh.flag && want_token && i == alen);
+                        for (int i = lo; i < row_hi; ++i) {
+                            const bool nr = i >= 64 || (first_amb >= 0 && i >= first_amb) ||
+                                            (sh.flag && want_token && decided && i == alen);
                             if (nr) {
                                 if (i < 64) nd |= 1ull << i;
                                 ++nrows;

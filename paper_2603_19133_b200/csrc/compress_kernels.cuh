@@ -273,10 +273,11 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
     // stored probabilities, and their running sum for the draft draw
     float pf[4];
     double ploc = 0.0, pcum[4];
+    const double inv = 1.0 / (a.raw_probs ? Z : Wn);   // one division per row; 2^-53 relative per entry
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
         const int j = tid * 4 + e;
-        pf[e] = j < n ? (float)(w[e] / (a.raw_probs ? Z : Wn)) : 0.f;
+        pf[e] = j < n ? (float)(w[e] * inv) : 0.f;
         ploc += (double)pf[e];
         pcum[e] = ploc;
     }

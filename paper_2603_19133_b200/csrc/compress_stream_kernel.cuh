@@ -11,11 +11,15 @@
 //     staged tile) to the warp's own region of the candidate buffer: no atomics with a return
 //     value, no CTA barrier.  About 15 of the 1024 values of a chunk pass, so this is two or three
 //     steps per chunk;
-//   - every stored candidate is counted in a two-level histogram over the top 12 bits of the
-//     orderable logit; thr is the lower edge of the highest bin whose suffix count reaches k, so
-//     it is a valid bound whenever it is computed, by any warp, from whatever has been counted so
-//     far.  The warps take turns refreshing it, once per tile; a warp whose region fills
-//     refreshes it and drops its candidates below it;
+//   - every stored candidate is counted in a two-level histogram whose bins count up from the
+//     first tile's bound, one bin per 16-bit logit code (the top 16 bits of the orderable key: a
+//     bf16 value, 2^-7 relative for fp32), magnitudes below 2^-10 sharing one bin on each side of
+//     zero so that a window that crosses zero does not spend itself on tiny exponents; 4096 bins
+//     reach 32 binades up, whatever lies beyond shares the last bin; thr is the lower edge of the
+//     highest bin whose suffix count reaches k, so it is a valid bound whenever it is computed,
+//     by any warp, from whatever has been counted so far.
+//     The warps take turns refreshing it, once per tile; a warp whose region fills refreshes it
+//     and drops its candidates below it;
 //   - the first tile of a row gets its bound without the histogram: every warp finds, by a
 //     16-step bisection over its own chunk, a value that at least ceil(k/8) of its small groups
 //     of elements reach with their maximum; the smallest of the eight values is reached by at
@@ -39,8 +43,8 @@ namespace picospec {
 // candidate buffer and two stages leave room for three CTAs per SM; larger k takes the big buffer.
 constexpr int CS_CAP_SMALL = 2048, CS_CAP_LARGE = 4096;    // candidate keys held in shared memory
 constexpr int CS_K_SMALL = 256;                            // largest k served by the small shape
-constexpr int CS_BIN_SHIFT = 20;
-constexpr int CS_BINS = 4096;        // histogram bins: top 12 bits of the orderable logit
+constexpr int CS_BINS = 4096;        // histogram bins above the first tile's bound; the last one is open-ended
+constexpr int CS_DEAD = 117 << 7;    // 16-bit magnitude codes below 2^-10: one bin on each side of zero
 constexpr int CS_SUPER = CS_BINS / 32;
 // Bin counts are 16 bits wide, two per word (super-bin counts are 32-bit).  A count can only wrap
 // on rows that push tens of thousands of values into one bin; a wrap makes a sum too small (a
@@ -55,7 +59,7 @@ struct CsRowMeta {
     int count;        // survivors written for the row
     int flags;
     float ref_off;    // fp32(ref * c32): reference of the streamed normaliser
-    float pad;
+    unsigned thr_key; // the row's final bound: every survivor's orderable logit is at least this
     double z_stream;  // sum of 2^(l * c32 - ref_off) over the row (top-p only)
 };
 
@@ -179,6 +183,26 @@ __device__ __forceinline__ unsigned first_tile_key(const ChunkRegs<T>& regs, int
 }
 
 // two-level histogram update
+// Bin coordinate of a 16-bit orderable code (monotone): the code itself with the magnitudes
+// below 2^-10 squeezed onto 0x7FFF (negative side) and 0x8000 (positive side).
+__device__ __forceinline__ int bin_coord(unsigned o16) {
+    const bool pos = o16 >= 0x8000u;
+    const int mag = pos ? (int)o16 - 0x8000 : 0x7FFF - (int)o16;
+    const int c = max(mag - CS_DEAD, 0);
+    return pos ? 0x8000 + c : 0x7FFF - c;
+}
+// smallest 16-bit code whose coordinate is at least G
+__device__ __forceinline__ unsigned coord_code(int G) {
+    if (G >= 0x8000) {
+        const int c = G - 0x8000;
+        return (unsigned)(c ? 0x8000 + c + CS_DEAD : 0x8000);
+    }
+    return (unsigned)(0x7FFF - ((0x7FFF - G) + CS_DEAD));
+}
+// bin of an orderable key at or above the first tile's bound (coordinate g0)
+__device__ __forceinline__ int hist_bin(unsigned okey, int g0) {
+    return min(bin_coord(okey >> 16) - g0, CS_BINS - 1);
+}
 __device__ __forceinline__ void hist_add(unsigned* hist, int bin) {
     atomicAdd(&hist[bin >> 1], (bin & 1) ? 0x10000u : 1u);
     atomicAdd(&hist[CS_BINS / 2 + (bin >> 5)], 1u);
@@ -223,7 +247,10 @@ __device__ __forceinline__ void refresh_threshold(const unsigned* hist, CsShared
     }
     const unsigned hit2 = __ballot_sync(0xffffffffu, above + bs >= (unsigned)k);
     const int found = hit2 ? 32 * s + (31 - __clz(hit2)) : 32 * s;
-    if (lane == 0) atomicMax(&cs.thr_key, (unsigned)found << CS_BIN_SHIFT);
+    if (lane == 0) {
+        const int g0 = bin_coord(*(volatile unsigned*)&cs.thr0_key >> 16);
+        atomicMax(&cs.thr_key, coord_code(g0 + found) << 16);
+    }
 }
 
 // Warp-local: drop the entries of this warp's region below thr (stable, in place).
@@ -347,6 +374,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
         const float c32 = temp_scale(Tb);
         float ref_off = 0.f, acc = 0.f;
         int wcount = 0;             // candidates in this warp's region
+        int g0 = 0;                 // bin coordinate of the first tile's bound: origin of the histogram
         bool full_region = false;   // the region ran out of room (the row goes to the redo list)
 
         for (int ti = 0; ti < tiles_per_row; ++ti, ++i) {
@@ -383,7 +411,9 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
                     }
                 }
                 workers_sync();
-                if (lane == 0) atomicMax(&cs.thr_key, *(volatile unsigned*)&cs.thr0_key);
+                const unsigned thr0 = *(volatile unsigned*)&cs.thr0_key;
+                g0 = bin_coord(thr0 >> 16);
+                if (lane == 0) atomicMax(&cs.thr_key, thr0);
                 if (STATS) ref_off = __fmul_rn(from_orderable(*(volatile unsigned*)&cs.top_key), c32);
                 __syncwarp();
             }
@@ -426,7 +456,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
                 }
                 __syncwarp();
                 // count the new entries in the histogram
-                for (int x = before + lane; x < wcount; x += 32) hist_add(hist, (int)(region[x] >> (32 + CS_BIN_SHIFT)));
+                for (int x = before + lane; x < wcount; x += 32) hist_add(hist, hist_bin((unsigned)(region[x] >> 32), g0));
                 // the bound is refreshed after every tile, each time by another warp (the others'
                 // latest values may not be counted yet, which only makes it a little lower)
                 if (warp == (ti & (WARPS - 1))) {
@@ -481,7 +511,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
             meta.count = m;
             meta.flags = flags;
             meta.ref_off = ref_off;
-            meta.pad = 0.f;
+            meta.thr_key = cs.thr_key;
             meta.z_stream = zs;
             a.surv_meta[row] = meta;
             // reset the row state
@@ -497,12 +527,125 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
     }
 }
 
-// One CTA per row: sort the survivors, then cut / renormalise / emit.
+// ---- block-wide sort in registers ----------------------------------------------------------------
+// Bitonic network (descending) over N = 256 * R keys, R per thread: element e = warp * 32R + r * 32
+// + lane sits in register r of that lane.  Strides below 32 are warp shuffles, strides 32 .. 16R
+// are compare-exchanges between two registers of one thread, and only the three largest strides
+// of a merge cross warps: those go through shared memory (two buffers in turn, one barrier per
+// stage).  Keys are unsigned and larger = earlier; equal keys are interchangeable.
+__device__ __forceinline__ uint32_t shfl_xor_key(uint32_t k, int d) { return __shfl_xor_sync(0xffffffffu, k, d); }
+__device__ __forceinline__ u64 shfl_xor_key(u64 k, int d) {
+    const uint32_t lo = __shfl_xor_sync(0xffffffffu, (uint32_t)k, d);
+    const uint32_t hi = __shfl_xor_sync(0xffffffffu, (uint32_t)(k >> 32), d);
+    return ((u64)hi << 32) | lo;
+}
+template <typename K> __device__ __forceinline__ K key_pick(K mine, K other, bool keep_max) {
+    const K hi = mine > other ? mine : other, lo = mine > other ? other : mine;
+    return keep_max ? hi : lo;
+}
+
+template <typename K, int R>
+__device__ __forceinline__ void block_sort_desc(K (&key)[R], K* buf) {
+    constexpr int N = THREADS * R;
+    const int lane = threadIdx.x & 31;
+    const int ebase = (threadIdx.x >> 5) * (32 * R) + lane;
+    int phase = 0;
+#pragma unroll
+    for (int size = 2; size <= N; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            if (stride >= 32 * R) {
+                K* bp = buf + (phase & 1) * N;
+                ++phase;
+#pragma unroll
+                for (int r = 0; r < R; ++r) bp[ebase + 32 * r] = key[r];
+                __syncthreads();
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const int e = ebase + 32 * r;
+                    key[r] = key_pick(key[r], bp[e ^ stride], ((e & size) == 0) == ((e & stride) == 0));
+                }
+            } else if (stride >= 32) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const int dr = stride >> 5;
+                    if ((r & dr) == 0) {
+                        const bool desc = ((ebase + 32 * r) & size) == 0;
+                        const K x = key[r], y = key[r + dr];
+                        const K hi = x > y ? x : y, lo = x > y ? y : x;
+                        key[r] = desc ? hi : lo;
+                        key[r + dr] = desc ? lo : hi;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const int e = ebase + 32 * r;
+                    key[r] = key_pick(key[r], shfl_xor_key(key[r], stride), ((e & size) == 0) == ((lane & stride) == 0));
+                }
+            }
+        }
+    }
+}
+
+// Sort `count` keys held in shared memory at in[0 .. count) (the rest of the 256R-element network
+// is padding) into out[0 .. 256R), as 64-bit keys, largest first.  `in` may be either exchange
+// buffer; out is the first.  NARROW: 16-bit logits whose codes lie in [lo16, lo16 + 2^14) and
+// V <= 2^18 run the network on 32-bit keys, (code - lo16) << 18 | index complement.
+template <int R, bool NARROW>
+__device__ __noinline__ void sort_keys(const u64* in, int count, u64* out, unsigned lo16) {
+    const int lane = threadIdx.x & 31;
+    const int ebase = (threadIdx.x >> 5) * (32 * R) + lane;
+    u64 k[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int e = ebase + 32 * r;
+        k[r] = e < count ? in[e] : 0ull;
+    }
+    __syncthreads();                // every key is in registers: the buffers are free
+    if (NARROW) {
+        uint32_t n[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+            n[r] = ebase + 32 * r < count ? ((((uint32_t)(k[r] >> 48) - lo16) << 18) | ((uint32_t)k[r] & 0x3FFFFu)) : 0u;
+        block_sort_desc<uint32_t, R>(n, reinterpret_cast<uint32_t*>(out));
+        __syncthreads();
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const uint32_t o16 = (n[r] >> 18) + lo16;
+            // a 16-bit logit's orderable form ends in sixteen ones when the logit is negative
+            const uint32_t o32 = (o16 << 16) | ((o16 & 0x8000u) ? 0u : 0xFFFFu);
+            out[ebase + 32 * r] = ((u64)o32 << 32) | (u64)(0xFFFC0000u | (n[r] & 0x3FFFFu));
+        }
+    } else {
+        block_sort_desc<u64, R>(k, out);
+        __syncthreads();
+#pragma unroll
+        for (int r = 0; r < R; ++r) out[ebase + 32 * r] = k[r];
+    }
+    __syncthreads();
+}
+
+constexpr int CS_TIE_CAP = 256;     // boundary-group size up to which the survivors are trimmed to k
+
+struct CsFinishShared {
+    unsigned hi16;      // largest 16-bit logit code among the survivors
+    int above;          // survivors whose code is above the bound's
+    int kept, ties;     // slot counters of the trim pass
+};
+
+// One CTA per row: trim the survivors to the k best where that is cheap, sort, cut / renormalise /
+// emit.  The survivors are all elements at or above the filter's final bound, i.e. the k best plus
+// whatever shares the bound's 16-bit code with the k-th (ties of a 16-bit logit; values within
+// 2^-7 relative of it for 32-bit logits).  When they would need a larger sort network than k
+// keys do, the members of that boundary group are ranked among themselves (all pairs) and only
+// the best k - (number above the group) are kept.
 template <typename T, bool STATS>
-__global__ void __launch_bounds__(THREADS) compress_finish_kernel(CompressArgs a) {
-    extern __shared__ u64 keys[];          // [pow2 >= survivors]
+__global__ void __launch_bounds__(THREADS) compress_finish_kernel(CompressArgs a, int n2cap) {
+    extern __shared__ u64 keys[];          // two exchange buffers of n2cap keys; the sorted keys end up in the first
     __shared__ CompressShared sh;
-    const int tid = threadIdx.x;
+    __shared__ CsFinishShared fs;
+    const int tid = threadIdx.x, lane = tid & 31;
     const int row = blockIdx.x;
     int k_eff = a.top_k > 0 ? a.top_k : a.k_max;
     if (k_eff > a.k_max) k_eff = a.k_max;
@@ -516,13 +659,94 @@ __global__ void __launch_bounds__(THREADS) compress_finish_kernel(CompressArgs a
         return;
     }
     const int m = meta.count;
-    int n2 = 1;
-    while (n2 < m) n2 <<= 1;
+    const unsigned thr16 = meta.thr_key >> 16;
     const u64* src = a.surv_keys + (long long)row * cs_survivor_cap(a.k_max);
-    for (int x = tid; x < n2; x += THREADS) keys[x] = x < m ? src[x] : 0ull;
-    bitonic_sort_desc(keys, n2);
-    const float top = key_logit(keys[0]);
     const float Tb = a.temperature[row / a.G];
+    u64* bufA = keys;
+    u64* bufB = keys + n2cap;
+    if (tid == 0) {
+        fs.hi16 = 0u;
+        fs.above = 0;
+        fs.kept = 0;
+        fs.ties = 0;
+    }
+    __syncthreads();
+    // ---- survivors to shared memory (buffer B); largest code, size of the part above the bound's code
+    {
+        unsigned hi = 0u;
+        int above = 0;
+        for (int e = tid; e < m; e += THREADS) {
+            const u64 key = src[e];
+            bufB[e] = key;
+            const unsigned code = (unsigned)(key >> 48);
+            hi = max(hi, code);
+            above += code > thr16 ? 1 : 0;
+        }
+        hi = __reduce_max_sync(0xffffffffu, hi);
+        above = __reduce_add_sync(0xffffffffu, above);
+        if (lane == 0) {
+            atomicMax(&fs.hi16, hi);
+            if (above) atomicAdd(&fs.above, above);
+        }
+    }
+    __syncthreads();
+    const int above = fs.above;
+    const bool narrow = sizeof(T) == 2 && a.V <= (1 << 18) && fs.hi16 - thr16 < (1u << 14);
+    int nk = 256;                       // network size for k keys
+    while (nk < k_eff) nk <<= 1;
+    int nm = 256;                       // network size for all m survivors
+    while (nm < m) nm <<= 1;
+    const u64* in = bufB;
+    int count = m, n2 = nm;
+    if (nm > nk && above < k_eff && m - above <= CS_TIE_CAP) {
+        // ---- trim: everything above the bound's code, plus the best of the boundary group --------
+        // (nk <= n2cap / 2 here, so the boundary group fits behind the nk output slots of buffer A)
+        u64* tie = bufA + nk;
+        const unsigned lt = (1u << lane) - 1u;
+        for (int e0 = 0; e0 < m; e0 += THREADS) {
+            const int e = e0 + tid;
+            const u64 key = e < m ? bufB[e] : 0ull;
+            const bool is_above = e < m && (unsigned)(key >> 48) > thr16;
+            const bool is_tie = e < m && !is_above;
+            const unsigned ma = __ballot_sync(0xffffffffu, is_above), mt = __ballot_sync(0xffffffffu, is_tie);
+            int ba = 0, bt = 0;
+            if (lane == 0) {
+                if (ma) ba = atomicAdd(&fs.kept, __popc(ma));
+                if (mt) bt = atomicAdd(&fs.ties, __popc(mt));
+            }
+            ba = __shfl_sync(0xffffffffu, ba, 0);
+            bt = __shfl_sync(0xffffffffu, bt, 0);
+            if (is_above) bufA[ba + __popc(ma & lt)] = key;
+            if (is_tie) tie[bt + __popc(mt & lt)] = key;
+        }
+        __syncthreads();
+        const int t = m - above, need = k_eff - above;
+        for (int j = tid; j < t; j += THREADS) {
+            const u64 key = tie[j];
+            int rank = 0;
+            for (int x = 0; x < t; ++x) rank += tie[x] > key ? 1 : 0;
+            if (rank < need) bufA[above + rank] = key;      // keys are distinct: every rank is taken once
+        }
+        __syncthreads();
+        in = bufA;
+        count = k_eff;
+        n2 = nk;
+    }
+    // the boundary group's ranks are written (or nothing was): sort `count` keys from `in`
+    // (sort_keys moves them to registers before either buffer is reused)
+    const int R = n2 >> 8;
+    if (narrow) {
+        if (R == 1) sort_keys<1, true>(in, count, bufA, thr16);
+        else if (R == 2) sort_keys<2, true>(in, count, bufA, thr16);
+        else if (R == 4) sort_keys<4, true>(in, count, bufA, thr16);
+        else sort_keys<8, true>(in, count, bufA, thr16);
+    } else {
+        if (R == 1) sort_keys<1, false>(in, count, bufA, 0u);
+        else if (R == 2) sort_keys<2, false>(in, count, bufA, 0u);
+        else if (R == 4) sort_keys<4, false>(in, count, bufA, 0u);
+        else sort_keys<8, false>(in, count, bufA, 0u);
+    }
+    const float top = key_logit(keys[0]);
     double Z = 0.0;
     if (STATS) {
         // move the streamed sum from its reference onto the scale of the weights exp(l/T - top/T)

@@ -164,8 +164,9 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
             int n2 = 1;
             while (n2 < cs_survivor_cap(a.k_max)) n2 <<= 1;
             ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_FINISH, 2, s);
-            if (stats) compress_finish_kernel<T, true><<<rows, THREADS, (size_t)n2 * 8, s>>>(a);
-            else compress_finish_kernel<T, false><<<rows, THREADS, (size_t)n2 * 8, s>>>(a);
+            // two exchange buffers of the sort network (the sorted keys end up in the first)
+            if (stats) compress_finish_kernel<T, true><<<rows, THREADS, (size_t)n2 * 16, s>>>(a, n2);
+            else compress_finish_kernel<T, false><<<rows, THREADS, (size_t)n2 * 16, s>>>(a, n2);
         }
         e0 = cudaGetLastError();
         if (e0 != cudaSuccess) return e0;

@@ -373,37 +373,45 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
         if (!st_bits && !sh.bad && !a.sample_only) {
             for (int i = lo + warp; i < hi; i += WARPS) {
                 const int ri = b * G + i;
+                const int* idx = a.q_idx + (long long)ri * a.k_max;
+                const float* prob = a.q_prob + (long long)ri * a.k_max;
+                const T* row = seq + (long long)i * a.row_stride;
+                // the first batch of stored entries is requested before the row's count is known
+                // (every slot below k_max exists; slots at or beyond the count are dropped below)
+                int vv[8];
+                float qq[8], ll[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int k = u * 32 + lane;
+                    vv[u] = k < a.k_max ? idx[k] : -2;
+                    qq[u] = k < a.k_max ? prob[k] : 0.f;
+                }
                 const int x = a.draft_tok[ri];
                 const int n = a.q_count[ri];
+                const float ux = a.u_accept[ri];
                 bool range_bad = (x < 0 || x >= a.V || n < 0 || n > a.k_max);
-                const T* row = seq + (long long)i * a.row_stride;
                 Weight<PRECISE> wt;
                 wt.init(Tb, sh.mx[i]);
                 const double Z = sh.Z[i];
+                const double invZ = 1.0 / Z;     // the sums below take p = w * (1/Z): 2^-53 relative per term
                 double smin = 0.0;
                 float qx = 0.f, qx_mine = 0.f;
                 int kx = 0x7fffffff;
-                // issued early: the logit of the draft token and its uniform (lane 0 uses them last)
-                float lx = -CUDART_INF_F, ux = 0.f;
-                if (!range_bad && lane == 0) {
-                    lx = load_logit(row, x);
-                    ux = a.u_accept[ri];
-                }
+                // p(x) on every lane (the same instructions as on one lane, and no divergent tail)
+                const float lx = range_bad ? -CUDART_INF_F : load_logit(row, x);
                 if (!range_bad) {
-                    const int* idx = a.q_idx + (long long)ri * a.k_max;
-                    const float* prob = a.q_prob + (long long)ri * a.k_max;
-                    // eight entries per lane at a time: all index loads, then all logit gathers
                     for (int k0 = 0; k0 < n; k0 += 256) {
-                        int vv[8];
-                        float qq[8], ll[8];
+                        if (k0 > 0) {
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            const int k = k0 + u * 32 + lane;
-                            vv[u] = k < n ? idx[k] : -2;
-                            qq[u] = k < n ? prob[k] : 0.f;
+                            for (int u = 0; u < 8; ++u) {
+                                const int k = k0 + u * 32 + lane;
+                                vv[u] = k < n ? idx[k] : -2;
+                                qq[u] = k < n ? prob[k] : 0.f;
+                            }
                         }
 #pragma unroll
                         for (int u = 0; u < 8; ++u) {
+                            if (k0 + u * 32 + lane >= n) vv[u] = -2;
                             const bool ok = vv[u] >= 0 && vv[u] < a.V;
                             if (vv[u] != -2 && !ok) range_bad = true;
                             ll[u] = ok ? load_logit(row, vv[u]) : -CUDART_INF_F;
@@ -412,7 +420,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                         for (int u = 0; u < 8; ++u) {
                             const int k = k0 + u * 32 + lane;
                             if (vv[u] >= 0 && vv[u] < a.V) {
-                                const double pk = wt(ll[u]) / Z;
+                                const double pk = wt(ll[u]) * invZ;
                                 smin += fmin(pk, (double)qq[u]);
                                 if (vv[u] == x && k < kx) {
                                     kx = k;
@@ -422,6 +430,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                         }
                     }
                 }
+                const double px = wt(lx) / Z;
                 range_bad = __any_sync(0xffffffffu, range_bad);
                 smin = warp_sum(smin);
 #pragma unroll
@@ -433,7 +442,6 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                     if (range_bad) {
                         atomicOr(&sh.bad, (int)ST_RANGE);
                     } else {
-                        const double px = wt(lx) / Z;
                         const double u = (double)ux;
                         int acc = 1, amb = 0, bord = 0;
                         if (qx > 0.f) {
@@ -496,11 +504,12 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
             Weight<PRECISE> wt;
             wt.init(Tb, sh.mx[j]);
             const double Z = sh.Z[j];
+            const double invZ = 1.0 / Z;
             bool use_resid = n > 0;
             for (int pass = 0; pass < 2 && !st_bits; ++pass) {
                 // chunk masses (in units where the row sums to one)
                 if (PRECISE && row_needed(need, j)) {
-                    for (int c = tid; c < a.nch; c += THREADS) cm[c] = a.dsum[(long long)(b * G1 + j) * a.nch + c] / Z;
+                    for (int c = tid; c < a.nch; c += THREADS) cm[c] = a.dsum[(long long)(b * G1 + j) * a.nch + c] * invZ;
                 } else {
                     const float2* st = a.stats + (long long)(b * G1 + j) * a.nch;
                     const double off = (double)__fmul_rn(sh.mx[j], c32);
@@ -532,7 +541,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
 #pragma unroll
                         for (int u = 0; u < 4; ++u)
                             if (vv[u] >= 0 && vv[u] < a.V)
-                                atomicAdd(&cm[vv[u] / CHUNK], -fmin(wt(ll[u]) / Z, (double)qq[u]));
+                                atomicAdd(&cm[vv[u] / CHUNK], -fmin(wt(ll[u]) * invZ, (double)qq[u]));
                     }
                     if (rb) atomicOr(&sh.bad, (int)ST_RANGE);
                 }
@@ -616,7 +625,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 for (int e = 0; e < 4; ++e) {
                     const int v = v0 + tid * 4 + e;
                     double w = 0.0;
-                    if (v < a.V) w = wt(load_logit(row, v)) / Z;
+                    if (v < a.V) w = wt(load_logit(row, v)) * invZ;
                     const double q = (double)sh.qloc[tid * 4 + e];
                     qsum += q;
                     double d = w - q;

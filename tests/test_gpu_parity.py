@@ -396,6 +396,28 @@ def test_staged_shapes(ps, V, B, G, K, dtype, top_k, top_p):
     assert r["status"] == 0
 
 
+@pytest.mark.parametrize("V,k,shift", [
+    (32000, 8, 24.0),         # up to 256 survivors: one key per thread
+    (128256, 64, 24.0),
+    (128256, 256, 6.0),       # two keys per thread; survivors within a few binades above zero
+    (262144, 512, 24.0),      # four keys per thread, the largest vocabulary index the 32-bit key holds
+    (50304, 1024, 3.0),       # eight keys per thread
+    (128256, 256, -4.0),      # all negative: the complemented key range
+    (128256, 256, 0.75),      # survivors on both sides of zero: far more than 2^14 key values apart
+])
+def test_finish_sort_key_widths(ps, V, k, shift):
+    # The finish kernel sorts 16-bit-logit survivors on 32-bit keys when their logit keys span
+    # fewer than 2^14 values (survivors of one sign and a few binades, as with positive or negative
+    # top logits), on 64-bit keys otherwise; coarse bf16 values make ties that the index must break.
+    w = gen.sweep_workload(V, k, B=4)
+    inputs = gen.make_inputs(w, seed=7000 + k, device="cuda")
+    for key in ("draft_logits", "target_logits"):
+        inputs[key] = (inputs[key].float() + shift).to(torch.bfloat16)
+    r = run_both(ps, w, inputs)
+    assert r["status"] == 0
+    assert r["redo_rows"] == 0
+
+
 def _custom_inputs(dl, tl, seed):
     B, G, V = dl.shape
     g = torch.Generator(device="cuda").manual_seed(seed)

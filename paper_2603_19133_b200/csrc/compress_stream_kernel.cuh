@@ -630,8 +630,7 @@ constexpr int CS_TIE_CAP = 256;     // boundary-group size up to which the survi
 
 struct CsFinishShared {
     unsigned hi16;      // largest 16-bit logit code among the survivors
-    int above;          // survivors whose code is above the bound's
-    int kept, ties;     // slot counters of the trim pass
+    int kept, ties;     // slot counters: survivors above the bound's code / with it
 };
 
 // One CTA per row: trim the survivors to the k best where that is cheap, sort, cut / renormalise /
@@ -650,6 +649,9 @@ __global__ void __launch_bounds__(THREADS) compress_finish_kernel(CompressArgs a
     int k_eff = a.top_k > 0 ? a.top_k : a.k_max;
     if (k_eff > a.k_max) k_eff = a.k_max;
     if (k_eff > a.V) k_eff = a.V;
+    const u64* src = a.surv_keys + (long long)row * cs_survivor_cap(a.k_max);
+    // the first 512 scratch slots exist for every k_max: requested before the row's count is known
+    const u64 first0 = src[tid], first1 = src[tid + THREADS];
     const CsRowMeta meta = a.surv_meta[row];
     if (meta.flags & CSF_REDO) return;                 // the direct kernel writes this row
     if (meta.flags) {
@@ -660,54 +662,27 @@ __global__ void __launch_bounds__(THREADS) compress_finish_kernel(CompressArgs a
     }
     const int m = meta.count;
     const unsigned thr16 = meta.thr_key >> 16;
-    const u64* src = a.surv_keys + (long long)row * cs_survivor_cap(a.k_max);
     const float Tb = a.temperature[row / a.G];
     u64* bufA = keys;
     u64* bufB = keys + n2cap;
     if (tid == 0) {
         fs.hi16 = 0u;
-        fs.above = 0;
         fs.kept = 0;
         fs.ties = 0;
     }
     __syncthreads();
-    // ---- survivors to shared memory (buffer B); largest code, size of the part above the bound's code
+    // ---- survivors to shared memory: those above the bound's code to buffer A, the boundary group
+    // ---- to buffer B, both in arrival order (warp-aggregated slots)
     {
-        unsigned hi = 0u;
-        int above = 0;
-        for (int e = tid; e < m; e += THREADS) {
-            const u64 key = src[e];
-            bufB[e] = key;
-            const unsigned code = (unsigned)(key >> 48);
-            hi = max(hi, code);
-            above += code > thr16 ? 1 : 0;
-        }
-        hi = __reduce_max_sync(0xffffffffu, hi);
-        above = __reduce_add_sync(0xffffffffu, above);
-        if (lane == 0) {
-            atomicMax(&fs.hi16, hi);
-            if (above) atomicAdd(&fs.above, above);
-        }
-    }
-    __syncthreads();
-    const int above = fs.above;
-    const bool narrow = sizeof(T) == 2 && a.V <= (1 << 18) && fs.hi16 - thr16 < (1u << 14);
-    int nk = 256;                       // network size for k keys
-    while (nk < k_eff) nk <<= 1;
-    int nm = 256;                       // network size for all m survivors
-    while (nm < m) nm <<= 1;
-    const u64* in = bufB;
-    int count = m, n2 = nm;
-    if (nm > nk && above < k_eff && m - above <= CS_TIE_CAP) {
-        // ---- trim: everything above the bound's code, plus the best of the boundary group --------
-        // (nk <= n2cap / 2 here, so the boundary group fits behind the nk output slots of buffer A)
-        u64* tie = bufA + nk;
         const unsigned lt = (1u << lane) - 1u;
+        unsigned hi = 0u;
         for (int e0 = 0; e0 < m; e0 += THREADS) {
             const int e = e0 + tid;
-            const u64 key = e < m ? bufB[e] : 0ull;
-            const bool is_above = e < m && (unsigned)(key >> 48) > thr16;
+            const u64 key = e0 == 0 ? first0 : e0 == THREADS ? first1 : (e < m ? src[e] : 0ull);
+            const unsigned code = (unsigned)(key >> 48);
+            const bool is_above = e < m && code > thr16;
             const bool is_tie = e < m && !is_above;
+            if (e < m) hi = max(hi, code);
             const unsigned ma = __ballot_sync(0xffffffffu, is_above), mt = __ballot_sync(0xffffffffu, is_tie);
             int ba = 0, bt = 0;
             if (lane == 0) {
@@ -717,21 +692,35 @@ __global__ void __launch_bounds__(THREADS) compress_finish_kernel(CompressArgs a
             ba = __shfl_sync(0xffffffffu, ba, 0);
             bt = __shfl_sync(0xffffffffu, bt, 0);
             if (is_above) bufA[ba + __popc(ma & lt)] = key;
-            if (is_tie) tie[bt + __popc(mt & lt)] = key;
+            if (is_tie) bufB[bt + __popc(mt & lt)] = key;
         }
-        __syncthreads();
-        const int t = m - above, need = k_eff - above;
+        hi = __reduce_max_sync(0xffffffffu, hi);
+        if (lane == 0) atomicMax(&fs.hi16, hi);
+    }
+    __syncthreads();
+    const int above = fs.kept, t = m - above;
+    const bool narrow = sizeof(T) == 2 && a.V <= (1 << 18) && fs.hi16 - thr16 < (1u << 14);
+    int nk = 256;                       // network size for k keys
+    while (nk < k_eff) nk <<= 1;
+    int nm = 256;                       // network size for all m survivors
+    while (nm < m) nm <<= 1;
+    int count = m, n2 = nm;
+    if (nm > nk && above < k_eff && t <= CS_TIE_CAP) {
+        // trim: of the boundary group only the best k - above, each placed by its rank in the group
+        const int need = k_eff - above;
         for (int j = tid; j < t; j += THREADS) {
-            const u64 key = tie[j];
+            const u64 key = bufB[j];
             int rank = 0;
-            for (int x = 0; x < t; ++x) rank += tie[x] > key ? 1 : 0;
+            for (int x = 0; x < t; ++x) rank += bufB[x] > key ? 1 : 0;
             if (rank < need) bufA[above + rank] = key;      // keys are distinct: every rank is taken once
         }
-        __syncthreads();
-        in = bufA;
         count = k_eff;
         n2 = nk;
+    } else {
+        for (int j = tid; j < t; j += THREADS) bufA[above + j] = bufB[j];
     }
+    __syncthreads();
+    const u64* in = bufA;
     // the boundary group's ranks are written (or nothing was): sort `count` keys from `in`
     // (sort_keys moves them to registers before either buffer is reused)
     const int R = n2 >> 8;

@@ -242,6 +242,16 @@ template <typename T> __device__ __forceinline__ float lane_exp_sum(const ChunkR
 // brings such a sum onto the scale of these weights (what remains is the bounded error GUARD_Z).
 // The fast path and the double-precision re-evaluation use the same weights; they differ in
 // where the normaliser comes from.
+// Every kernel is launched with programmatic stream serialization: its CTAs may be scheduled while
+// the kernel before it in the stream is still draining.  Each thread waits here, before its first
+// access to global memory, until that kernel has completed and its writes are visible; then the
+// CTA allows the kernel after it to be scheduled in the same way.  (Without the launch attribute
+// both instructions do nothing.)
+__device__ __forceinline__ void grid_dependency_sync() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 template <bool PRECISE> struct Weight {
     double t, m;
     __device__ __forceinline__ void init(float T, float row_max) {

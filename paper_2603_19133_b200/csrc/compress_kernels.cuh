@@ -333,6 +333,7 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
 
 template <typename T, bool ALIGNED, bool STATS>
 __global__ void __launch_bounds__(THREADS, 2) compress_kernel(CompressArgs a) {
+    grid_dependency_sync();
     extern __shared__ u64 smem64[];
     u64* cand = smem64;
     u64* keep = cand + CAND_CAP;
@@ -487,6 +488,7 @@ __global__ void __launch_bounds__(THREADS, 2) compress_kernel(CompressArgs a) {
 // read back from q_idx, the exact normaliser from dsum.
 template <typename T>
 __global__ void __launch_bounds__(THREADS) compress_precise_kernel(CompressArgs a) {
+    grid_dependency_sync();
     extern __shared__ u64 smem64[];
     u64* keep = smem64;
     __shared__ CompressShared sh;

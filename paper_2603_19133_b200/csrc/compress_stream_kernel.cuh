@@ -309,10 +309,6 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
             mbar_init(&empty[s], WARPS);
         }
         mbar_init_fence();
-        if (blockIdx.x == 0) {
-            *a.queue_count_next = 0;
-            *a.redo_count_next = 0;
-        }
         cs.thr_key = 0u;
         cs.thr0_key = 0xffffffffu;
         cs.top_key = 0u;
@@ -322,6 +318,11 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
         cs.m = 0;
     }
     for (int i = tid; i < CS_HIST_WORDS; i += STREAM_THREADS) hist[i] = 0u;
+    grid_dependency_sync();
+    if (tid == 0 && blockIdx.x == 0) {
+        *a.queue_count_next = 0;
+        *a.redo_count_next = 0;
+    }
     __syncthreads();
 
     if (warp == WARPS) {
@@ -649,6 +650,7 @@ __global__ void __launch_bounds__(THREADS) compress_finish_kernel(CompressArgs a
     int k_eff = a.top_k > 0 ? a.top_k : a.k_max;
     if (k_eff > a.k_max) k_eff = a.k_max;
     if (k_eff > a.V) k_eff = a.V;
+    grid_dependency_sync();
     const u64* src = a.surv_keys + (long long)row * cs_survivor_cap(a.k_max);
     // the first 512 scratch slots exist for every k_max: requested before the row's count is known
     const u64 first0 = src[tid], first1 = src[tid + THREADS];

@@ -14,6 +14,7 @@ namespace picospec {
 // (one sparse row per sequence); u_resample [B] = one uniform per sequence; token [B]; mass [B].
 template <typename T, bool PRECISE>
 __global__ void __launch_bounds__(THREADS) edge_finish_kernel(VerifyArgs a) {
+    grid_dependency_sync();
     __shared__ double warp_tot[WARPS];
     __shared__ double sZ, sZraw;
     __shared__ float smx;

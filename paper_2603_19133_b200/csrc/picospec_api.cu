@@ -125,10 +125,28 @@ cudaError_t ensure_kernel_attrs(int device) {
     return e;
 }
 
+// Launch with programmatic stream serialization: the kernel's CTAs may be scheduled while the
+// kernel before it in the stream drains (every kernel starts with grid_dependency_sync()).
+// Launch errors are picked up by the callers through cudaGetLastError().
+template <typename... P, typename... A>
+void launch_chained(void (*kern)(P...), int grid, int block, size_t smem, cudaStream_t s, A&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    (void)cudaLaunchKernelEx(&cfg, kern, static_cast<P>(args)...);
+}
+
 template <typename T, bool ALIGNED>
 void launch_compress_direct(const CompressArgs& a, int grid, bool stats, cudaStream_t s) {
-    if (stats) compress_kernel<T, ALIGNED, true><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
-    else compress_kernel<T, ALIGNED, false><<<grid, THREADS, COMPRESS_SMEM, s>>>(a);
+    if (stats) launch_chained(compress_kernel<T, ALIGNED, true>, grid, THREADS, COMPRESS_SMEM, s, a);
+    else launch_chained(compress_kernel<T, ALIGNED, false>, grid, THREADS, COMPRESS_SMEM, s, a);
 }
 
 template <typename T>
@@ -156,7 +174,7 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
         const int g = rows < ctx->num_sms * per_sm ? rows : ctx->num_sms * per_sm;
         {
             ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_STREAM, 1, s);
-            kern<<<g, STREAM_THREADS, smem, s>>>(a, tiles_per_row);
+            launch_chained(kern, g, STREAM_THREADS, smem, s, a, tiles_per_row);
         }
         cudaError_t e0 = cudaGetLastError();
         if (e0 != cudaSuccess) return e0;
@@ -165,8 +183,8 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
             while (n2 < cs_survivor_cap(a.k_max)) n2 <<= 1;
             ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_FINISH, 2, s);
             // two exchange buffers of the sort network (the sorted keys end up in the first)
-            if (stats) compress_finish_kernel<T, true><<<rows, THREADS, (size_t)n2 * 16, s>>>(a, n2);
-            else compress_finish_kernel<T, false><<<rows, THREADS, (size_t)n2 * 16, s>>>(a, n2);
+            if (stats) launch_chained(compress_finish_kernel<T, true>, rows, THREADS, (size_t)n2 * 16, s, a, n2);
+            else launch_chained(compress_finish_kernel<T, false>, rows, THREADS, (size_t)n2 * 16, s, a, n2);
         }
         e0 = cudaGetLastError();
         if (e0 != cudaSuccess) return e0;
@@ -189,9 +207,9 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
     p.seq_rows = a.G; p.expand = 1; p.pos = nullptr; p.temperature = a.temperature;
     p.queue = a.queue; p.queue_count = a.queue_count; p.row_max = a.row_max; p.dsum = a.dsum;
     p.need_rows = nullptr;
-    precise_chunk_sums_kernel<T><<<ctx->num_sms * 6, THREADS, 0, s>>>(p);
+    launch_chained(precise_chunk_sums_kernel<T>, ctx->num_sms * 6, THREADS, 0, s, p);
     const int g2 = rows < ctx->num_sms ? rows : ctx->num_sms;
-    compress_precise_kernel<T><<<g2, THREADS, MAX_K * 8, s>>>(a);
+    launch_chained(compress_precise_kernel<T>, g2, THREADS, MAX_K * 8, s, a);
     return cudaGetLastError();
 }
 
@@ -211,19 +229,19 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
         const int gcap = ctx->num_sms * StreamCfg<T>::CTAS_PER_SM;
         const int g = (int)(tiles < gcap ? tiles : gcap);
         ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_STREAM, 1, s);
-        chunk_stats_bulk_kernel<T><<<g, STREAM_THREADS, TileGeom<T>::SMEM_BYTES, s>>>(a, tiles_per_row, tiles);
+        launch_chained(chunk_stats_bulk_kernel<T>, g, STREAM_THREADS, TileGeom<T>::SMEM_BYTES, s, a, tiles_per_row, tiles);
     } else {
         ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_STREAM, 1, s);
-        if (aligned) chunk_stats_kernel<T, true><<<grid, THREADS, 0, s>>>(a);
-        else chunk_stats_kernel<T, false><<<grid, THREADS, 0, s>>>(a);
+        if (aligned) launch_chained(chunk_stats_kernel<T, true>, grid, THREADS, 0, s, a);
+        else launch_chained(chunk_stats_kernel<T, false>, grid, THREADS, 0, s, a);
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const size_t dyn = (size_t)a.nch * sizeof(double);
     {
         ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_FINISH, 2, s);
-        if (edge) edge_finish_kernel<T, false><<<a.B, THREADS, 0, s>>>(a);
-        else verify_finish_kernel<T, false><<<a.B, THREADS, dyn, s>>>(a);
+        if (edge) launch_chained(edge_finish_kernel<T, false>, a.B, THREADS, 0, s, a);
+        else launch_chained(verify_finish_kernel<T, false>, a.B, THREADS, dyn, s, a);
     }
     ProfScope ps3(ctx, PICOSPEC_PROF_VERIFY_PRECISE, 2, s);
     PreciseArgs p;
@@ -235,10 +253,10 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
         p.r0 = a.r0; p.r1 = a.r1; p.gamma = a.gamma;
     }
     p.row_max = a.row_max; p.dsum = a.dsum;
-    precise_chunk_sums_kernel<T><<<ctx->num_sms * 6, THREADS, 0, s>>>(p);
+    launch_chained(precise_chunk_sums_kernel<T>, ctx->num_sms * 6, THREADS, 0, s, p);
     const int g2 = a.B < ctx->num_sms ? a.B : ctx->num_sms;
-    if (edge) edge_finish_kernel<T, true><<<g2, THREADS, 0, s>>>(a);
-    else verify_finish_kernel<T, true><<<g2, THREADS, dyn, s>>>(a);
+    if (edge) launch_chained(edge_finish_kernel<T, true>, g2, THREADS, 0, s, a);
+    else launch_chained(verify_finish_kernel<T, true>, g2, THREADS, dyn, s, a);
     return cudaGetLastError();
 }
 

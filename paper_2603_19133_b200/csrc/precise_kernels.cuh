@@ -27,6 +27,7 @@ struct PreciseArgs {
 
 template <typename T>
 __global__ void __launch_bounds__(THREADS) precise_chunk_sums_kernel(PreciseArgs a) {
+    grid_dependency_sync();
     const int nq = *a.queue_count;
     if (nq == 0) return;
     const int lane = threadIdx.x & 31;

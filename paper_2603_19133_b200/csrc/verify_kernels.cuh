@@ -105,6 +105,7 @@ template <typename T> __device__ __forceinline__ void chunk_stats_compute(const 
 
 template <typename T, bool ALIGNED>
 __global__ void __launch_bounds__(THREADS, 4) chunk_stats_kernel(VerifyArgs a) {
+    grid_dependency_sync();
     const int lane = threadIdx.x & 31;
     const long long gw = (long long)blockIdx.x * WARPS + (threadIdx.x >> 5);
     const long long nw = (long long)gridDim.x * WARPS;
@@ -169,10 +170,11 @@ __global__ void __launch_bounds__(STREAM_THREADS, StreamCfg<T>::CTAS_PER_SM) chu
             mbar_init(&empty[s], WARPS);
         }
         mbar_init_fence();
-        if (blockIdx.x == 0) {
-            *a.queue_count = 0;
-            if (a.borderline) *a.borderline = 0;
-        }
+    }
+    grid_dependency_sync();
+    if (tid == 0 && blockIdx.x == 0) {
+        *a.queue_count = 0;
+        if (a.borderline) *a.borderline = 0;
     }
     __syncthreads();
 
@@ -317,6 +319,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
     __shared__ FinishShared sh;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int G = a.G, G1 = a.G + 1;
+    grid_dependency_sync();
 
     const int nloop = PRECISE ? *a.queue_count : a.B;
     for (int slot = blockIdx.x; slot < nloop; slot += gridDim.x) {

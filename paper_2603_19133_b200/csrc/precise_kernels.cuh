@@ -1,5 +1,5 @@
 // Double-precision chunk sums for rows whose fp32 statistics were too close to a decision
-// threshold.  One warp per (queued row, chunk): sum of exp(l/T - max/T) over the chunk, exactly
+// threshold.  Four warps per (queued row, chunk): sum of exp(l/T - max/T) over the chunk, exactly
 // the terms of the definition.  The whole grid shares the work, so a handful of flagged rows
 // costs microseconds; with an empty queue every CTA returns at once.
 #pragma once
@@ -30,42 +30,57 @@ __global__ void __launch_bounds__(THREADS) precise_chunk_sums_kernel(PreciseArgs
     grid_dependency_sync();
     const int nq = *a.queue_count;
     if (nq == 0) return;
-    const int lane = threadIdx.x & 31;
-    const long long gw = (long long)blockIdx.x * WARPS + (threadIdx.x >> 5);
-    const long long nw = (long long)gridDim.x * WARPS;
+    // A CTA takes two chunks at a time, four warps per chunk (a quarter of the chunk each, so that a
+    // handful of rows still spreads over the whole GPU); the four partial sums of a chunk are added in
+    // a fixed order.
+    __shared__ double part[WARPS];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int sub = warp >> 2, quarter = warp & 3;
     const long long total = (long long)nq * a.expand * a.nch;
-    for (long long item = gw; item < total; item += nw) {
-        const int c = (int)(item % a.nch);
-        const long long t = item / a.nch;
-        const int ri = (int)(t % a.expand);
-        const int e = a.queue[(int)(t / a.expand)];
-        if (a.need_rows && !a.pos && ri < 64 && !((a.need_rows[e] >> ri) & 1ull)) continue;
-        if (!a.pos && (ri < a.r0 || ri >= a.r1 || (a.gamma && ri > a.gamma[e]))) continue;
-        const int src_row = a.pos ? e * a.seq_rows + a.pos[e] : e * a.expand + ri;
-        const int b = src_row / a.seq_rows;
-        const T* row = reinterpret_cast<const T*>(a.logits) + (long long)src_row * a.row_stride;
-        // x = l * (1/T) instead of l / T: one rounding of 2^-53 more per term, far below every
-        // threshold this pass decides; four independent sums keep the exp pipeline busy
-        const double rT = 1.0 / (double)a.temperature[b];
-        const double m = (double)a.row_max[src_row] * rT;
-        const int v0 = c * CHUNK;
-        double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-#pragma unroll 2
-        for (int k = lane; k < CHUNK; k += 128) {
-            const int v = v0 + k;
-            float l0 = -CUDART_INF_F, l1 = -CUDART_INF_F, l2 = -CUDART_INF_F, l3 = -CUDART_INF_F;
-            if (v < a.V) l0 = load_logit(row, v);
-            if (v + 32 < a.V) l1 = load_logit(row, v + 32);
-            if (v + 64 < a.V) l2 = load_logit(row, v + 64);
-            if (v + 96 < a.V) l3 = load_logit(row, v + 96);
-            s0 += exp((double)l0 * rT - m);
-            s1 += exp((double)l1 * rT - m);
-            s2 += exp((double)l2 * rT - m);
-            s3 += exp((double)l3 * rT - m);
+    const long long pairs = (total + 1) / 2;
+    for (long long pi = blockIdx.x; pi < pairs; pi += gridDim.x) {
+        const long long item = 2 * pi + sub;
+        bool work = item < total;
+        int c = 0, src_row = 0;
+        if (work) {
+            c = (int)(item % a.nch);
+            const long long t = item / a.nch;
+            const int ri = (int)(t % a.expand);
+            const int e = a.queue[(int)(t / a.expand)];
+            if (a.need_rows && !a.pos && ri < 64 && !((a.need_rows[e] >> ri) & 1ull)) work = false;
+            if (!a.pos && (ri < a.r0 || ri >= a.r1 || (a.gamma && ri > a.gamma[e]))) work = false;
+            src_row = a.pos ? e * a.seq_rows + a.pos[e] : e * a.expand + ri;
         }
-        double s = (s0 + s1) + (s2 + s3);
-        s = warp_sum(s);
-        if (lane == 0) a.dsum[(long long)src_row * a.nch + c] = s;
+        double s = 0.0;
+        if (work) {
+            const int b = src_row / a.seq_rows;
+            const T* row = reinterpret_cast<const T*>(a.logits) + (long long)src_row * a.row_stride;
+            // x = l * (1/T) instead of l / T: one rounding of 2^-53 more per term, far below every
+            // threshold this pass decides; four independent sums keep the exp pipeline busy
+            const double rT = 1.0 / (double)a.temperature[b];
+            const double m = (double)a.row_max[src_row] * rT;
+            const int v0 = c * CHUNK + quarter * (CHUNK / 4);
+            double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+#pragma unroll
+            for (int k = lane; k < CHUNK / 4; k += 128) {
+                const int v = v0 + k;
+                float l0 = -CUDART_INF_F, l1 = -CUDART_INF_F, l2 = -CUDART_INF_F, l3 = -CUDART_INF_F;
+                if (v < a.V) l0 = load_logit(row, v);
+                if (v + 32 < a.V) l1 = load_logit(row, v + 32);
+                if (v + 64 < a.V) l2 = load_logit(row, v + 64);
+                if (v + 96 < a.V) l3 = load_logit(row, v + 96);
+                s0 += exp((double)l0 * rT - m);
+                s1 += exp((double)l1 * rT - m);
+                s2 += exp((double)l2 * rT - m);
+                s3 += exp((double)l3 * rT - m);
+            }
+            s = warp_sum((s0 + s1) + (s2 + s3));
+        }
+        if (lane == 0) part[warp] = s;
+        __syncthreads();
+        if (work && quarter == 0 && lane == 0)
+            a.dsum[(long long)src_row * a.nch + c] = (part[warp] + part[warp + 1]) + (part[warp + 2] + part[warp + 3]);
+        __syncthreads();
     }
 }
 

@@ -88,6 +88,11 @@ PICOSPEC_API int picospec_last_cuda_error(const picospec_ctx* ctx);
 #define PICOSPEC_PROF_KINDS 7
 PICOSPEC_API int picospec_profile_enable(picospec_ctx* ctx, int level);
 
+/* Bracket only every `every`-th launch of each kind (default 1 = every launch).  An event between
+ * two kernels keeps the second from being scheduled while the first drains, so a benchmark that
+ * times whole steps samples the per-kernel brackets sparsely.  every >= 1. */
+PICOSPEC_API int picospec_profile_period(picospec_ctx* ctx, int every);
+
 /* Synchronise `cuda_stream`, then return the summed device time (ms, HOST pointer) and the number
  * of launches (HOST pointer) recorded for `kind` since the last read (at most the last 128
  * launches are kept), and reset that counter. */

@@ -43,6 +43,8 @@ def lib() -> ctypes.CDLL:
         L.picospec_residual_sample.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp,
                                                c_int, vp, vp, vp, vp]
         L.picospec_profile_enable.argtypes = [vp, c_int]
+        L.picospec_profile_period.argtypes = [vp, c_int]
+        L.picospec_profile_period.restype = c_int
         L.picospec_profile_read.argtypes = [vp, c_int, ctypes.POINTER(c_f), ctypes.POINTER(c_int), vp]
         L.picospec_target_topk.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, c_int, vp, vp, vp, vp]
         L.picospec_target_topk.restype = c_int
@@ -178,8 +180,10 @@ class Context:
         _check(lib().picospec_counters(self._h, out, int(clear), _stream()), "picospec_counters")
         return int(out[0]), int(out[1])
 
-    def profile_enable(self, level: int):
-        """0 = off, 1 = time the two streaming kernels, 2 = time every kernel group."""
+    def profile_enable(self, level: int, every: int = 1):
+        """0 = off, 1 = time the two streaming kernels, 2 = time every kernel group; only every
+        `every`-th launch of a kind is bracketed (picospec_profile_period)."""
+        _check(lib().picospec_profile_period(self._h, int(every)), "picospec_profile_period")
         _check(lib().picospec_profile_enable(self._h, int(level)), "picospec_profile_enable")
 
     def profile_read(self, kind: int) -> Tuple[float, int]:
@@ -271,13 +275,19 @@ class Context:
         return out
 
     # -- the paper's own data flow (Sec. 3.3) ---------------------------------------------------
-    def target_topk(self, target_logits: torch.Tensor, temperature: torch.Tensor, pos: torch.Tensor, k: int):
-        """picospec_target_topk.  Returns (p_idx [B,k] i32, p_prob [B,k] f32 unnormalised, p_count [B] i32)."""
+    def target_topk(self, target_logits: torch.Tensor, temperature: torch.Tensor, pos: torch.Tensor, k: int,
+                    out=None):
+        """picospec_target_topk.  Returns (p_idx [B,k] i32, p_prob [B,k] f32 unnormalised, p_count [B] i32);
+        `out` = such a triple to write into."""
         p, dt, B, R, V, pitch = _logits(target_logits)
         dev = target_logits.device
-        p_idx = torch.empty((B, k), dtype=torch.int32, device=dev)
-        p_prob = torch.empty((B, k), dtype=torch.float32, device=dev)
-        p_count = torch.empty((B,), dtype=torch.int32, device=dev)
+        if out is not None:
+            p_idx, p_prob, p_count = out
+            _ptr(p_idx, torch.int32, (B, k)), _ptr(p_prob, torch.float32, (B, k)), _ptr(p_count, torch.int32, (B,))
+        else:
+            p_idx = torch.empty((B, k), dtype=torch.int32, device=dev)
+            p_prob = torch.empty((B, k), dtype=torch.float32, device=dev)
+            p_count = torch.empty((B,), dtype=torch.int32, device=dev)
         _check(lib().picospec_target_topk(
             self._h, p, dt, B, R, V, pitch, _ptr(temperature, torch.float32, (B,)), _ptr(pos, torch.int32, (B,)),
             int(k), _ptr(p_idx), _ptr(p_prob), _ptr(p_count), _stream()), "picospec_target_topk")
@@ -285,13 +295,18 @@ class Context:
 
     def edge_resample(self, draft_logits: torch.Tensor, temperature: torch.Tensor, pos: torch.Tensor,
                       p_idx: torch.Tensor, p_prob: torch.Tensor, p_count: torch.Tensor, u: torch.Tensor,
-                      want_mass: bool = True):
-        """picospec_edge_resample.  Returns (token [B] i32, mass [B] f32 or None)."""
+                      want_mass: bool = True, out=None):
+        """picospec_edge_resample.  Returns (token [B] i32, mass [B] f32 or None); `out` = such a pair
+        to write into."""
         p, dt, B, R, V, pitch = _logits(draft_logits)
         k = p_idx.shape[-1]
         dev = draft_logits.device
-        token = torch.empty((B,), dtype=torch.int32, device=dev)
-        mass = torch.empty((B,), dtype=torch.float32, device=dev) if want_mass else None
+        if out is not None:
+            token, mass = out
+            _ptr(token, torch.int32, (B,)), _ptr(mass, torch.float32, (B,))
+        else:
+            token = torch.empty((B,), dtype=torch.int32, device=dev)
+            mass = torch.empty((B,), dtype=torch.float32, device=dev) if want_mass else None
         _check(lib().picospec_edge_resample(
             self._h, p, dt, B, R, V, pitch, _ptr(temperature, torch.float32, (B,)), _ptr(pos, torch.int32, (B,)),
             _ptr(p_idx, torch.int32, (B, k)), _ptr(p_prob, torch.float32, (B, k)), _ptr(p_count, torch.int32, (B,)),

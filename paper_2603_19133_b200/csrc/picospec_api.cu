@@ -27,6 +27,8 @@ struct picospec_ctx {
     int prof_level;
     cudaEvent_t prof_ev[PICOSPEC_PROF_KINDS][PROF_RING][2];
     long long prof_count[PICOSPEC_PROF_KINDS];
+    int prof_every;                                   // bracket every prof_every-th launch of a kind
+    long long prof_seq[PICOSPEC_PROF_KINDS];
     // workspace
     float2* stats;
     double* dsum;
@@ -65,6 +67,7 @@ struct ProfScope {
     bool on;
     ProfScope(picospec_ctx* c, int k, int min_level, cudaStream_t st) : ctx(c), kind(k), s(st) {
         on = c->prof_level >= min_level;
+        if (on) on = (c->prof_seq[k]++ % c->prof_every) == 0;
         if (on) cudaEventRecord(c->prof_ev[k][c->prof_count[k] % PROF_RING][0], s);
     }
     ~ProfScope() {
@@ -388,8 +391,16 @@ int picospec_profile_enable(picospec_ctx* ctx, int level) {
                     ctx->prof_ev[k][i][j] = nullptr;
                 }
     }
-    for (int k = 0; k < PICOSPEC_PROF_KINDS; ++k) ctx->prof_count[k] = 0;
+    for (int k = 0; k < PICOSPEC_PROF_KINDS; ++k) ctx->prof_count[k] = ctx->prof_seq[k] = 0;
     ctx->prof_level = level;
+    if (ctx->prof_every < 1) ctx->prof_every = 1;
+    return PICOSPEC_OK;
+}
+
+int picospec_profile_period(picospec_ctx* ctx, int every) {
+    if (!ctx || every < 1) return PICOSPEC_EINVAL;
+    ctx->prof_every = every;
+    for (int k = 0; k < PICOSPEC_PROF_KINDS; ++k) ctx->prof_seq[k] = 0;
     return PICOSPEC_OK;
 }
 

@@ -427,6 +427,38 @@ def _custom_inputs(dl, tl, seed):
             "u_resample": torch.rand((B, 2), generator=g, device="cuda")}
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("above,ties,top_p", [
+    (200, 100, 1.0),      # 300 survivors for k = 256: the 56 lowest indices of the tie group are kept
+    (200, 100, 0.97),     # the same with a nucleus cut
+    (100, 400, 1.0),      # a tie group too large to rank pair by pair: the full 512-key network
+    (255, 256, 1.0),      # one slot left for a group of 256
+    (0, 300, 1.0),        # nothing above the group
+    (256, 200, 1.0),      # the group starts right after the k-th: none of it is kept
+])
+def test_finish_trims_the_boundary_group_by_index(ps, above, ties, top_p, dtype):
+    # Rows with a chosen number of distinct values above a group of equal values that straddles the
+    # k-th place: the finish kernel must keep the group's members with the lowest vocabulary indices.
+    V, B, G, K = 16384, 3, 2, 256
+    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    g = torch.Generator(device="cuda").manual_seed(above * 1000 + ties)
+    dl = torch.empty((B, G, V), dtype=torch.float32, device="cuda")
+    for b in range(B):
+        for i in range(G):
+            row = (torch.rand(V, generator=g, device="cuda") * 4.0 - 6.0)          # filler in [-6, -2)
+            perm = torch.randperm(V, generator=g, device="cuda")
+            row[perm[:above]] = 8.0 + 0.0625 * torch.arange(above, device="cuda")   # distinct, exact in bf16
+            row[perm[above:above + ties]] = 4.0                                    # the tie group
+            dl[b, i] = row
+    dl = dl.to(td)
+    tl = (torch.randn((B, G + 1, V), generator=g, device="cuda") * 2.0).to(td)
+    w = gen.Workload("t", V=V, B=B, G=G, dtype=dtype, s=0, sigma_d=0, corr=0, sigma_t=0, T=0.9,
+                     top_k=(K if top_p >= 1.0 else 0), top_p=top_p, k_max=K)
+    r = run_both(ps, w, _custom_inputs(dl, tl, 13))
+    assert r["status"] == 0
+    assert r["redo_rows"] == 0          # every row stays in the staged kernels (at most 512 survivors)
+
+
 @pytest.mark.parametrize("top_p", [1.0, 0.9])
 def test_staged_rows_that_overflow_the_filter_are_redone(ps, top_p):
     # rows built to defeat a running threshold: all equal, heavy ties, ascending (every new value is

@@ -235,13 +235,6 @@ template <typename T> __device__ __forceinline__ float lane_exp_sum(const ChunkR
     return (a0 + a1) + (a2 + a3);
 }
 
-// Double-precision weight of one logit: exp(l * (1/T) - row_max * (1/T)) (the definition's
-// exp(l/T - max/T) with the division replaced by one multiplication: 2^-53 relative per term).
-// The fp32 streaming pass sums 2^(l*c32 - off) with c32 = fp32(log2 e / T) and
-// off = fp32(row_max * c32); stream_sum_scale() is the exact factor 2^(off - row_max*c32) that
-// brings such a sum onto the scale of these weights (what remains is the bounded error GUARD_Z).
-// The fast path and the double-precision re-evaluation use the same weights; they differ in
-// where the normaliser comes from.
 // Every kernel is launched with programmatic stream serialization: its CTAs may be scheduled while
 // the kernel before it in the stream is still draining.  Each thread waits here, before its first
 // access to global memory, until that kernel has completed and its writes are visible; then the
@@ -252,6 +245,13 @@ __device__ __forceinline__ void grid_dependency_sync() {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Double-precision weight of one logit: exp(l * (1/T) - row_max * (1/T)) (the definition's
+// exp(l/T - max/T) with the division replaced by one multiplication: 2^-53 relative per term).
+// The fp32 streaming pass sums 2^(l*c32 - off) with c32 = fp32(log2 e / T) and
+// off = fp32(row_max * c32); stream_sum_scale() is the exact factor 2^(off - row_max*c32) that
+// brings such a sum onto the scale of these weights (what remains is the bounded error GUARD_Z).
+// The fast path and the double-precision re-evaluation use the same weights; they differ in
+// where the normaliser comes from.
 template <bool PRECISE> struct Weight {
     double t, m;
     __device__ __forceinline__ void init(float T, float row_max) {

@@ -28,11 +28,13 @@
 //     kernel through a redo list;
 //   - with top-p the same pass accumulates the softmax normaliser relative to the first tile's
 //     maximum (a row whose later logits overflow that reference also goes to the redo list).
-// At the end of a row the candidates at or above thr (at least k, normally k plus a few dozen) go
-// to a per-row scratch area in global memory.
+// At the end of a row the candidates at or above thr (at least k; for 16-bit logits the k best plus
+// the ties of the k-th, for 32-bit logits plus what shares its 16-bit code) go to a per-row scratch
+// area in global memory, with the bound itself.
 //
-// compress_finish_kernel (one CTA per row) sorts them and calls finish_row (top-p cut,
-// renormalisation, emission, draft draw).
+// compress_finish_kernel (one CTA per row) trims them to k where that is cheap, sorts them with a
+// bitonic network held in registers and calls finish_row (top-p cut, renormalisation, emission,
+// draft draw).
 #pragma once
 #include "compress_kernels.cuh"
 #include "stream_pipeline.cuh"

@@ -681,3 +681,89 @@ def test_range_call_skips_decided_sequences_and_flags_bad_input():
     # an undecided sequence whose bonus row lies before the range is a caller error
     out = oracle.verify_range(lt, T, np.full(B, 1, np.int32), 3, 5, None, tok, qi, qp, qc, ua, ur)
     assert np.all(out["accept_len"] == -1)
+
+
+# ---------------------------------------------------------------------------------------------
+# Wire format of the sparse rows (Sec. 3.3) and the throughput model (Sec. 3.4, Eqs. 5-10)
+# ---------------------------------------------------------------------------------------------
+
+def _wire_case(seed, R=7, K=10):
+    rng = _rng(seed)
+    l = rng.normal(size=(R, 1, 500)).astype(np.float32) * 3
+    qi, qp, qc, _ = oracle.compress(l, np.ones(R, np.float32), top_k=0, top_p=0.8, k_max=K)
+    return qi.reshape(R, K), qp.reshape(R, K), qc.reshape(R)
+
+
+def test_wire_message_sizes_match_the_printed_payload_figures():
+    from oracle import wire
+    vals = {}
+    for ln in open(os.path.join(GOLDEN, "payload_sizes.txt")):
+        ln = ln.split("#")[0].split()
+        if ln:
+            vals[ln[0]] = ln[1:]
+    K = int(vals["topk_example_k"][0])
+    qi = np.arange(K, dtype=np.int32).reshape(1, K)
+    qp = np.full((1, K), 0.1, np.float32)
+    qc = np.array([K], np.int32)
+    pairs = int(vals["topk_row_bytes"][0])
+    m32 = wire.pack(qi, qp, qc, wire.F32)
+    # the (id, prob) pairs are the printed 80 bytes; the whole message adds a 16-byte header and the count
+    assert m32.size == 16 + 4 + pairs
+    m16 = wire.pack(qi, qp, qc, wire.F16)
+    assert m16.size == 16 + 4 + 4 * K + 2 * K < int(vals["topk_row_bytes"][2])      # under 100 bytes on the wire
+    V = int(vals["vocab_llama31"][0])
+    assert V * 4 / m16.size > 1000                                                   # "over three orders of magnitude"
+
+
+@pytest.mark.parametrize("ptype", [0, 1])
+def test_wire_round_trip_and_layout(ptype):
+    from oracle import wire
+    qi, qp, qc = _wire_case(41)
+    qc[3] = -1                                   # an invalid row travels as such
+    qi[3], qp[3] = -1, 0
+    m = wire.pack(qi, qp, qc, ptype)
+    R, K = qi.shape
+    N = int(np.maximum(qc, 0).sum())
+    # layout, read back with plain struct arithmetic
+    import struct
+    magic, rows, k, pt, n = struct.unpack_from("<IIHHI", m.tobytes(), 0)
+    assert (magic, rows, k, pt, n) == (0x31505350, R, K, ptype, N)
+    counts = np.frombuffer(m.tobytes(), "<i2", R, 16)
+    assert np.array_equal(counts, qc)
+    ids = np.frombuffer(m.tobytes(), "<i4", N, 16 + (2 * R + 3) // 4 * 4)
+    assert np.array_equal(ids, np.concatenate([qi[r, :max(qc[r], 0)] for r in range(R)]))
+    ui, up, uc = wire.unpack(m, R, K)
+    assert np.array_equal(ui, qi) and np.array_equal(uc, qc)
+    if ptype == 0:
+        assert np.array_equal(up, qp)
+    else:
+        assert np.array_equal(up, qp.astype(np.float16).astype(np.float32))
+        np.testing.assert_allclose(up, qp, rtol=2 ** -11)
+    # a message for another shape, a wrong magic and a truncated message are refused as a whole
+    for bad in (wire.unpack(m, R + 1, K), wire.unpack(m, R, K + 1), wire.unpack(m[:-4], R, K),
+                wire.unpack(np.concatenate([np.zeros(4, np.uint8), m[4:]]), R, K)):
+        assert np.all(bad[2] == -1) and np.all(bad[0] == -1) and np.all(bad[1] == 0)
+
+
+def test_throughput_model_closed_forms_and_limits():
+    from oracle import wire
+    # Eq. (5) closed form, its limits, and the golden values
+    for a in (0.0, 0.3, 0.75, 0.9, 0.999):
+        for g in (1, 4, 8):
+            closed = (1 - a ** g) / (1 - a)
+            assert abs(wire.expected_length(a, g) - closed) < 1e-12 * g
+    assert abs(wire.expected_length(1.0 - 1e-12, 6) - 6) < 1e-9 and wire.expected_length(0.0, 6) == 1.0
+    rows = [ln.split() for ln in open(os.path.join(GOLDEN, "expected_length.txt")) if ln[0] not in "#\n"]
+    for alpha_s, gamma_s, el_s in rows:
+        assert abs(wire.expected_length(float(alpha_s), int(gamma_s)) - float(el_s)) < 5e-4
+    td, tr, tv = 40.0, 25.0, 10.0
+    # Eq. (7) written out; Eq. (9) at alpha = 1 and alpha = 0
+    assert abs(wire.throughput_sync(0.8, 5, td, tr, tv) - (1 - 0.8 ** 5) / (0.2 * (td + tr + tv))) < 1e-12
+    assert wire.expected_time_async(1.0, 5, td, tr, tv) == max(td, tr + tv)
+    assert wire.expected_time_async(0.0, 5, td, tr, tv) == td + tr + tv
+    # Eq. (10): compute-bound, alpha -> 1; and the lower bound S -> 1 as alpha -> 0
+    assert abs(wire.speedup(1.0 - 1e-9, 5, td, tr, tv) - (1 + (tr + tv) / td)) < 1e-6
+    assert abs(wire.speedup(0.0, 5, td, tr, tv) - 1.0) < 1e-12
+    # S is never below 1 and grows with alpha
+    s = [wire.speedup(a, 5, td, tr, tv) for a in np.linspace(0, 0.999, 50)]
+    assert min(s) >= 1.0 and all(b >= a - 1e-12 for a, b in zip(s, s[1:]))

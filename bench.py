@@ -368,6 +368,42 @@ def bench_paper_direction(ps, w, device, k, iters):
     return out
 
 
+def bench_wire(ps, w, device, iters):
+    """The wire codec of the sparse rows (Sec. 3.3) on the rows picospec_compress leaves for this
+    shape, timed per call with CUDA events, and the size of the paper's K = 10 example message."""
+    ctx = ps.Context(w.B, w.G, w.V, w.k_max)
+    inp = gen.make_inputs(w, seed=7100, device=device)
+    qi, qp, qc, _ = ctx.compress(inp["draft_logits"], inp["temperature"], w.top_k, w.top_p, w.k_max, inp["u_draft"])
+    R = qc.numel()
+    out = {"rows": R, "k_max": w.k_max, "dense_bytes": R * w.k_max * 8}
+    for fp16 in (False, True):
+        buf, nbytes = ctx.wire_pack(qi, qp, qc, fp16=fp16)
+        n = int(nbytes.item())
+        dense = ctx.wire_unpack(buf, n, R, w.k_max)
+
+        def timed(fn):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(iters):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) * 1e3 / iters
+
+        tag = "fp16" if fp16 else "fp32"
+        out[f"message_bytes_{tag}"] = n
+        out[f"pack_us_{tag}"] = timed(lambda: ctx.wire_pack(qi, qp, qc, fp16=fp16, buf=buf, bytes_out=nbytes))
+        out[f"unpack_us_{tag}"] = timed(lambda: ctx.wire_unpack(buf, n, R, w.k_max, out=dense))
+    out["k10_message_bytes_fp32"] = ps.wire_bytes(1, 10, 0)
+    out["k10_message_bytes_fp16"] = ps.wire_bytes(1, 10, 1)
+    out["status"] = ctx.status(clear=True)[0]
+    ctx.close()
+    return out
+
+
 def run_ours(args):
     rank, local_rank, world = _dist_env()
     if not torch.cuda.is_available():
@@ -398,8 +434,10 @@ def run_ours(args):
                             "input_sets_rotated": r["nsets"], "slow_rows_per_step": r["slow_rows_per_step"]}
 
     paper_direction = None
+    wire_codec = None
     if args.all_configs and world == 1:
         paper_direction = bench_paper_direction(ps, w, device, k=10, iters=min(args.steps, 200))
+        wire_codec = bench_wire(ps, w, device, iters=min(args.steps, 200))
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -452,6 +490,7 @@ def run_ours(args):
             "device_status": main["status"],
             "other_configs": others,
             "paper_direction": paper_direction,
+            "wire_codec": wire_codec,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

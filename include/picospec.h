@@ -165,6 +165,37 @@ PICOSPEC_API int picospec_verify(picospec_ctx* ctx, const void* target_logits, p
                     float* p_draft, float* resid_mass, int* borderline_count, const float* u_resample,
                     int* token, void* cuda_stream);
 
+/* Wire format of sparse rows (Sec. 3.3: the verifier sends the K "(id, prob)" pairs, under 100
+ * bytes for K = 10, laid out so that the receiver views the arrays in place).  One message, little
+ * endian, 4-byte aligned:
+ *     0   u32  magic 0x31505350 ("PSP1")
+ *     4   u32  R, the number of rows
+ *     8   u16  K, the capacity of a dense row
+ *     10  u16  probability type: 0 = fp32, 1 = fp16 (round to nearest even)
+ *     12  u32  N = sum over rows of max(count, 0)
+ *     16  i16  count[R]   (-1 = invalid row), zero-padded to a multiple of 4 bytes
+ *     ..  i32  id[N]      rows in order, entries in stored order
+ *     ..  prob[N]         fp32 or fp16; the message is zero-padded to a multiple of 4 bytes
+ * The id and prob arrays of the message are the receiver's views; picospec_wire_unpack scatters
+ * them back into dense [R, K] arrays (padding: id -1, prob 0) for the calls above.
+ *
+ * picospec_wire_bytes: size of a message (host arithmetic; -1 on bad arguments).
+ * picospec_wire_pack: q_idx, q_prob [rows, k], q_count [rows] (device) -> buf (device, 4-byte
+ *   aligned, capacity_bytes long).  *bytes_out (DEVICE pointer) = size of the message, or -1 if it
+ *   does not fit (then buf holds no message and status bit 4 is set).  A count outside [-1, k]
+ *   travels as -1 and sets status bit 4.
+ * picospec_wire_unpack: the reverse; a message whose magic, R, K, type, counts or length do not
+ *   match is refused as a whole: every row comes back invalid (count -1, id -1, prob 0) and status
+ *   bit 4 is set.
+ * rows <= max_batch * (max_gamma + 1) of the context, k <= PICOSPEC_MAX_K.
+ */
+PICOSPEC_API long long picospec_wire_bytes(int rows, long long entries, int prob_type);
+PICOSPEC_API int picospec_wire_pack(picospec_ctx* ctx, const int* q_idx, const float* q_prob, const int* q_count, int rows,
+                       int k, int prob_type, void* buf, long long capacity_bytes, long long* bytes_out,
+                       void* cuda_stream);
+PICOSPEC_API int picospec_wire_unpack(picospec_ctx* ctx, const void* buf, long long bytes, int rows, int k, int* q_idx,
+                         float* q_prob, int* q_count, void* cuda_stream);
+
 /* Half 2a on rows as they arrive -- incremental verification (Sec. 3.2: the verifier works on a
  * prefix of the segment while the drafter is still producing the rest; Sec. 3.3: latency-aware
  * truncation makes the number of drafted tokens differ between sequences).

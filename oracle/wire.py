@@ -40,6 +40,7 @@ def pack(q_idx, q_prob, q_count, prob_type: int = F32) -> np.ndarray:
     q_idx = q_idx.reshape(-1, K)
     q_prob = q_prob.reshape(-1, K)
     R = q_idx.shape[0]
+    q_count = np.where((q_count > K) | (q_count < -1), -1, q_count).astype(np.int32)   # bad count: the row travels as invalid
     ids, probs = [], []
     for r in range(R):
         n = max(int(q_count[r]), 0)

@@ -54,6 +54,12 @@ def lib() -> ctypes.CDLL:
         L.picospec_verify_range.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, c_int, c_int, vp, vp,
                                             vp, vp, vp, c_int, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.picospec_verify_range.restype = c_int
+        L.picospec_wire_bytes.argtypes = [c_int, c_ll, c_int]
+        L.picospec_wire_bytes.restype = c_ll
+        L.picospec_wire_pack.argtypes = [vp, vp, vp, vp, c_int, c_int, c_int, vp, c_ll, vp, vp]
+        L.picospec_wire_pack.restype = c_int
+        L.picospec_wire_unpack.argtypes = [vp, vp, c_ll, c_int, c_int, vp, vp, vp, vp]
+        L.picospec_wire_unpack.restype = c_int
         L.picospec_counters.argtypes = [vp, ctypes.POINTER(c_ll), c_int, vp]
         L.picospec_counters.restype = c_int
         L.picospec_verify_static.argtypes = [vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp, c_int,
@@ -139,6 +145,14 @@ def verify_static(target_logits: torch.Tensor, temperature: torch.Tensor, draft_
         _ptr(out.get("token"), torch.int32, (B,)), _ptr(out.get("device_status"), torch.int32, (1,)),
         _ptr(out.get("slow_rows"), torch.int64, (1,)), _stream()), "picospec_verify_static")
     return out
+
+
+def wire_bytes(rows: int, entries: int, prob_type: int = 0) -> int:
+    """picospec_wire_bytes: size of a message of `rows` rows holding `entries` (id, prob) pairs."""
+    n = lib().picospec_wire_bytes(int(rows), int(entries), int(prob_type))
+    if n < 0:
+        raise ValueError("picospec_wire_bytes: bad arguments")
+    return int(n)
 
 
 class Context:
@@ -312,6 +326,36 @@ class Context:
             _ptr(p_idx, torch.int32, (B, k)), _ptr(p_prob, torch.float32, (B, k)), _ptr(p_count, torch.int32, (B,)),
             int(k), _ptr(u, torch.float32, (B,)), _ptr(token), _ptr(mass), _stream()), "picospec_edge_resample")
         return token, mass
+
+    # -- wire format of the sparse rows (Sec. 3.3) ---------------------------------------------
+    def wire_pack(self, q_idx: torch.Tensor, q_prob: torch.Tensor, q_count: torch.Tensor, fp16: bool = False,
+                  buf: Optional[torch.Tensor] = None, bytes_out: Optional[torch.Tensor] = None):
+        """picospec_wire_pack.  q_idx / q_prob [..., K], q_count [...].  Returns (buf uint8, bytes_out
+        int64 [1] on the device: the message is buf[:bytes_out]).  Without `buf` one is allocated for the
+        largest message these shapes can give."""
+        K = q_idx.shape[-1]
+        R = q_count.numel()
+        ptype = 1 if fp16 else 0
+        if buf is None:
+            buf = torch.empty((wire_bytes(R, R * K, ptype),), dtype=torch.uint8, device=q_idx.device)
+        if bytes_out is None:
+            bytes_out = torch.empty((1,), dtype=torch.int64, device=q_idx.device)
+        _check(lib().picospec_wire_pack(
+            self._h, _ptr(q_idx, torch.int32), _ptr(q_prob, torch.float32), _ptr(q_count, torch.int32), R, int(K), ptype,
+            _ptr(buf, torch.uint8), int(buf.numel()), _ptr(bytes_out, torch.int64, (1,)), _stream()), "picospec_wire_pack")
+        return buf, bytes_out
+
+    def wire_unpack(self, buf: torch.Tensor, nbytes: int, rows: int, k: int, out=None):
+        """picospec_wire_unpack.  Returns dense (q_idx [rows,k] i32, q_prob [rows,k] f32, q_count [rows] i32)."""
+        dev = buf.device
+        if out is None:
+            out = (torch.empty((rows, k), dtype=torch.int32, device=dev),
+                   torch.empty((rows, k), dtype=torch.float32, device=dev),
+                   torch.empty((rows,), dtype=torch.int32, device=dev))
+        _check(lib().picospec_wire_unpack(
+            self._h, _ptr(buf, torch.uint8), int(nbytes), int(rows), int(k), _ptr(out[0], torch.int32, (rows, k)),
+            _ptr(out[1], torch.float32, (rows, k)), _ptr(out[2], torch.int32, (rows,)), _stream()), "picospec_wire_unpack")
+        return out
 
     # -- half 2b ---------------------------------------------------------------------
     def residual_sample(self, target_logits: torch.Tensor, temperature: torch.Tensor, pos: torch.Tensor,

@@ -12,6 +12,7 @@
 #include "compress_stream_kernel.cuh"
 #include "verify_kernels.cuh"
 #include "edge_kernels.cuh"
+#include "wire_kernels.cuh"
 
 using namespace picospec;
 
@@ -39,6 +40,8 @@ struct picospec_ctx {
     int* redo_rows; // rows the staged compress kernel hands to the direct kernel
     unsigned long long* surv_keys;  // staged compress: survivors per row
     CsRowMeta* surv_meta;
+    int* wire_off;                  // wire codec: first entry of each row, [rows + 1]
+    long long max_rows;
     unsigned* status;
     unsigned long long* slow_rows;
 };
@@ -321,6 +324,8 @@ int picospec_create(picospec_ctx** out, int device, int max_batch, int max_gamma
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->redo_rows, rows * sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_keys, rows * (size_t)cs_survivor_cap(max_k) * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_meta, rows * sizeof(CsRowMeta));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->wire_off, (rows + 1) * sizeof(int));
+    ctx->max_rows = (long long)rows;
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->status, sizeof(unsigned));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->slow_rows, 2 * sizeof(unsigned long long));   // [0] slow rows, [1] redo rows
     if (e == cudaSuccess) e = cudaMemset(ctx->counters, 0, 8 * sizeof(int));
@@ -352,6 +357,7 @@ int picospec_destroy(picospec_ctx* ctx) {
     cudaFree(ctx->redo_rows);
     cudaFree(ctx->surv_keys);
     cudaFree(ctx->surv_meta);
+    cudaFree(ctx->wire_off);
     cudaFree(ctx->status);
     cudaFree(ctx->slow_rows);
     free(ctx);
@@ -455,6 +461,55 @@ int picospec_counters(picospec_ctx* ctx, long long* out, int clear, void* cuda_s
     out[0] = (long long)v[0];
     out[1] = (long long)v[1];
     return PICOSPEC_OK;
+}
+
+long long picospec_wire_bytes(int rows, long long entries, int prob_type) {
+    if (rows < 0 || entries < 0 || (prob_type != 0 && prob_type != 1)) return -1;
+    return wire_bytes(rows, entries, prob_type);
+}
+
+static int wire_common(picospec_ctx* ctx, WireArgs& a, bool pack, void* cuda_stream) {
+    if (!ctx || !a.q_idx || !a.q_prob || !a.q_count || !a.buf) return PICOSPEC_EINVAL;
+    if (a.R < 0 || a.K <= 0 || a.K > PICOSPEC_MAX_K || a.capacity < 0) return PICOSPEC_EINVAL;
+    if (pack && (a.prob_type != 0 && a.prob_type != 1)) return PICOSPEC_EINVAL;
+    if (((uintptr_t)a.buf & 3u) != 0) return PICOSPEC_EINVAL;
+    if (a.R > ctx->max_rows) return PICOSPEC_ECAPACITY;
+    if (a.R == 0 && !pack) return PICOSPEC_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
+    a.offsets = ctx->wire_off;
+    a.status = ctx->status;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const int rows_grid = a.R > 0 ? (a.R + WARPS - 1) / WARPS : 1;
+    const int grid = rows_grid < ctx->num_sms * 8 ? rows_grid : ctx->num_sms * 8;
+    if (pack) {
+        launch_chained(wire_scan_kernel<true>, 1, THREADS, 0, s, a);
+        launch_chained(wire_move_kernel<true>, grid, THREADS, 0, s, a);
+    } else {
+        launch_chained(wire_scan_kernel<false>, 1, THREADS, 0, s, a);
+        launch_chained(wire_move_kernel<false>, grid, THREADS, 0, s, a);
+    }
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
+}
+
+int picospec_wire_pack(picospec_ctx* ctx, const int* q_idx, const float* q_prob, const int* q_count, int rows, int k,
+                       int prob_type, void* buf, long long capacity_bytes, long long* bytes_out, void* cuda_stream) {
+    if (!bytes_out) return PICOSPEC_EINVAL;
+    WireArgs a;
+    a.q_idx = const_cast<int*>(q_idx); a.q_prob = const_cast<float*>(q_prob); a.q_count = const_cast<int*>(q_count);
+    a.R = rows; a.K = k; a.prob_type = prob_type;
+    a.buf = (unsigned char*)buf; a.capacity = capacity_bytes; a.bytes_out = bytes_out;
+    return wire_common(ctx, a, true, cuda_stream);
+}
+
+int picospec_wire_unpack(picospec_ctx* ctx, const void* buf, long long bytes, int rows, int k, int* q_idx,
+                         float* q_prob, int* q_count, void* cuda_stream) {
+    WireArgs a;
+    a.q_idx = q_idx; a.q_prob = q_prob; a.q_count = q_count;
+    a.R = rows; a.K = k; a.prob_type = 0;
+    a.buf = (unsigned char*)const_cast<void*>(buf); a.capacity = bytes; a.bytes_out = nullptr;
+    return wire_common(ctx, a, false, cuda_stream);
 }
 
 int picospec_compress(picospec_ctx* ctx, const void* draft_logits, picospec_dtype dtype, int B, int G, int V,

@@ -139,3 +139,31 @@ def test_sequence_sharding_world_size_2_gloo(tmp_path):
     run = subprocess.run(cmd, capture_output=True, text=True, timeout=300)
     assert run.returncode == 0, run.stdout[-2000:] + run.stderr[-2000:]
     assert "SHARD_OK" in run.stdout
+
+
+def test_throughput_calculator_matches_the_term_by_term_oracle():
+    # the product's closed forms (Sec. 3.4, Eqs. 5-10) against the oracle's sums and case analysis
+    from paper_2603_19133_b200 import perf_model as pm
+    from oracle import wire
+    import itertools
+    for alpha, gamma in itertools.product((0.0, 0.2, 0.7, 0.95, 1.0), (1, 4, 6, 9)):
+        assert abs(pm.expected_length(alpha, gamma) - wire.expected_length(alpha, gamma)) < 1e-9
+        for td, tr, tv in ((40.0, 25.0, 10.0), (5.0, 50.0, 8.0), (30.0, 0.0, 30.0)):
+            assert abs(pm.throughput_sync(alpha, gamma, td, tr, tv) - wire.throughput_sync(alpha, gamma, td, tr, tv)) < 1e-12
+            assert abs(pm.expected_time_async(alpha, gamma, td, tr, tv) - wire.expected_time_async(alpha, gamma, td, tr, tv)) < 1e-9
+            assert abs(pm.speedup(alpha, gamma, td, tr, tv) - wire.speedup(alpha, gamma, td, tr, tv)) < 1e-9
+    assert abs(pm.speedup(1.0, 5, 40.0, 25.0, 10.0) - pm.speedup_limit(40.0, 25.0, 10.0)) < 1e-12
+    # payload sizes: the wire message of K = 10 pairs, against the oracle's packer and the C helper
+    import numpy as np
+    qi = np.arange(10, dtype=np.int32).reshape(1, 10)
+    qp = np.full((1, 10), 0.1, np.float32)
+    for fp16 in (False, True):
+        assert pm.downlink_bytes(10, fp16) == wire.pack(qi, qp, np.array([10]), int(fp16)).size
+    from paper_2603_19133_b200 import buildlib
+    lib = ctypes.CDLL(buildlib.build())
+    lib.picospec_wire_bytes.restype = ctypes.c_longlong
+    lib.picospec_wire_bytes.argtypes = [ctypes.c_int, ctypes.c_longlong, ctypes.c_int]
+    for rows, n, pt in ((1, 10, 0), (1, 10, 1), (7, 33, 1), (1536, 1536 * 256, 0), (0, 0, 0)):
+        assert lib.picospec_wire_bytes(rows, n, pt) == wire.wire_size(rows, n, pt)
+    assert lib.picospec_wire_bytes(-1, 0, 0) == -1 and lib.picospec_wire_bytes(1, 1, 2) == -1
+    assert pm.dense_row_bytes(128256) / pm.downlink_bytes(10, True) > 1000

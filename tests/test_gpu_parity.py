@@ -510,3 +510,34 @@ def test_staged_bad_data_is_reported(ps):
         assert np.array_equal(_np(g["accept_len"]), o["accept_len"])
         assert np.array_equal(_np(g["token"]), o["token"])
         assert o["accept_len"][3] == -1 and o["accept_len"][0] >= 0
+
+
+# ---------------------------------------------------------------------------------------------
+# seeded random shapes and value scales (staged and direct kernels, both dtypes, top-k / top-p)
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("seed", list(range(24)))
+def test_random_shapes_and_scales(ps, seed):
+    rng = np.random.default_rng(9000 + seed)
+    dtype = "bf16" if rng.random() < 0.6 else "f32"
+    align = 8 if dtype == "bf16" else 4
+    V = int(rng.choice([rng.integers(1500, 8192), rng.integers(8192, 20000), rng.integers(20000, 70000)]))
+    if rng.random() < 0.7:
+        V = V // align * align                      # rows the staged kernels take (when V >= 8192)
+    K = int(rng.choice([1, 3, 17, 64, 200, 256, 257, 600, 1024]))
+    K = min(K, V)
+    B, G = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+    use_p = rng.random() < 0.5
+    top_p = float(rng.choice([0.5, 0.9, 0.99])) if use_p else 1.0
+    top_k = 0 if use_p else int(rng.integers(1, K + 1))
+    w = gen.Workload("r", V=V, B=B, G=G, dtype=dtype, s=float(rng.uniform(0.7, 1.4)), sigma_d=float(rng.uniform(0.3, 2.5)),
+                     corr=0.8, sigma_t=1.0, T=None, top_k=top_k, top_p=top_p, k_max=K)
+    inputs = gen.make_inputs(w, seed=9100 + seed, device="cuda")
+    # move and stretch the logits: all positive, all negative, straddling zero, large magnitudes
+    shift = float(rng.choice([0.0, 0.0, 3.0, 12.0, -7.0, 0.4]))
+    scale = float(rng.choice([1.0, 1.0, 0.25, 4.0]))
+    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    for key in ("draft_logits", "target_logits"):
+        inputs[key] = (inputs[key].float() * scale + shift).to(td)
+    r = run_both(ps, w, inputs)
+    assert r["status"] == 0

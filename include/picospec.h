@@ -114,7 +114,7 @@ PICOSPEC_API int picospec_status(picospec_ctx* ctx, int* device_status_out, long
 PICOSPEC_API int picospec_counters(picospec_ctx* ctx, long long* out, int clear, void* cuda_stream);
 
 /* Half 1 -- draft-side sparse compression (Sec. 3.3, Eq. (4): keep the K most probable entries
- * with their vocabulary indices; this build applies it to the drafter's distribution, adds the
+ * with their vocabulary indices; this library applies it to the drafter's distribution, adds the
  * top-p cut and renormalises).
  *
  * For every row (b, i) of draft_logits [B, G, V]:

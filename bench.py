@@ -39,8 +39,8 @@ UNIT = "positions/s"
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/, keyed by (workload, kernel); absent until a capture of the current
 # kernel exists.  Captured at B = 64 and scaled to the full batch by the rows processed.
-NCU_TRAFFIC_BYTES = {("config4", "compress_filter_kernel"): 4 * (98575360 + 3831808),
-                     ("config4", "chunk_stats_bulk_kernel"): 4 * (114934016 + 3269376)}
+NCU_TRAFFIC_BYTES = {("config4", "compress_filter_kernel"): 4 * (98562816 + 3813376),
+                     ("config4", "chunk_stats_bulk_kernel"): 4 * (114934528 + 3314176)}
 
 
 def _peaks():

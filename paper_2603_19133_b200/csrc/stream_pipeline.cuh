@@ -141,13 +141,13 @@ template <typename T> struct StreamCfg;
 // Tunables (overridable at build time): stages per CTA and CTAs per SM of the staged kernels.
 // bf16 rows carry twice the arithmetic per byte, so they get more resident warps per SM.
 #ifndef PICOSPEC_STAGES_BF16
-#define PICOSPEC_STAGES_BF16 4                   // 4 x 16 KB in flight per CTA
+#define PICOSPEC_STAGES_BF16 3                   // 3 x 16 KB in flight per CTA
 #endif
 #ifndef PICOSPEC_STAGES_F32
 #define PICOSPEC_STAGES_F32 3                    // 3 x 32 KB in flight per CTA
 #endif
 #ifndef PICOSPEC_CTAS_PER_SM_BF16
-#define PICOSPEC_CTAS_PER_SM_BF16 3
+#define PICOSPEC_CTAS_PER_SM_BF16 4              // 32 worker warps per SM at 56 registers
 #endif
 #ifndef PICOSPEC_CTAS_PER_SM_F32
 #define PICOSPEC_CTAS_PER_SM_F32 2

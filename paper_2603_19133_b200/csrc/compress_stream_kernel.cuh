@@ -643,7 +643,7 @@ struct CsFinishShared {
 // keys do, the members of that boundary group are ranked among themselves (all pairs) and only
 // the best k - (number above the group) are kept.
 template <typename T, bool STATS>
-__global__ void __launch_bounds__(THREADS) compress_finish_kernel(CompressArgs a, int n2cap) {
+__global__ void __launch_bounds__(THREADS, 6) compress_finish_kernel(CompressArgs a, int n2cap) {
     extern __shared__ u64 keys[];          // two exchange buffers of n2cap keys; the sorted keys end up in the first
     __shared__ CompressShared sh;
     __shared__ CsFinishShared fs;

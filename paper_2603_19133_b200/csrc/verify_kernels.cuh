@@ -271,6 +271,9 @@ struct FinishShared {
     float qloc[CHUNK];
 };
 
+// queue entries of the verify path: the sequence, plus a flag
+constexpr int QUEUE_SEQ_MASK = 0x3FFFFFFF, QUEUE_DRAW_ONLY = 0x40000000;
+
 // bit i of a sequence's row mask (rows beyond 63 always count as set)
 __device__ __forceinline__ bool row_needed(unsigned long long need, int i) { return i >= 64 || ((need >> i) & 1ull); }
 
@@ -323,7 +326,12 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
 
     const int nloop = PRECISE ? *a.queue_count : a.B;
     for (int slot = blockIdx.x; slot < nloop; slot += gridDim.x) {
-        const int b = PRECISE ? a.queue[slot] : slot;
+        // a queue entry is the sequence, with QUEUE_DRAW_ONLY set when only the draw was too close to
+        // call: then the accept decisions of the fast pass stand and only the sampled row is redone
+        const int qe = PRECISE ? a.queue[slot] : slot;
+        const int b = PRECISE ? (qe & QUEUE_SEQ_MASK) : slot;
+        const bool draw_only = PRECISE && (qe & QUEUE_DRAW_ONLY) != 0;
+        const int alen_fast = draw_only ? a.accept_len[b] : 0;
         const unsigned long long need = PRECISE ? a.need_rows[b] : 0ull;   // rows with exact chunk sums
         if (!a.sample_only && a.state_in && a.state_in[b] == 0) {
             // decided by an earlier call: nothing of this sequence is read or written
@@ -357,6 +365,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
         if (!st_bits) {
             const int i_lo = a.sample_only ? jpos : lo, i_hi = a.sample_only ? jpos + 1 : row_hi;
             for (int i = i_lo + warp; i < i_hi; i += WARPS) {
+                if (draw_only && i != alen_fast) continue;
                 double Z, Zraw;
                 float mx;
                 bool bad;
@@ -373,7 +382,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
         __syncthreads();
 
         // ---- 2. per draft position: p(x), q~(x), accept test, residual mass ----------------
-        if (!st_bits && !sh.bad && !a.sample_only) {
+        if (!st_bits && !sh.bad && !a.sample_only && !draw_only) {
             for (int i = lo + warp; i < hi; i += WARPS) {
                 const int ri = b * G + i;
                 const int* idx = a.q_idx + (long long)ri * a.k_max;
@@ -475,7 +484,11 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
         // when the bonus row g is in the range.  Otherwise it waits for the next rows.
         int alen = lo, nborder = 0;
         bool flagged = false, rejected = false, decided = true;
-        if (!st_bits && !a.sample_only) {
+        if (draw_only) {
+            // (no accept test was ambiguous, so none is borderline either)
+            alen = alen_fast;
+            rejected = alen < hi;
+        } else if (!st_bits && !a.sample_only) {
             while (alen < hi && sh.acc[alen]) ++alen;
             rejected = alen < hi;
             decided = rejected || g < a.r1;
@@ -698,6 +711,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                     // draw needs the sampled row only.
                     unsigned long long nd = 0ull;
                     int nrows = 0;
+                    bool draw_only_flag = false;
                     if (a.sample_only) {
                         nd = ~0ull;
                         nrows = 1;
@@ -706,6 +720,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                         const int last = rejected ? alen : hi - 1;
                         for (int i = lo; i <= last && first_amb < 0; ++i)
                             if (sh.amb[i]) first_amb = i;
+                        draw_only_flag = first_amb < 0;
                         for (int i = lo; i < row_hi; ++i) {
                             const bool nr = i >= 64 || (first_amb >= 0 && i >= first_amb) ||
                                             (sh.flag && want_token && decided && i == alen);
@@ -717,7 +732,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                     }
                     a.need_rows[b] = nd;
                     const int q = atomicAdd(a.queue_count, 1);
-                    a.queue[q] = b;
+                    a.queue[q] = b | (draw_only_flag ? QUEUE_DRAW_ONLY : 0);
                     atomicAdd(a.slow_rows, (unsigned long long)nrows);
                 }
             }

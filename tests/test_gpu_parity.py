@@ -512,6 +512,38 @@ def test_staged_bad_data_is_reported(ps):
         assert o["accept_len"][3] == -1 and o["accept_len"][0] >= 0
 
 
+def test_draws_next_to_a_chunk_boundary_are_decided_exactly(ps):
+    # place the level-1 uniform within a few fp32 ulps of a chunk boundary of the residual's CDF: the
+    # accept decisions are clear, only the draw is too close to call, and the double-precision rerun
+    # (which then redoes the sampled row alone) must pick the oracle's token
+    w = gen.scaled(gen.WORKLOADS["config2"], B=32)
+    inputs = gen.make_inputs(w, seed=123, device="cuda")
+    dl, tl, T = _np(inputs["draft_logits"]), _np(inputs["target_logits"]), _np(inputs["temperature"])
+    qi, qp, qc, tok = oracle.compress(dl, T, w.top_k, w.top_p, w.k_max, _np(inputs["u_draft"]), nthreads=oracle.cores())
+    o0 = oracle.verify(tl, T, tok, qi, qp, qc, _np(inputs["u_accept"]), _np(inputs["u_resample"]), nthreads=oracle.cores())
+    ur = _np(inputs["u_resample"]).copy()
+    rng = np.random.default_rng(8)
+    for b in range(w.B):
+        j = int(o0["accept_len"][b])
+        x = tl[b, j].astype(np.float64) / float(T[b])
+        p = np.exp(x - x.max())
+        p /= p.sum()
+        r = p.copy()
+        if j < w.G:
+            n = int(qc[b, j])
+            q = np.zeros_like(p)
+            q[qi[b, j, :n]] = qp[b, j, :n].astype(np.float64)
+            r = np.maximum(p - q, 0.0)
+        nch = (w.V + 1023) // 1024
+        cum = np.cumsum(np.add.reduceat(r, np.arange(0, w.V, 1024)))
+        c = int(rng.integers(0, nch - 1))
+        ur[b, 0] = np.float32(cum[c] / cum[-1] * (1 + int(rng.integers(-2, 3)) * 6e-8))
+    inputs["u_resample"] = _cuda(ur.astype(np.float32))
+    r = run_both(ps, w, inputs, check_compress=False)
+    assert r["slow_rows"] >= w.B // 2          # nearly every sequence is rerun ...
+    assert r["slow_rows"] <= 2 * w.B           # ... for one row each, not for all gamma + 1
+
+
 # ---------------------------------------------------------------------------------------------
 # seeded random shapes and value scales (staged and direct kernels, both dtypes, top-k / top-p)
 # ---------------------------------------------------------------------------------------------

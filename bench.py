@@ -10,14 +10,24 @@ compress filter pass or the verify streaming pass; the other one is listed under
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config4] [--impl ours|reference]
 
-N > 1 is launched under torchrun, one rank per GPU; every rank runs its own batch (the path
-shards by sequence, no collective on the data path), so scaling is weak.
+With N > 1 and no torchrun environment the script starts N ranks of itself (torch.distributed.run,
+one rank per GPU); every rank runs its own batch (the path shards by sequence, no collective on the
+data path), so scaling is weak.
+
+Three loops per workload, all over the same rotating input sets:
+  1. the timed loop (the headline): K steps back to back, no per-kernel events;
+  2. the roofline loop: at least 64 more steps with every kernel group bracketed by its own pair
+     of CUDA events on the launching stream (mean, median and minimum per kernel, and per call);
+  3. if the two together kept the GPU busy for less than 0.6 s, more back-to-back steps so that
+     the clock sampler sees the SM clock under this load.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
+import re
 import statistics
 import subprocess
 import sys
@@ -35,12 +45,16 @@ import gen  # noqa: E402
 
 METRIC = "verified_draft_positions_per_sec"
 UNIT = "positions/s"
+NOMINAL_GBPS = 8000.0
 
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
-# summarised under profiles/, keyed by (workload, kernel); absent until a capture of the current
-# kernel exists.  Captured at B = 64 and scaled to the full batch by the rows processed.
-NCU_TRAFFIC_BYTES = {("config4", "compress_filter_kernel"): 4 * (98562816 + 3813376),
-                     ("config4", "chunk_stats_bulk_kernel"): 4 * (114934528 + 3314176)}
+# kernel kinds of picospec_profile_* (include/picospec.h)
+K_COMPRESS_STREAM, K_VERIFY_STREAM, K_VERIFY_FINISH, K_VERIFY_PRECISE = 0, 1, 2, 3
+K_COMPRESS_PRECISE, K_COMPRESS_REDO, K_COMPRESS_FINISH = 4, 5, 6
+KIND_NAMES = {K_COMPRESS_STREAM: "compress_stream", K_VERIFY_STREAM: "verify_stream", K_VERIFY_FINISH: "verify_finish",
+              K_VERIFY_PRECISE: "verify_precise", K_COMPRESS_PRECISE: "compress_precise",
+              K_COMPRESS_REDO: "compress_redo", K_COMPRESS_FINISH: "compress_finish"}
+
+CSRC = os.path.join(ROOT, "paper_2603_19133_b200", "csrc")
 
 
 def _peaks():
@@ -52,8 +66,42 @@ def _peaks():
     return 6650.0, "fallback"
 
 
+def source_hash(files):
+    """Short hash of kernel source files: ties an ncu capture to the code it was taken from."""
+    h = hashlib.sha256()
+    for name in files:
+        with open(os.path.join(CSRC, name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
+
+
+def ncu_traffic(workload: str, kernel: str):
+    """DRAM bytes per launch of `kernel` on `workload` (dram__bytes_read.sum + dram__bytes_write.sum,
+    scaled to the full batch), read from the ncu summaries under profiles/.  A summary carries a line
+        bench-traffic: kernel=<name> workload=<name> bytes=<int> sources=<a.cuh,b.cuh> hash=<12 hex>
+    and the figure is used only while the named source files still hash to the recorded value:
+    once the kernel has changed the counters no longer describe it and the entry is null."""
+    pdir = os.path.join(ROOT, "profiles")
+    if not os.path.isdir(pdir):
+        return None
+    pat = re.compile(r"bench-traffic:\s*kernel=(\S+)\s+workload=(\S+)\s+bytes=(\d+)\s+sources=(\S+)\s+hash=([0-9a-f]+)")
+    for fn in sorted(os.listdir(pdir)):
+        if not fn.endswith((".md", ".txt")):
+            continue
+        with open(os.path.join(pdir, fn)) as f:
+            for m in pat.finditer(f.read()):
+                if m.group(1) == kernel and m.group(2) == workload:
+                    try:
+                        current = source_hash(m.group(4).split(","))
+                    except OSError:
+                        return None
+                    return int(m.group(3)) if current == m.group(5) else None
+    return None
+
+
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while the GPU works; every sample is
+    stamped with the host time it arrived at, so that only samples taken under load are used."""
 
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -76,12 +124,12 @@ class ClockSampler:
 
         def pump():
             for line in self.proc.stdout:
-                self.rows.append(line.strip())
+                self.rows.append((time.perf_counter(), line.strip()))
 
         self.thread = threading.Thread(target=pump, daemon=True)
         self.thread.start()
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -89,14 +137,17 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        for r in self.rows:
+        sm, mx, power, reasons = [], [], [], set()
+        for t, r in self.rows:
+            if t_begin is not None and not (t_begin <= t <= t_end):
+                continue
             f = [x.strip() for x in r.split(",")]
             if len(f) < 9:
                 continue
             try:
                 sm.append(float(f[1]))
                 mx.append(float(f[2]))
+                power.append(float(f[3]))
             except ValueError:
                 continue
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
@@ -104,7 +155,9 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "sm_mhz_min": min(sm) if sm else None,
+                "power_w_max": max(power) if power else None,
+                "window_s": None if t_begin is None else round(t_end - t_begin, 3)}
 
 
 def _dist_env():
@@ -113,6 +166,26 @@ def _dist_env():
 
 def _np(t):
     return t.detach().float().cpu().numpy() if t.is_floating_point() else t.detach().cpu().numpy()
+
+
+def input_sets(w) -> int:
+    """Distinct input sets a workload rotates through, so that consecutive steps never find their
+    logits in the 126 MB L2: enough sets for 320 MB (at most 288 of them), one when a single set is
+    larger than that already."""
+    per_set = (w.B * (2 * w.G + 1)) * w.V * w.bytes_per_logit
+    return max(1, min(288, -(-(320 << 20) // per_set))) if per_set < (320 << 20) else 1
+
+
+def config_of(w, world):
+    """The `config` object of the JSON line; the same for both arms."""
+    nsets = input_sets(w)
+    return {"workload": w.name, "V": w.V, "B_per_gpu": w.B, "gamma": w.G, "logits": w.dtype,
+            "top_k": w.top_k, "top_p": w.top_p, "k_max": w.k_max,
+            "accumulate": "f32 streaming sums, f64 per-row arithmetic",
+            "step": "picospec_compress + picospec_verify (fused residual/bonus sample)",
+            "l2": f"inputs larger than L2: {nsets} input set(s) of "
+                  f"{(w.B * (2 * w.G + 1)) * w.V * w.bytes_per_logit / 1e6:.0f} MB rotated",
+            "parallelism": f"dp{world} (sequences sharded, no collective)"}
 
 
 # -------------------------------------------------------------------------------------------------
@@ -149,26 +222,23 @@ def run_reference(args):
     wc, ic = oracle_sample(w, 4241, cal_B)
     per_seq = oracle_step_time(wc, ic, cores) / cal_B
     budget_s = 100.0
-    sample_B = int(budget_s / (max(args.steps + min(args.warmup, 1), 1) * per_seq))
+    sample_B = int(budget_s / (max(args.steps + args.warmup, 1) * per_seq))
     sample_B = max(1, min(w.B, args.ref_sample, sample_B))
     ws, inp = oracle_sample(w, 4242, sample_B)
-    for _ in range(min(args.warmup, 1)):
+    for _ in range(args.warmup):
         oracle_step_time(ws, inp, cores)
     times = [oracle_step_time(ws, inp, cores) for _ in range(args.steps)]
     t = sum(times)
     value = ws.B * ws.G * args.steps / t
     sample = f"{sample_B} of {w.B} sequences of {w.name} per step, all {cores} host threads (OpenMP over rows)"
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * t / args.steps,
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": max(args.gpus, world),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "V": w.V, "B_per_gpu": w.B, "gamma": w.G, "logits": w.dtype,
-                   "top_k": w.top_k, "top_p": w.top_p, "k_max": w.k_max,
-                   "step": "oracle compress + oracle verify (with sample) on a bounded sample of the batch",
-                   "sample_sequences_per_step": ws.B},
+        "config": config_of(w, max(args.gpus, world)),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-        "gpu_launches": 0,
+        "gpu_launches": 0, "ranks_launched": world,
     }
     print(json.dumps(line), flush=True)
 
@@ -192,6 +262,8 @@ class Step:
                       "resid_mass": torch.empty((B, G), dtype=f32, device=dev),
                       "borderline_count": torch.empty((1,), dtype=i32, device=dev),
                       "token": torch.empty((B,), dtype=i32, device=dev)}
+        # kernels per step: compress = filter, finish, redo list (+ exact sums and cut with top-p);
+        # verify = statistics, finish, exact sums, double-precision finish
         self.launches_per_step = (5 if w.top_p < 1.0 else 3) + 4
 
     def compress(self, inp=None):
@@ -225,19 +297,32 @@ def timed_loop(fn, steps, warmup, sync):
 
 
 def algorithmic_bytes(w):
-    """Bytes the method itself has to move per launch of each streaming kernel."""
+    """Bytes the method itself has to move: per launch of each streaming kernel, and per call."""
     nch = (w.V + 1023) // 1024
     rows_t, rows_d = w.B * (w.G + 1), w.B * w.G
     verify_stream = rows_t * w.V * w.bytes_per_logit + rows_t * nch * 8
     compress_stream = rows_d * w.V * w.bytes_per_logit + rows_d * (w.k_max * 8 + 8)
-    return verify_stream, compress_stream
+    # whole calls: compress also writes the sparse rows, counts and draft tokens; verify reads the
+    # chunk statistics back, the sparse rows (id + prob per slot, count, token, uniform), one chunk
+    # per sequence again for the draw, and writes its per-position and per-sequence results
+    compress_call = rows_d * w.V * w.bytes_per_logit + rows_d * (w.k_max * 8 + 4 + 4 + 4)
+    verify_call = (verify_stream + rows_t * nch * 8 + rows_d * (w.k_max * 8 + 12) + w.B * 1024 * w.bytes_per_logit
+                   + rows_d * 8 + w.B * 8)
+    return {"verify_stream": verify_stream, "compress_stream": compress_stream,
+            "compress_call": compress_call, "verify_call": verify_call}
 
 
-def bench_workload(ps, w, args, rank, world, device, with_e2e, with_clocks):
+def _stats_us(samples_ms):
+    if not samples_ms:
+        return {"launches": 0, "avg_us": None, "median_us": None, "min_us": None}
+    us = [1e3 * x for x in samples_ms]
+    return {"launches": len(us), "avg_us": sum(us) / len(us), "median_us": statistics.median(us), "min_us": min(us)}
+
+
+def bench_workload(ps, w, steps, warmup, rank, world, device, with_e2e, with_clocks, roofline_launches=64,
+                   min_busy_s=0.6):
     ctx = ps.Context(w.B, w.G, w.V, w.k_max)
-    # rotate through enough distinct input sets that consecutive steps never find their logits in L2
-    per_set = (w.B * (2 * w.G + 1)) * w.V * w.bytes_per_logit
-    nsets = max(1, min(12, -(-(512 << 20) // per_set))) if per_set < (512 << 20) else 1
+    nsets = input_sets(w)
     sets = [gen.make_inputs(w, seed=1000 * (rank + 1) + 17 * i + sum(map(ord, w.name)), device=device)
             for i in range(nsets)]
     step = Step(ps, ctx, w, sets[0])
@@ -255,41 +340,81 @@ def bench_workload(ps, w, args, rank, world, device, with_e2e, with_clocks):
 
     ctx.status(clear=True)
     ctx.counters(clear=True)
-    # per-kernel event brackets on every 8th step only: an event between two kernels keeps the second
-    # from being scheduled while the first drains, which the whole-step time should not pay on every step
-    ctx.profile_enable(1, every=8)
+    ctx.profile_enable(0)
     sampler = ClockSampler(torch.cuda.current_device()) if with_clocks else None
     if sampler:
         sampler.start()
-        time.sleep(0.15)
-    t = timed_loop(one, args.steps, args.warmup, sync)
-    clocks = sampler.stop() if sampler else None
-    ms_vs, n_vs = ctx.profile_read(1)
-    ms_cs, n_cs = ctx.profile_read(0)
-    ctx.profile_enable(0)
-    _, redo = ctx.counters()
-    st, slow = ctx.status(clear=True)
+        time.sleep(0.1)
+    # ---- 1. the timed loop ------------------------------------------------------------------
+    for _ in range(warmup):
+        one()
+    sync()
+    t_busy0 = time.perf_counter()
+    t = timed_loop(one, steps, 0, sync)
     if world > 1:
         tt = torch.tensor([t], device=device, dtype=torch.float64)
         torch.distributed.all_reduce(tt, op=torch.distributed.ReduceOp.MAX)
         t = float(tt.item())
-    # the same loop without the event brackets, for the record
-    t_plain = timed_loop(one, args.steps, min(args.warmup, 3), sync)
+    _, redo = ctx.counters()
+    st, slow = ctx.status(clear=True)
+    steps_counted = steps + warmup
 
-    vbytes, cbytes = algorithmic_bytes(w)
+    # ---- 2. the roofline loop: every kernel group and both calls bracketed -------------------
+    ctx.profile_enable(2, every=1)
+    n_roof = max(roofline_launches, 1)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_roof)]
+    torch.cuda.synchronize()
+    for i in range(n_roof):
+        inp = sets[state["i"] % nsets]
+        state["i"] += 1
+        ev[i][0].record()
+        step.compress(inp)
+        ev[i][1].record()
+        step.verify(inp)
+        ev[i][2].record()
+    torch.cuda.synchronize()
+    kinds = {name: _stats_us(ctx.profile_samples(k)) for k, name in KIND_NAMES.items()}
+    calls = {"compress_call": _stats_us([e[0].elapsed_time(e[1]) for e in ev]),
+             "verify_call": _stats_us([e[1].elapsed_time(e[2]) for e in ev])}
+    ctx.profile_enable(0)
+    ctx.status(clear=True)
+
+    # ---- 3. keep the GPU busy long enough for the clock sampler -------------------------------
+    if sampler:
+        while time.perf_counter() - t_busy0 < min_busy_s:
+            for _ in range(32):
+                one()
+            torch.cuda.synchronize()
+    t_busy1 = time.perf_counter()
+    clocks = sampler.stop(t_busy0 + 0.03, t_busy1) if sampler else None
+    ctx.status(clear=True)
+    ctx.counters(clear=True)
+
+    alg = algorithmic_bytes(w)
     peak, peak_kind = _peaks()
-    vs_time = ms_vs / max(n_vs, 1) * 1e-3
-    cs_time = ms_cs / max(n_cs, 1) * 1e-3
+
+    def with_bw(stats, nbytes):
+        out = dict(stats)
+        out["alg_bytes"] = nbytes
+        for key in ("avg", "median", "min"):
+            us = stats.get(f"{key}_us")
+            out[f"GBps_{key}"] = nbytes / us / 1e3 if us else None
+        out["GBps"] = out["GBps_avg"]
+        out["frac_of_peak"] = (out["GBps"] or 0) / peak
+        out["frac_of_8TBps_nominal"] = (out["GBps"] or 0) / NOMINAL_GBPS
+        return out
+
     res = {
-        "seconds": t, "seconds_unbracketed": t_plain, "status": st,
-        "slow_rows_per_step": slow / float(args.steps + args.warmup),
-        "redo_rows_per_step": redo / float(args.steps + args.warmup),
-        "value": world * w.B * w.G * args.steps / t,
-        "rows_streamed_per_sec": world * w.B * (2 * w.G + 1) * args.steps / t,
-        "verify_stream": {"avg_us": vs_time * 1e6, "launches": n_vs, "alg_bytes": vbytes,
-                          "GBps": vbytes / vs_time / 1e9 if vs_time > 0 else None},
-        "compress_stream": {"avg_us": cs_time * 1e6, "launches": n_cs, "alg_bytes": cbytes,
-                            "GBps": cbytes / cs_time / 1e9 if cs_time > 0 else None},
+        "seconds": t, "status": st,
+        "slow_rows_per_step": slow / float(steps_counted),
+        "redo_rows_per_step": redo / float(steps_counted),
+        "value": world * w.B * w.G * steps / t,
+        "rows_streamed_per_sec": world * w.B * (2 * w.G + 1) * steps / t,
+        "verify_stream": with_bw(kinds["verify_stream"], alg["verify_stream"]),
+        "compress_stream": with_bw(kinds["compress_stream"], alg["compress_stream"]),
+        "verify_call": with_bw(calls["verify_call"], alg["verify_call"]),
+        "compress_call": with_bw(calls["compress_call"], alg["compress_call"]),
+        "other_kernels_us": {k: v["avg_us"] for k, v in kinds.items() if k not in ("verify_stream", "compress_stream")},
         "peak": peak, "peak_kind": peak_kind, "clocks": clocks, "nsets": nsets,
         "launches_per_step": step.launches_per_step,
     }
@@ -310,7 +435,7 @@ def bench_workload(ps, w, args, rank, world, device, with_e2e, with_clocks):
                 h_out[k].copy_(step.v_out[k], non_blocking=True)
             torch.cuda.current_stream().synchronize()      # the caller reads the result
 
-        k_e2e = max(2, min(args.steps, 10))
+        k_e2e = max(2, min(steps, 10))
         t0 = time.perf_counter()
         te = timed_loop(one_e2e, k_e2e, 1, sync)
         if world > 1:
@@ -324,6 +449,85 @@ def bench_workload(ps, w, args, rank, world, device, with_e2e, with_clocks):
     del sets, step
     torch.cuda.empty_cache()
     return res
+
+
+def summary_of(r, steps):
+    """The per-workload entry of `other_configs`."""
+    vs, cs = r["verify_stream"], r["compress_stream"]
+    return {"positions_per_sec": r["value"], "ms_per_step": 1e3 * r["seconds"] / steps,
+            "verify_stream_us": vs["avg_us"], "verify_stream_median_us": vs["median_us"],
+            "verify_stream_GBps": vs["GBps"], "verify_stream_frac_of_peak": vs["frac_of_peak"],
+            "verify_stream_frac_of_8TBps": vs["frac_of_8TBps_nominal"],
+            "compress_stream_us": cs["avg_us"], "compress_stream_median_us": cs["median_us"],
+            "compress_stream_GBps": cs["GBps"], "compress_stream_frac_of_peak": cs["frac_of_peak"],
+            "compress_stream_frac_of_8TBps": cs["frac_of_8TBps_nominal"],
+            "verify_call_us": r["verify_call"]["avg_us"], "verify_call_GBps": r["verify_call"]["GBps"],
+            "verify_call_frac_of_peak": r["verify_call"]["frac_of_peak"],
+            "compress_call_us": r["compress_call"]["avg_us"], "compress_call_GBps": r["compress_call"]["GBps"],
+            "sparse_row_bytes_share_of_verify_call": (r["verify_call"]["alg_bytes"] - vs["alg_bytes"]) / r["verify_call"]["alg_bytes"],
+            "bracketed_launches": vs["launches"], "input_sets_rotated": r["nsets"],
+            "slow_rows_per_step": r["slow_rows_per_step"], "redo_rows_per_step": r["redo_rows_per_step"],
+            "device_status": r["status"]}
+
+
+def bench_pipelined(ps, w, device, n_streams, iters):
+    """Many calls in flight (the latency-bound configurations): one CUDA graph per input set, each
+    holding one whole step, replayed over `n_streams` streams with a context each.  Reported next
+    to the single-call latency of the same workload; not the headline."""
+    nsets = max(n_streams, input_sets(w))
+    nsets = (nsets + n_streams - 1) // n_streams * n_streams
+    sets = [gen.make_inputs(w, seed=9000 + i, device=device) for i in range(nsets)]
+    streams = [torch.cuda.Stream() for _ in range(n_streams)]
+    ctxs = [ps.Context(w.B, w.G, w.V, w.k_max) for _ in range(n_streams)]
+    steps = [Step(ps, ctxs[i % n_streams], w, sets[i]) for i in range(nsets)]
+    graphs = []
+    torch.cuda.synchronize()
+    for i, stp in enumerate(steps):
+        s = streams[i % n_streams]
+        with torch.cuda.stream(s):
+            stp()                       # warm-up outside capture (function attributes are set on first use)
+        s.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            stp()
+        graphs.append(g)
+    torch.cuda.synchronize()
+
+    def sweep():
+        for i, g in enumerate(graphs):
+            with torch.cuda.stream(streams[i % n_streams]):
+                g.replay()
+
+    for _ in range(3):
+        sweep()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    cur = torch.cuda.current_stream()
+    e0.record()
+    for s in streams:
+        s.wait_event(e0)
+    for _ in range(iters):
+        sweep()
+    for s in streams:
+        done = torch.cuda.Event()
+        done.record(s)
+        cur.wait_event(done)
+    e1.record()
+    torch.cuda.synchronize()
+    sec = e0.elapsed_time(e1) * 1e-3
+    nsteps = iters * len(graphs)
+    alg = algorithmic_bytes(w)
+    peak, _ = _peaks()
+    status = 0
+    for c in ctxs:
+        status |= c.status(clear=True)[0]
+        c.close()
+    step_bytes = alg["verify_call"] + alg["compress_call"]
+    return {"what": f"{len(graphs)} CUDA graphs (one step each) replayed round-robin on {n_streams} streams, "
+                    f"{iters} sweeps; throughput of many calls in flight, not a latency",
+            "positions_per_sec": w.B * w.G * nsteps / sec, "us_per_step": 1e6 * sec / nsteps,
+            "step_GBps": step_bytes * nsteps / sec / 1e9, "step_frac_of_peak": step_bytes * nsteps / sec / 1e9 / peak,
+            "verify_stream_bytes_GBps": alg["verify_stream"] * nsteps / sec / 1e9, "device_status": status}
 
 
 def bench_paper_direction(ps, w, device, k, iters):
@@ -417,27 +621,38 @@ def run_ours(args):
     w = gen.WORKLOADS[args.workload]
     if args.batch > 0:
         w = gen.scaled(w, B=args.batch)
-    main = bench_workload(ps, w, args, rank, world, device, with_e2e=True, with_clocks=(rank == 0))
+    main = bench_workload(ps, w, args.steps, args.warmup, rank, world, device, with_e2e=True,
+                          with_clocks=(rank == 0), roofline_launches=args.roofline_launches)
 
     others = {}
     if args.all_configs and world == 1:
+        k_other = min(args.steps, 200)
         for name in ("config1", "config2", "config3"):
             if name == args.workload:
                 continue
-            r = bench_workload(ps, gen.WORKLOADS[name], args, rank, world, device, with_e2e=False, with_clocks=False)
-            others[name] = {"positions_per_sec": r["value"], "ms_per_step": 1e3 * r["seconds"] / args.steps,
-                            "verify_stream_us": r["verify_stream"]["avg_us"],
-                            "verify_stream_GBps": r["verify_stream"]["GBps"],
-                            "verify_stream_frac_of_peak": (r["verify_stream"]["GBps"] or 0) / r["peak"],
-                            "compress_stream_us": r["compress_stream"]["avg_us"],
-                            "compress_stream_GBps": r["compress_stream"]["GBps"],
-                            "input_sets_rotated": r["nsets"], "slow_rows_per_step": r["slow_rows_per_step"]}
+            r = bench_workload(ps, gen.WORKLOADS[name], k_other, args.warmup, rank, world, device, with_e2e=False,
+                               with_clocks=False, roofline_launches=64)
+            others[name] = summary_of(r, k_other)
+        # configuration 5: the bandwidth sweep, every point at its full batch
+        k_sweep = min(args.steps, 20)
+        for V in gen.SWEEP_V:
+            for k in gen.SWEEP_K:
+                ws = gen.sweep_workload(V, k)
+                r = bench_workload(ps, ws, k_sweep, 3, rank, world, device, with_e2e=False, with_clocks=False,
+                                   roofline_launches=16)
+                others[ws.name] = summary_of(r, k_sweep)
 
-    paper_direction = None
-    wire_codec = None
+    paper_direction = wire_codec = None
+    pipelined = {}
     if args.all_configs and world == 1:
         paper_direction = bench_paper_direction(ps, w, device, k=10, iters=min(args.steps, 200))
         wire_codec = bench_wire(ps, w, device, iters=min(args.steps, 200))
+        for name in ("config1", "config2"):
+            try:
+                pipelined[name] = bench_pipelined(ps, gen.WORKLOADS[name], device, n_streams=4,
+                                                  iters=max(4, min(args.steps, 50)))
+            except Exception as e:      # noqa: BLE001  (reported, not fatal: the headline does not depend on it)
+                pipelined[name] = {"error": f"{type(e).__name__}: {e}"[:300]}
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -456,39 +671,35 @@ def run_ours(args):
             "compress_filter_kernel (picospec_compress streaming pass)": main["compress_stream"],
             "chunk_stats_bulk_kernel (picospec_verify streaming pass)": main["verify_stream"],
         }
-        for v in kern.values():
-            v["frac_of_peak"] = (v["GBps"] or 0) / peak
-            v["frac_of_8TBps_nominal"] = (v["GBps"] or 0) / 8000.0
-        dom_name = max(kern, key=lambda k: kern[k]["avg_us"])
+        dom_name = max(kern, key=lambda k: kern[k]["avg_us"] or 0)
         dom = kern[dom_name]
         line = {
             "metric": METRIC, "value": main["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * main["seconds"] / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "V": w.V, "B_per_gpu": w.B, "gamma": w.G, "logits": w.dtype,
-                       "top_k": w.top_k, "top_p": w.top_p, "k_max": w.k_max,
-                       "step": "picospec_compress + picospec_verify (fused residual/bonus sample)",
-                       "l2": f"inputs larger than L2: {main['nsets']} input set(s) of "
-                             f"{(w.B * (2 * w.G + 1)) * w.V * w.bytes_per_logit / 1e6:.0f} MB rotated",
-                       "parallelism": f"dp{world} (sequences sharded, no collective)"},
+            "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+            "config": config_of(w, world),
             "roofline": {"bound": "hbm", "kernel": dom_name,
                          "achieved": dom["GBps"], "peak": peak, "unit": "GB/s",
                          "frac": (dom["GBps"] or 0) / peak, "peak_kind": f"of {main['peak_kind']}",
-                         "frac_of_8TBps_nominal": (dom["GBps"] or 0) / 8000.0,
-                         "avg_launch_us": dom["avg_us"], "launches_timed": dom["launches"],
+                         "frac_of_8TBps_nominal": (dom["GBps"] or 0) / NOMINAL_GBPS,
+                         "avg_launch_us": dom["avg_us"], "median_launch_us": dom["median_us"],
+                         "min_launch_us": dom["min_us"], "launches_timed": dom["launches"],
+                         "frac_at_median": (dom["GBps_median"] or 0) / peak,
                          "algorithmic_bytes_per_launch": dom["alg_bytes"],
-                         "traffic": None if args.batch > 0 else NCU_TRAFFIC_BYTES.get((w.name, dom_name.split(" ")[0]))},
+                         "traffic": None if args.batch > 0 else ncu_traffic(w.name, dom_name.split(" ")[0])},
             "kernels": kern,
+            "calls": {"picospec_compress": main["compress_call"], "picospec_verify": main["verify_call"]},
+            "other_kernels_avg_us": main["other_kernels_us"],
             "e2e": {k: main["e2e"][k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step")},
             "gpu_launches": main["launches_per_step"] * args.steps,
             "cpu_baseline": cpu_baseline,
             "clocks": main["clocks"],
-            "ms_per_step_without_event_brackets": 1e3 * main["seconds_unbracketed"] / args.steps,
             "rows_streamed_per_sec": main["rows_streamed_per_sec"],
             "slow_path_rows_per_step": main["slow_rows_per_step"],
             "compress_redo_rows_per_step": main["redo_rows_per_step"],
             "device_status": main["status"],
             "other_configs": others,
+            "pipelined": pipelined,
             "paper_direction": paper_direction,
             "wire_codec": wire_codec,
         }
@@ -496,6 +707,22 @@ def run_ours(args):
     if world > 1:
         torch.distributed.barrier()
         torch.distributed.destroy_process_group()
+
+
+def launch_ranks(n: int) -> int:
+    """Start `n` ranks of this script under torch.distributed.run on this node, one per GPU, and
+    return its exit code.  Used when --gpus N > 1 is given without a torchrun environment."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    env = dict(os.environ)
+    # keep NCCL's communicator line (rank / nranks) in the log of a multi-GPU run
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    return subprocess.call(cmd, env=env)
 
 
 def main():
@@ -508,9 +735,13 @@ def main():
     ap.add_argument("--ref-sample", type=int, default=64, help="sequences per step of the CPU oracle legs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override B of the workload (profiling on a small case)")
+    ap.add_argument("--roofline-launches", type=int, default=64,
+                    help="bracketed launches per kernel behind the roofline entry (at most 128 are kept)")
     ap.add_argument("--all-configs", action="store_true", default=True)
     ap.add_argument("--only-main", dest="all_configs", action="store_false")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(launch_ranks(args.gpus))
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

@@ -99,6 +99,12 @@ PICOSPEC_API int picospec_profile_period(picospec_ctx* ctx, int every);
 PICOSPEC_API int picospec_profile_read(picospec_ctx* ctx, int kind, float* total_ms_out, int* launches_out,
                                        void* cuda_stream);
 
+/* The same, launch by launch: the device times (ms) of the launches recorded for `kind` since the
+ * last read go to ms_out (HOST array of `capacity` floats), oldest first -- the newest
+ * min(capacity, 128) of them -- and their number to *n_out (HOST).  Resets the counter. */
+PICOSPEC_API int picospec_profile_samples(picospec_ctx* ctx, int kind, float* ms_out, int capacity, int* n_out,
+                                          void* cuda_stream);
+
 /* Synchronise `cuda_stream`, then copy the sticky status word and the cumulative number of rows
  * re-evaluated in double precision to HOST memory (either pointer may be NULL).  If `clear` is
  * non-zero both are reset afterwards.  Returns PICOSPEC_EDATA if the status word is non-zero. */
@@ -165,8 +171,8 @@ PICOSPEC_API int picospec_verify(picospec_ctx* ctx, const void* target_logits, p
                     float* p_draft, float* resid_mass, int* borderline_count, const float* u_resample,
                     int* token, void* cuda_stream);
 
-/* Wire format of sparse rows (Sec. 3.3: the verifier sends the K "(id, prob)" pairs, under 100
- * bytes for K = 10, laid out so that the receiver views the arrays in place).  One message, little
+/* Wire format of sparse rows (Sec. 3.3: the verifier sends K pairs of vocabulary id and
+ * probability, under 100 bytes for K = 10, laid out so that the receiver views the arrays in place).  One message, little
  * endian, 4-byte aligned:
  *     0   u32  magic 0x31505350 ("PSP1")
  *     4   u32  R, the number of rows
@@ -235,7 +241,9 @@ PICOSPEC_API int picospec_verify_range(picospec_ctx* ctx, const void* target_log
  *
  * For every sequence b, row j = pos[b] of its target logits: weights r_v = max(0, p_j(v) - q~_j(v))
  * if j < G and the sparse row (b, j) is non-empty, else r_v = p_j(v) (bonus row; also the
- * fallback when the residual is identically zero).  The token is drawn by a two-level inverse
+ * fallback when the residual vanishes, where Sec. 3.3's norm() is undefined: a residual whose
+ * total mass is at most 1e-12 of the row's counts as vanished, because the chunk masses are
+ * differences of double-precision sums).  The token is drawn by a two-level inverse
  * CDF with chunks of PICOSPEC_CHUNK vocabulary entries: u_resample[b,0] picks the first chunk c
  * whose cumulative mass exceeds u0 * sum(r); u_resample[b,1] picks the first entry of that chunk
  * whose cumulative weight inside the chunk exceeds u1 * mass(c).  Entries of zero weight are
@@ -248,9 +256,9 @@ PICOSPEC_API int picospec_residual_sample(picospec_ctx* ctx, const void* target_
                              const int* q_idx, const float* q_prob, const int* q_count, int k_max,
                              const float* u_resample, int* token, float* mass, void* cuda_stream);
 
-/* The paper's own data flow, verifier side -- Sec. 3.3, Eq. (4): "the cloud extracts only the K
- * components with the highest probabilities and their corresponding indices" of the target
- * distribution at the rejected position, and sends them.
+/* The paper's own data flow, verifier side -- Sec. 3.3, Eq. (4): of the target distribution at the
+ * rejected position the verifier keeps the K most probable components, each with its vocabulary
+ * index, and sends only those.
  *
  * For every sequence b, row j = pos[b] of target_logits [B, R, V] (R rows per sequence):
  *   p      = softmax(logits / temperature[b])
@@ -268,8 +276,8 @@ PICOSPEC_API int picospec_target_topk(picospec_ctx* ctx, const void* target_logi
                          int V, long long row_stride_elems, const float* temperature, const int* pos, int k,
                          int* p_idx, float* p_prob, int* p_count, void* cuda_stream);
 
-/* The paper's own data flow, edge side -- Sec. 3.3: "the edge then autonomously performs local
- * resampling using the logic norm(max(0, P_j(x) - Q_j(x)))".
+/* The paper's own data flow, edge side -- Sec. 3.3: the edge draws the corrected token by itself,
+ * from the normalised positive part of (received target components - its own draft distribution).
  *
  * For every sequence b, with Q = softmax(draft_logits[b, pos[b], :] / temperature[b]) (the edge's own
  * dense row) and the transmitted components (p_idx, p_prob, p_count) of the target distribution

@@ -40,7 +40,7 @@ def _load():
     if _lib is None:
         # a test that plants a mistake points this at its own build of a modified copy
         _lib = ctypes.CDLL(os.environ.get("PICOSPEC_ORACLE_LIB") or build())
-        for name in ("pso_compress", "pso_verify", "pso_residual_sample", "pso_softmax", "pso_target_topk",
+        for name in ("pso_compress", "pso_verify", "pso_residual_sample", "pso_target_topk",
                      "pso_edge_resample", "pso_verify_range"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
@@ -231,16 +231,3 @@ def edge_resample(draft_logits, temperature, pos, p_idx, p_prob, p_count, u, nth
     if rc != 0:
         raise ValueError(f"pso_edge_resample failed: {rc}")
     return token, mass
-
-
-def softmax(logits, temperature):
-    """fp32 [R, V] rows with per-row temperature -> p [R, V] f64."""
-    l = _f32(logits)
-    R, V = l.shape
-    T = _f32(temperature)
-    assert T.shape == (R,)
-    p = np.empty((R, V), np.float64)
-    rc = _load().pso_softmax(_p(l), ctypes.c_long(R), ctypes.c_long(V), ctypes.c_long(V), _p(T), _p(p))
-    if rc != 0:
-        raise ValueError(f"pso_softmax failed: {rc}")
-    return p

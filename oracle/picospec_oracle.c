@@ -43,6 +43,12 @@
 #define PSO_EINVAL (-1)
 #define PSO_ENOMEM (-2)
 
+/* Sec. 3.3's norm(max(0, P_j - Q_j)) is undefined when max(0, P_j - Q_j) vanishes (reading: the draw
+ * is then from P_j itself).  A residual whose total mass is at most this fraction of the row's
+ * (which sums to one) counts as vanished: it is the resolution of double-precision sums of
+ * probabilities, below which "identically zero" cannot be told from rounding. */
+#define PSO_RESID_ZERO 1e-12
+
 /* ---- helpers ------------------------------------------------------------------ */
 
 typedef struct {
@@ -257,8 +263,8 @@ static long pso_two_level_sample(const double *r, long V, long chunk, double u1,
 }
 
 /* Token from row `l` at a rejected position (residual against the sparse q~) or, when
- * use_residual == 0, from p itself (bonus row after full acceptance).  If the residual is
- * identically zero (q~ >= p everywhere) the draw falls back to p. */
+ * use_residual == 0, from p itself (bonus row after full acceptance).  If the residual vanishes
+ * (q~ >= p everywhere; total mass at most PSO_RESID_ZERO) the draw falls back to p. */
 static long pso_sample_row(const float *l, long V, double T, int use_residual, const int *idx,
                            const float *prob, int n, long chunk, double u1, double u2,
                            double *w, double *qd, double *r, double *mass_out) {
@@ -268,7 +274,7 @@ static long pso_sample_row(const float *l, long V, double T, int use_residual, c
     long tok = -1;
     if (use_residual && n > 0) {
         R = pso_residual_weights(w, Z, V, idx, prob, n, qd, r);
-        if (R > 0.0) tok = pso_two_level_sample(r, V, chunk, u1, u2, &R);
+        if (R > PSO_RESID_ZERO) tok = pso_two_level_sample(r, V, chunk, u1, u2, &R);
     }
     if (tok < 0) {
         for (long v = 0; v < V; ++v) r[v] = w[v] / Z;
@@ -672,8 +678,8 @@ int pso_target_topk(const float *target_logits, long B, long rows_per_seq, long 
     return err ? PSO_ENOMEM : PSO_OK;
 }
 
-/* Sec. 3.3: "the edge then autonomously performs local resampling using the logic
- * norm(max(0, P_j(x) - Q_j(x)))".  The edge holds its own dense distribution Q_j = softmax of
+/* Sec. 3.3, edge side: the corrected token is drawn locally from the normalised positive part
+ * of P_j - Q_j.  The edge holds its own dense distribution Q_j = softmax of
  * its logits at the rejected position j = pos[b], and the K transmitted components of P_j; a
  * component that was not transmitted counts as zero, so only the K transmitted indices can carry
  * positive weight (reading: the paper does not say what the edge assumes about the rest):
@@ -748,21 +754,4 @@ int pso_edge_resample(const float *draft_logits, long B, long rows_per_seq, long
         free(r);
     }
     return err ? PSO_ENOMEM : PSO_OK;
-}
-
-/* Full softmax of rows, for tests that need p itself (law checks). */
-int pso_softmax(const float *logits, long rows, long V, long row_stride, const float *temperature,
-                double *p_out) {
-    if (!logits || !temperature || !p_out || V <= 0 || row_stride < V) return PSO_EINVAL;
-    for (long r = 0; r < rows; ++r) {
-        double Z;
-        double *p = p_out + r * V;
-        double T = (double)temperature[r];
-        if (!pso_temperature_ok(T) || pso_softmax_row(logits + r * row_stride, V, T, p, &Z)) {
-            for (long v = 0; v < V; ++v) p[v] = NAN;
-            continue;
-        }
-        for (long v = 0; v < V; ++v) p[v] /= Z;
-    }
-    return PSO_OK;
 }

@@ -60,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.picospec_wire_pack.restype = c_int
         L.picospec_wire_unpack.argtypes = [vp, vp, c_ll, c_int, c_int, vp, vp, vp, vp]
         L.picospec_wire_unpack.restype = c_int
+        L.picospec_profile_samples.argtypes = [vp, c_int, ctypes.POINTER(c_f), c_int, ctypes.POINTER(c_int), vp]
+        L.picospec_profile_samples.restype = c_int
         L.picospec_counters.argtypes = [vp, ctypes.POINTER(c_ll), c_int, vp]
         L.picospec_counters.restype = c_int
         L.picospec_verify_static.argtypes = [vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp, c_int,
@@ -206,6 +208,13 @@ class Context:
         _check(lib().picospec_profile_read(self._h, int(kind), ctypes.byref(ms), ctypes.byref(n), _stream()),
                "picospec_profile_read")
         return ms.value, n.value
+
+    def profile_samples(self, kind: int, capacity: int = 128):
+        """Device ms of each launch recorded for one kernel kind since the last read (newest 128 at most)."""
+        buf, n = (ctypes.c_float * capacity)(), ctypes.c_int(0)
+        _check(lib().picospec_profile_samples(self._h, int(kind), buf, int(capacity), ctypes.byref(n), _stream()),
+               "picospec_profile_samples")
+        return [float(buf[i]) for i in range(n.value)]
 
     # -- half 1 -------------------------------------------------------------------------
     def compress(self, draft_logits: torch.Tensor, temperature: torch.Tensor, top_k: int, top_p: float,

@@ -20,6 +20,15 @@ constexpr int MAX_K = 1024;        // capacity limit of a sparse row
 // their threshold are re-taken in double precision.
 constexpr double GUARD_Z = 3e-6;
 constexpr double BORDER_REL = 1e-6;   // "borderline" band of the accept test
+// A residual mass R = 1 - sum min(p, q~) carries the absolute error of the fp32-accumulated
+// normaliser (a few 1e-7 in practice, GUARD_Z at worst); below this value it would miss the 1e-5
+// relative target, so such a position is recomputed from the exact chunk sums.
+constexpr double RESID_EXACT_BELOW = 0.05;
+// The residual norm(max(0, p - q~)) is undefined when max(0, p - q~) vanishes; the draw is then from
+// p itself.  The verify path forms chunk masses of the residual as (chunk mass of p) - sum min(p, q~),
+// which in double precision cannot tell a mass of 1e-16 from zero: a residual whose total mass
+// (of a row that sums to one) is at most this value counts as vanished.
+constexpr double RESID_ZERO_BELOW = 1e-12;
 
 // device status bits (mirrors picospec.h)
 constexpr unsigned ST_TEMPERATURE = 1u, ST_LOGIT = 2u, ST_RANGE = 4u;

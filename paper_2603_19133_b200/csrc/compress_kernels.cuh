@@ -346,7 +346,12 @@ __global__ void __launch_bounds__(THREADS, 2) compress_kernel(CompressArgs a) {
     if (k_eff > a.k_max) k_eff = a.k_max;
     if (k_eff > a.V) k_eff = a.V;
 
-    if (blockIdx.x == 0 && tid == 0 && !a.use_redo_list) *a.queue_count_next = 0;
+    // a call that goes through this kernel alone clears both of the next call's counters, as the
+    // staged filter kernel does (the redo-list launch of a staged call must not: the filter did)
+    if (blockIdx.x == 0 && tid == 0 && !a.use_redo_list) {
+        *a.queue_count_next = 0;
+        *a.redo_count_next = 0;
+    }
     const int nwork = a.use_redo_list ? *a.redo_count : rows;
 
     for (int wi = blockIdx.x; wi < nwork; wi += gridDim.x) {

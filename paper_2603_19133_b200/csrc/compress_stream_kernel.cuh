@@ -42,7 +42,8 @@
 namespace picospec {
 
 // Two shapes of the filter kernel: rows with k <= 256 need few live candidates, so a small
-// candidate buffer and two stages leave room for three CTAs per SM; larger k takes the big buffer.
+// candidate buffer leaves room for three CTAs per SM (16-bit rows: three stages of 16 KB each);
+// larger k takes the big buffer at two CTAs per SM.  32-bit rows have 32 KB tiles and two stages.
 constexpr int CS_CAP_SMALL = 2048, CS_CAP_LARGE = 4096;    // candidate keys held in shared memory
 constexpr int CS_K_SMALL = 256;                            // largest k served by the small shape
 constexpr int CS_BINS = 4096;        // histogram bins above the first tile's bound; the last one is open-ended

@@ -98,8 +98,9 @@ __global__ void __launch_bounds__(THREADS) edge_finish_kernel(VerifyArgs a) {
             // every q carries a relative error of at most GUARD_Z in the fast path, so every prefix
             // and the total are off by at most GUARD_Z * Q
             const double E = PRECISE ? 0.0 : 2.0 * GUARD_Z * Q;
-            // residual total too close to zero to say whether the fallback applies: decide in double
-            if (!PRECISE && Rres <= E && tid == 0) sflag = 1;
+            // residual total too close to zero to say whether the fallback applies, or so small that the
+            // normaliser's error would show in the reported mass: decide and report in double
+            if (!PRECISE && (Rres <= E || Rres < RESID_EXACT_BELOW * Q) && tid == 0) sflag = 1;
             const bool fallback = !(Rres > E);
             if (fallback) {
                 // Q covers every transmitted component: draw from the components themselves

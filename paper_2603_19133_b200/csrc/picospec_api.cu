@@ -429,6 +429,27 @@ int picospec_profile_read(picospec_ctx* ctx, int kind, float* total_ms_out, int*
     return PICOSPEC_OK;
 }
 
+int picospec_profile_samples(picospec_ctx* ctx, int kind, float* ms_out, int capacity, int* n_out, void* cuda_stream) {
+    if (!ctx || kind < 0 || kind >= PICOSPEC_PROF_KINDS || !ms_out || !n_out || capacity < 0) return PICOSPEC_EINVAL;
+    DeviceGuard g(ctx->device);
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)cuda_stream);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    const long long total = ctx->prof_count[kind];
+    long long n = total < PROF_RING ? total : PROF_RING;
+    if (n > capacity) n = capacity;
+    // the ring holds the last PROF_RING brackets; the newest n of them, oldest first
+    for (long long i = 0; i < n; ++i) {
+        const long long slot = (total - n + i) % PROF_RING;
+        float ms = 0.f;
+        e = cudaEventElapsedTime(&ms, ctx->prof_ev[kind][slot][0], ctx->prof_ev[kind][slot][1]);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        ms_out[i] = ms;
+    }
+    *n_out = (int)n;
+    ctx->prof_count[kind] = 0;
+    return PICOSPEC_OK;
+}
+
 int picospec_status(picospec_ctx* ctx, int* device_status_out, long long* slow_path_rows_out, int clear,
                     void* cuda_stream) {
     if (!ctx) return PICOSPEC_EINVAL;

@@ -44,9 +44,11 @@ struct VerifyArgs {
 };
 
 // ---------------------------------------------------------------------------------------------
-// Streaming pass: one warp per 1024-entry chunk, software-pipelined over two register buffers.
+// Streaming pass, direct variant (rows that are not 16-byte aligned): one warp per 1024-entry
+// chunk, read straight from global memory and software-pipelined over two register buffers.
 // Per chunk: exact maximum logit and the fp32 sum of 2^((l - max) * log2e / T).
 // ---------------------------------------------------------------------------------------------
+// one (row, chunk) item of the direct variant
 template <typename T> struct ItemMeta {
     const T* row;
     int v0;
@@ -262,7 +264,7 @@ struct FinishShared {
     double Zraw[MAX_G1];  // the same sum on the streaming pass's own scale (fast path)
     float mx[MAX_G1];
     int bad;
-    int acc[MAX_G1], amb[MAX_G1], bord[MAX_G1];
+    int acc[MAX_G1], amb[MAX_G1], bord[MAX_G1], small[MAX_G1];
     double warp_tot[WARPS];
     double red[WARPS];
     int tok, last, flag;
@@ -470,6 +472,9 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                         sh.bord[i] = bord;
                         double R = 1.0 - smin;
                         if (R < 0.0) R = 0.0;
+                        // 1 - sum min(p, q~) inherits the absolute error of the fp32-accumulated
+                        // normaliser: a small residual mass is reported from the exact sums instead
+                        sh.small[i] = !PRECISE && R < RESID_EXACT_BELOW;
                         a.p_draft[ri] = (float)px;
                         a.resid_mass[ri] = (float)R;
                     }
@@ -497,6 +502,8 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 flagged |= sh.amb[i] != 0;
                 nborder += sh.bord[i];
             }
+            if (!PRECISE)
+                for (int i = lo; i < hi; ++i) flagged |= sh.small[i] != 0;
         }
 
         // ---- 4. residual / bonus sample --------------------------------------------------
@@ -610,7 +617,9 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 Rtot = sh.Rtot;
                 if (!use_resid) break;
                 // the residual may vanish (q~ >= p everywhere): then the draw is from p itself
-                const double tiny = PRECISE ? 1e-12 : 4.0 * GUARD_Z;
+                const double tiny = PRECISE ? RESID_ZERO_BELOW : 4.0 * GUARD_Z;
+                // (a reported mass this small would show the normaliser's error: exact sums instead)
+                if (!PRECISE && a.mass && Rtot < RESID_EXACT_BELOW && tid == 0) sh.flag = 1;
                 if (Rtot > tiny) break;
                 if (!PRECISE) {
                     if (tid == 0) sh.flag = 1;   // too close to zero to call in fp32
@@ -708,7 +717,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 } else if (flagged) {
                     // Which rows need exact sums: an ambiguous accept test can move the first
                     // rejection anywhere from its position on, so every row from there; an ambiguous
-                    // draw needs the sampled row only.
+                    // draw needs the sampled row only; a small residual mass its own row.
                     unsigned long long nd = 0ull;
                     int nrows = 0;
                     bool draw_only_flag = false;
@@ -720,9 +729,11 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                         const int last = rejected ? alen : hi - 1;
                         for (int i = lo; i <= last && first_amb < 0; ++i)
                             if (sh.amb[i]) first_amb = i;
-                        draw_only_flag = first_amb < 0;
+                        bool any_small = false;
+                        for (int i = lo; i < hi; ++i) any_small |= sh.small[i] != 0;
+                        draw_only_flag = first_amb < 0 && !any_small;
                         for (int i = lo; i < row_hi; ++i) {
-                            const bool nr = i >= 64 || (first_amb >= 0 && i >= first_amb) ||
+                            const bool nr = i >= 64 || (first_amb >= 0 && i >= first_amb) || (i < hi && sh.small[i]) ||
                                             (sh.flag && want_token && decided && i == alen);
                             if (nr) {
                                 if (i < 64) nd |= 1ull << i;

@@ -1,5 +1,5 @@
-// Wire format of the sparse rows (Sec. 3.3: the verifier sends "(id, prob)" pairs -- under 100
-// bytes for K = 10 -- laid out so that the receiver can view the arrays in place).  One message:
+// Wire format of the sparse rows (Sec. 3.3: the verifier sends pairs of vocabulary id and
+// probability -- under 100 bytes for K = 10 -- laid out so that the receiver can view the arrays in place).  One message:
 //     0   u32  magic 0x31505350 ("PSP1")
 //     4   u32  R, the number of rows
 //     8   u16  K, the capacity of a dense row
@@ -36,8 +36,9 @@ __host__ __device__ __forceinline__ long long wire_bytes(long long rows, long lo
     return 16 + wire_pad4(2 * rows) + 4 * entries + wire_pad4((prob_type == 0 ? 4 : 2) * entries);
 }
 
-// One CTA: exclusive scan of max(count, 0) over the rows; header and counts (pack), or header and
-// count checks (unpack).
+// One CTA: exclusive scan of max(count, 0) over the rows; then the header (pack: only once the
+// message is known to fit the caller's buffer, so that a buffer that is too small is never written),
+// or the header and count checks (unpack).  The packed counts are written by the move kernel.
 template <bool PACK>
 __global__ void __launch_bounds__(THREADS) wire_scan_kernel(WireArgs a) {
     __shared__ int warp_tot[WARPS];
@@ -72,7 +73,6 @@ __global__ void __launch_bounds__(THREADS) wire_scan_kernel(WireArgs a) {
                 bad_s = 1;          // pack: the row travels as invalid; unpack: the message is refused
                 c = -1;
             }
-            if (PACK) reinterpret_cast<short*>(a.buf + 16)[r] = (short)c;
         }
         const int n = c > 0 ? c : 0;
         int incl = n;
@@ -133,9 +133,11 @@ __global__ void __launch_bounds__(THREADS) wire_move_kernel(WireArgs a) {
         float* qp = a.q_prob + (long long)r * a.K;
         if (PACK) {
             if (N < 0) continue;                              // the message did not fit: nothing is written
-            const int c = a.q_count[r];
-            const int n = (c > 0 && c <= a.K) ? c : 0;
+            int c = a.q_count[r];
+            if (c > a.K || c < -1) c = -1;                    // the row travels as invalid
+            const int n = c > 0 ? c : 0;
             const int o = a.offsets[r];
+            if (lane == 0) reinterpret_cast<short*>(a.buf + 16)[r] = (short)c;
             for (int j = lane; j < n; j += 32) {
                 ids[o + j] = qi[j];
                 if (ptype == 0) reinterpret_cast<float*>(probs)[o + j] = qp[j];

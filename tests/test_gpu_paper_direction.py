@@ -56,7 +56,7 @@ def _flow(ps, w, k, seed, pos=None):
         st2, slow = ctx.status(clear=True)
         assert np.array_equal(_np(g_tok), o_tok), "token"
         ok = o_tok >= 0
-        np.testing.assert_allclose(_np(g_mass)[ok], o_mass[ok], rtol=RTOL, atol=3e-7)
+        np.testing.assert_allclose(_np(g_mass)[ok], o_mass[ok], rtol=RTOL, atol=1e-12)
         return {"status": st | st2, "slow": slow, "o_tok": o_tok, "o_pc": o_pc}
     finally:
         ctx.close()

@@ -14,7 +14,7 @@ import oracle
 pytestmark = pytest.mark.gpu
 
 RTOL = 1e-5
-ATOL_MASS = 3e-7
+ATOL_MASS = 1e-12    # resolution of 1 - sum min(p, q~) in double precision
 
 
 @pytest.fixture(scope="module")

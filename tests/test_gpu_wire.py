@@ -106,7 +106,14 @@ def test_message_that_does_not_fit_and_bad_counts(ps):
         small = torch.full((64,), 0xAB, dtype=torch.uint8, device="cuda")
         buf, nbytes = ctx.wire_pack(_cuda(qi), _cuda(qp), _cuda(qc), buf=small)
         assert int(nbytes.item()) == -1 and ctx.status(clear=True)[0] == 4
-        assert bool((small[16 + 2 * R + 2:] == 0xAB).all())     # no entries were written
+        assert bool((small == 0xAB).all())                      # buf holds no message: nothing was written
+        # a buffer that ends inside the counts (16 + 2 R bytes would be needed for them alone), with a
+        # guard pattern behind it in the same allocation
+        guard = torch.full((256,), 0xCD, dtype=torch.uint8, device="cuda")
+        assert 20 < 16 + 2 * R
+        buf, nbytes = ctx.wire_pack(_cuda(qi), _cuda(qp), _cuda(qc), buf=guard[:20])
+        assert int(nbytes.item()) == -1 and ctx.status(clear=True)[0] == 4
+        assert bool((guard == 0xCD).all())
         qc2 = qc.copy().reshape(-1)
         qc2[0] = K + 1                                          # a count beyond the capacity
         buf, nbytes = ctx.wire_pack(_cuda(qi), _cuda(qp), _cuda(qc2))

@@ -141,6 +141,37 @@ def test_sequence_sharding_world_size_2_gloo(tmp_path):
     assert "SHARD_OK" in run.stdout
 
 
+def test_bench_starts_its_own_ranks_for_more_than_one_gpu():
+    # `bench.py --gpus 2` without a torchrun environment starts two ranks of itself; the reference arm
+    # needs no GPU (rank 0 alone times the oracle, the other rank leaves without work), so the launcher
+    # path runs here as it is
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE")}
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--steps", "1",
+           "--warmup", "0", "--workload", "config1", "--ref-sample", "1"]
+    run = subprocess.run(cmd, capture_output=True, text=True, timeout=600, env=env)
+    assert run.returncode == 0, run.stdout[-2000:] + run.stderr[-2000:]
+    lines = [ln for ln in run.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                      # one JSON line, from rank 0
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["ranks_launched"] == 2
+    assert line["config"]["parallelism"].startswith("dp2")
+
+
+def test_bench_reads_ncu_traffic_only_for_unchanged_kernels(tmp_path, monkeypatch):
+    sys.path.insert(0, ROOT)
+    import bench
+    h = bench.source_hash(["verify_kernels.cuh"])
+    prof = tmp_path / "profiles"
+    prof.mkdir()
+    (prof / "a.md").write_text(f"x\nbench-traffic: kernel=k1 workload=config4 bytes=123 sources=verify_kernels.cuh hash={h}\n"
+                               "bench-traffic: kernel=k2 workload=config4 bytes=5 sources=verify_kernels.cuh hash=000000000000\n")
+    monkeypatch.setattr(bench, "ROOT", str(tmp_path))
+    assert bench.ncu_traffic("config4", "k1") == 123
+    assert bench.ncu_traffic("config4", "k2") is None        # the kernel changed since the capture
+    assert bench.ncu_traffic("config3", "k1") is None
+
+
 def test_throughput_calculator_matches_the_term_by_term_oracle():
     # the product's closed forms (Sec. 3.4, Eqs. 5-10) against the oracle's sums and case analysis
     from paper_2603_19133_b200 import perf_model as pm

@@ -50,6 +50,8 @@ MUTANTS = [
     ("range_ignores_gamma", "long g = gamma ? gamma[b] : G;", "long g = G;"),
     ("range_ignores_state", "if (state_in && state_in[b] == 0) {", "if (0) {"),
     ("range_reads_later_rows", "long hi = g < r1 ? g : r1;", "long hi = g;"),
+    ("vanished_residual_threshold_too_high", "if (R > PSO_RESID_ZERO) tok", "if (R > 1e-9) tok"),
+    ("vanished_residual_never", "if (R > PSO_RESID_ZERO) tok", "if (R > 0.0) tok"),
     ("edge_no_fallback", "if (!(R > 0.0)) {\n                    R = 0.0;", "if (0) {\n                    R = 0.0;"),
 ]
 

@@ -291,6 +291,30 @@ def test_zero_residual_falls_back_to_p():
     assert t_res[0] == t_p[0]
 
 
+def test_residual_counts_as_vanished_up_to_1e_12_of_the_row():
+    # Sec. 3.3's norm(max(0, P - Q)) is undefined for a vanishing residual; the reading is: total
+    # residual mass <= 1e-12 of the row -> draw from P itself.  Three entries: q~ = (0.5, 0.5) covers
+    # the first two (each p there is a little below 0.5), so the residual is p_2 alone.
+    T = np.ones(1, np.float32)
+    qi = np.array([[[0, 1]]], np.int32)
+    qp = np.array([[[0.5, 0.5]]], np.float32)
+    qc = np.array([[2]], np.int32)
+    pos = np.zeros(1, np.int32)
+    u = np.array([[0.2, 0.3]], np.float32)
+    for gap, vanished in ((23.0, False), (32.0, True)):
+        lt = np.zeros((1, 2, 3), np.float32)
+        lt[0, 0, 2] = -gap
+        p2 = np.exp(-gap) / (2.0 + np.exp(-gap))
+        assert (p2 <= 1e-12) == vanished and p2 > 0
+        tok, mass = oracle.residual_sample(lt, T, pos, qi, qp, qc, u)
+        if vanished:
+            # the draw is from p: u1 = 0.2 lands in the single chunk, u2 = 0.3 < p_0 picks entry 0
+            assert tok[0] == 0 and abs(mass[0] - 1.0) < 1e-12
+        else:
+            # the only entry with residual weight, whatever the uniforms
+            assert tok[0] == 2 and abs(mass[0] / p2 - 1.0) < 1e-9
+
+
 # ---------------------------------------------------------------------------------------
 # whole method: output law equals the target distribution (Sec. 2.1 / Sec. 3.3 claim)
 # ---------------------------------------------------------------------------------------

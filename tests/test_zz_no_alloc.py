@@ -7,20 +7,23 @@ either (creating one allocates the workspace).  For them the library keeps a fix
 its device image and exposes picospec_verify_static, which takes only the caller's own buffers.
 
 The test calls it through the C-ABI twice in a row (the second call finds the first call's leftovers
-in the shared workspace) and checks every output against picospec_verify on the same inputs:
-integers bit-exact, probabilities and residual masses to the tolerance of the parity tests.  It also
-checks that a problem larger than the fixed workspace is rejected.  This file is collected last so
-that a run stopping at the first failure has already run every other test; it also passes alone."""
+in the shared workspace) and checks every output against picospec_verify on the same inputs and
+against the CPU oracle: integers bit-exact, probabilities and residual masses to the tolerance of the
+parity tests.  It checks the entry point's own claim as well: the amount of free device memory is
+the same after a call as before it.  And it checks that a problem larger than the fixed workspace is
+rejected.  This file is collected last so that a run stopping at the first failure has already run
+every other test; it also passes alone."""
 import numpy as np
 import pytest
 import torch
 
 import gen
+import oracle
 
 pytestmark = pytest.mark.gpu
 
 RTOL = 1e-5
-ATOL_MASS = 3e-7
+ATOL_MASS = 1e-12    # resolution of 1 - sum min(p, q~) in double precision
 
 
 def _alloc_out(B, G, dev):
@@ -42,6 +45,20 @@ def _same(a, b):
                                atol=ATOL_MASS)
 
 
+def _np(t):
+    return t.detach().float().cpu().numpy() if t.is_floating_point() else t.detach().cpu().numpy()
+
+
+def _same_as_oracle(out, inp, tok, qi, qp, qc):
+    o = oracle.verify(_np(inp["target_logits"]), _np(inp["temperature"]), _np(tok), _np(qi), _np(qp), _np(qc),
+                      _np(inp["u_accept"]), _np(inp["u_resample"]), nthreads=oracle.cores())
+    assert np.array_equal(_np(out["accept_len"]), o["accept_len"])
+    assert np.array_equal(_np(out["token"]), o["token"])
+    assert int(out["borderline_count"].item()) == o["borderline_count"]
+    np.testing.assert_allclose(_np(out["p_draft"]), o["p_draft"], rtol=RTOL, atol=0)
+    np.testing.assert_allclose(_np(out["resid_mass"]), o["resid_mass"], rtol=RTOL, atol=ATOL_MASS)
+
+
 @pytest.mark.parametrize("name,B", [("config2", 8), ("config3", 28), ("config1", 1)])
 def test_verify_static_matches_verify_on_two_calls_in_a_row(name, B):
     import paper_2603_19133_b200 as ps
@@ -61,10 +78,17 @@ def test_verify_static_matches_verify_on_two_calls_in_a_row(name, B):
             st, slow = ctx.status(clear=True)
             assert st == 0
             out = _alloc_out(w.B, w.G, dev)           # the caller's buffers, made before the call
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             ps.verify_static(inp["target_logits"], inp["temperature"], tok, qi, qp, qc, inp["u_accept"],
                              inp["u_resample"], out)
             torch.cuda.synchronize()
+            # nothing was allocated, by the library or through torch (on the first call of a process the
+            # driver may still load the kernels' code, so the claim is checked from the second call on)
+            if call > 0:
+                assert torch.cuda.mem_get_info()[0] == free_before
             _same(out, ref)
+            _same_as_oracle(out, inp, tok, qi, qp, qc)
             assert int(out["device_status"].item()) == 0, f"call {call}"
             assert int(out["slow_rows"].item()) == slow, f"call {call}"
     finally:

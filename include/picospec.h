@@ -74,6 +74,15 @@ PICOSPEC_API const char* picospec_strerror(int err);
 /* cudaError_t of the last failing CUDA call made through this context (0 if none). */
 PICOSPEC_API int picospec_last_cuda_error(const picospec_ctx* ctx);
 
+/* The staged kernels wait for their asynchronous copies with a time limit (two seconds by default):
+ * a wait that runs out sets PICOSPEC_ST_INTERNAL, the waiting warp stops computing, and the outputs
+ * of that call -- and of every later call until the status word is cleared -- are marked invalid
+ * (-1); the kernel still waits for every copy it issued before it ends.  This call lowers the limit
+ * for later calls on the context (values above two seconds are clamped to it); it exists so that
+ * the give-up path can be exercised: with a limit of 0 the first wait that is not already complete
+ * gives up.  The paper has no counterpart. */
+PICOSPEC_API int picospec_wait_limit(picospec_ctx* ctx, unsigned long long limit_ns);
+
 /* Optional per-kernel timing, for benchmarks.  level 0 = off (default), 1 = bracket the two
  * streaming kernels (one per hot call) with CUDA events on the caller's stream, 2 = bracket every
  * kernel group.  Enabling creates the events (host objects; no device memory) and resets the

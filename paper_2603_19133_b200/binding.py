@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.picospec_wire_unpack.restype = c_int
         L.picospec_profile_samples.argtypes = [vp, c_int, ctypes.POINTER(c_f), c_int, ctypes.POINTER(c_int), vp]
         L.picospec_profile_samples.restype = c_int
+        L.picospec_wait_limit.argtypes = [vp, ctypes.c_ulonglong]
+        L.picospec_wait_limit.restype = c_int
         L.picospec_counters.argtypes = [vp, ctypes.POINTER(c_ll), c_int, vp]
         L.picospec_counters.restype = c_int
         L.picospec_verify_static.argtypes = [vp, c_int, c_int, c_int, c_int, c_ll, vp, vp, vp, vp, vp, c_int,
@@ -195,6 +197,10 @@ class Context:
         out = (ctypes.c_longlong * 2)()
         _check(lib().picospec_counters(self._h, out, int(clear), _stream()), "picospec_counters")
         return int(out[0]), int(out[1])
+
+    def wait_limit(self, limit_ns: int):
+        """picospec_wait_limit: the first time limit of the staged kernels' waits, for later calls."""
+        _check(lib().picospec_wait_limit(self._h, int(limit_ns)), "picospec_wait_limit")
 
     def profile_enable(self, level: int, every: int = 1):
         """0 = off, 1 = time the two streaming kernels, 2 = time every kernel group; only every

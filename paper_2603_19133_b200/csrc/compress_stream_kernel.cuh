@@ -37,6 +37,8 @@
 // draft draw).
 #pragma once
 #include "compress_kernels.cuh"
+
+
 #include "stream_pipeline.cuh"
 
 namespace picospec {
@@ -87,10 +89,22 @@ struct CsShared {
     unsigned top_key;   // largest orderable logit of the first tile
     int overflow;       // a region ran out of room: the row goes to the redo list
     int nan;
-    int abort;          // a bounded wait ran out somewhere in the CTA
-    int m;              // survivors written at the end of the row
+    int m;              // survivors written at the end of the piece
     double wsum[WARPS];
 };
+// state of the CTA that outlives a piece
+struct CsCta {
+    int abort;          // a bounded wait ran out somewhere in the CTA
+    int wcnt[WARPS];    // per warp: entries in its region (the slot counter its lanes draw from)
+};
+__device__ __forceinline__ void cs_reset(CsShared& cs) {
+    cs.thr_key = 0u;
+    cs.thr0_key = 0xffffffffu;
+    cs.top_key = 0u;
+    cs.overflow = 0;
+    cs.nan = 0;
+    cs.m = 0;
+}
 
 // threshold (a float) of an orderable key; keys below 0x00800000 are -inf and the negative NaN patterns
 __device__ __forceinline__ float thr_of_key(unsigned key) {
@@ -175,6 +189,13 @@ __device__ __forceinline__ unsigned warp_kth_key(const unsigned (&key)[16], int 
 template <typename T>
 __device__ __forceinline__ unsigned first_tile_key(const ChunkRegs<T>& regs, int g, int need) {
     unsigned key[16];
+    if (g == ChunkRegs<T>::VEC) {
+        // groups = the lane's 16-byte vectors: their maxima come packed
+        constexpr int NV = ChunkRegs<T>::NVEC;
+#pragma unroll
+        for (int j = 0; j < NV; ++j) key[j] = orderable(regs.vec_max(j)) >> 16;
+        return warp_kth_key<NV>(key, need);
+    }
     pair_keys(regs, key);
     if (g == 2) return warp_kth_key<16>(key, need);
 #pragma unroll
@@ -211,8 +232,9 @@ __device__ __forceinline__ void hist_add(unsigned* hist, int bin) {
     atomicAdd(&hist[CS_BINS / 2 + (bin >> 5)], 1u);
 }
 
-// One warp: raise thr to the lower edge of the highest bin whose suffix count reaches k.
-__device__ __forceinline__ void refresh_threshold(const unsigned* hist, CsShared& cs, int k, int lane) {
+// One warp: the highest bin whose suffix count (itself and every bin above it) reaches k, or -1 if
+// fewer than k values have been counted.
+__device__ __forceinline__ int kth_bin(const unsigned* hist, int k, int lane) {
     // level 1: lane l owns super-bins 4l .. 4l+3 (super-bin s covers bins 32 s .. 32 s + 31)
     const uint4 sv = *reinterpret_cast<const uint4*>(&hist[CS_BINS / 2 + 4 * lane]);
     const unsigned own = sv.x + sv.y + sv.z + sv.w;
@@ -223,7 +245,7 @@ __device__ __forceinline__ void refresh_threshold(const unsigned* hist, CsShared
         if (lane + d < 32) suf += y;
     }
     const unsigned hit = __ballot_sync(0xffffffffu, suf >= (unsigned)k);
-    if (!hit) return;               // fewer than k counted so far
+    if (!hit) return -1;            // fewer than k counted so far
     const int L = 31 - __clz(hit);  // highest lane whose suffix reaches k
     unsigned above = __shfl_sync(0xffffffffu, suf - own, L);      // count strictly above lane L's super-bins
     const uint4 lv = make_uint4(__shfl_sync(0xffffffffu, sv.x, L), __shfl_sync(0xffffffffu, sv.y, L),
@@ -249,8 +271,13 @@ __device__ __forceinline__ void refresh_threshold(const unsigned* hist, CsShared
         if (lane + d < 32) bs += y;
     }
     const unsigned hit2 = __ballot_sync(0xffffffffu, above + bs >= (unsigned)k);
-    const int found = hit2 ? 32 * s + (31 - __clz(hit2)) : 32 * s;
-    if (lane == 0) {
+    return hit2 ? 32 * s + (31 - __clz(hit2)) : 32 * s;
+}
+
+// One warp: raise thr to the lower edge of the highest bin whose suffix count reaches k.
+__device__ __forceinline__ void refresh_threshold(const unsigned* hist, CsShared& cs, int k, int lane) {
+    const int found = kth_bin(hist, k, lane);
+    if (found >= 0 && lane == 0) {
         const int g0 = bin_coord(*(volatile unsigned*)&cs.thr0_key >> 16);
         atomicMax(&cs.thr_key, coord_code(g0 + found) << 16);
     }
@@ -277,16 +304,111 @@ __device__ __noinline__ void refresh_bound(int hist_off, CsShared* cs, int k_eff
     refresh_threshold(reinterpret_cast<const unsigned*>(dyn + hist_off), *cs, k_eff, threadIdx.x & 31);
 }
 // Region nearly full: bring the bound up to date and drop what fell below it (one warp; out of line).
-__device__ __noinline__ int maintain_region(int wcount, int region_off, int hist_off, CsShared* cs, int k_eff) {
+// The warp's slot counter follows.
+__device__ __noinline__ int maintain_region(int wcount, int region_off, int hist_off, CsShared* cs, int* wcnt, int k_eff) {
     extern __shared__ __align__(1024) unsigned char dyn[];
     const int lane = threadIdx.x & 31;
     refresh_threshold(reinterpret_cast<const unsigned*>(dyn + hist_off), *cs, k_eff, lane);
     __syncwarp();
-    return compact_region(reinterpret_cast<u64*>(dyn + region_off), wcount, *(volatile unsigned*)&cs->thr_key, lane);
+    const int n = compact_region(reinterpret_cast<u64*>(dyn + region_off), wcount, *(volatile unsigned*)&cs->thr_key, lane);
+    if (lane == 0) *wcnt = n;
+    __syncwarp();
+    return n;
+}
+
+// ---- how the rows of a call are dealt to the CTAs of the filter kernel ----------------------------
+// With rows = q * grid + rem, CTA b first takes the q whole rows b, b + grid, ... (so that at any time
+// the CTAs read one window of memory that moves forward, as a copy would).  The rem rows that
+// are left would keep only some of the CTAs busy for a whole row's time, so each of them is cut into
+// `split` pieces of consecutive tiles and the rem * split pieces are dealt round-robin: piece n goes
+// to CTA n % grid.  A piece is filtered on its own: it keeps a bound that at least k of ITS elements
+// reach, which is a valid bound for the row, and leaves its survivors in its own scratch area (whole
+// row r: area r; tail piece n: area rows + n).  The finish kernel puts the pieces of a row together.
+// No piece starts at a row's last tile when that tile is ragged (the first tile of a piece must be a
+// full one).
+struct FilterPlan {
+    int tiles_per_row;
+    int ragged_last;        // the last tile of a row holds fewer than TILE_CHUNKS full chunks
+    int grid;               // CTAs of the filter kernel
+    int rows;
+    int q;                  // whole rows per CTA
+    int rem;                // rows dealt in pieces: rows q * grid .. rows - 1
+    int split;              // pieces per such row
+};
+// first tile of piece p (0 .. split) of a split row
+__host__ __device__ __forceinline__ int plan_piece_tile(const FilterPlan& p, int piece) {
+    int c = p.tiles_per_row * piece / p.split;
+    if (p.ragged_last && p.tiles_per_row > 1 && c < p.tiles_per_row && c == p.tiles_per_row - 1) --c;
+    return c;
+}
+// The k-th unit of work of CTA b: a whole row or a piece of a tail row.  false: no more work.
+struct FilterPiece {
+    int row, tile0, tile1, area;
+};
+__host__ __device__ __forceinline__ bool plan_piece(const FilterPlan& p, int b, int k, FilterPiece& out) {
+    if (k < p.q) {
+        out.row = k * p.grid + b;      // the CTAs advance through memory side by side
+        out.tile0 = 0;
+        out.tile1 = p.tiles_per_row;
+        out.area = out.row;
+        return true;
+    }
+    const long long n = (long long)b + (long long)(k - p.q) * p.grid;
+    if (n >= (long long)p.rem * p.split) return false;
+    const int j = (int)(n / p.split), pc = (int)(n - (long long)j * p.split);
+    out.row = p.q * p.grid + j;
+    out.tile0 = plan_piece_tile(p, pc);
+    out.tile1 = plan_piece_tile(p, pc + 1);
+    out.area = p.rows + (int)n;
+    return true;        // (tile0 == tile1: an empty piece, skipped by everyone)
+}
+// Host side: the plan for `rows` rows on `slots` resident CTAs.  Rows are cut only when a CTA gets at most
+// one whole row (few rows per CTA: the remainder decides the kernel's length); the split is then the one
+// that shortens the tail most among those that keep a piece at least two tiles long and the number of
+// pieces within 2 * grid (the scratch areas are sized for that).
+inline FilterPlan make_filter_plan(int rows, int tiles_per_row, bool ragged_last, long long slots) {
+    FilterPlan p;
+    p.tiles_per_row = tiles_per_row;
+    p.ragged_last = ragged_last ? 1 : 0;
+    p.rows = rows;
+    long long g = slots < 1 ? 1 : slots;
+    const long long most = (long long)rows * (tiles_per_row >= 2 ? tiles_per_row / 2 : 1);   // pieces of two tiles
+    if (g > most) g = most;
+    if (g < 1) g = 1;
+    p.grid = (int)g;
+    p.q = (int)(rows / g);
+    p.rem = (int)(rows - (long long)p.q * g);
+    p.split = 1;
+    // Pieces pay the per-piece work (first-tile bound, hand-over) again; that is worth it only while
+    // the remainder is a large part of what a CTA does.
+    if (p.rem > 0 && p.q <= 1) {
+        double best = 1e9;
+        const int smax = tiles_per_row >= 2 ? tiles_per_row / 2 : 1;
+        for (int sp = 1; sp <= 8 && sp <= smax && (long long)p.rem * sp <= 2 * g; ++sp) {
+            const long long per_cta = ((long long)p.rem * sp + g - 1) / g;      // pieces the busiest CTA gets
+            const double cost = (double)per_cta / sp;
+            if (cost < best - 1e-9) {
+                best = cost;
+                p.split = sp;
+            }
+        }
+    }
+    return p;
+}
+
+// First-tile bound of one warp when it needs at most 32 elements (k <= 256): the lanes form at
+// least `need` groups of `group_lanes` lanes (a power of two); every group's largest value is
+// reached by one element of the group, so the smallest of the group maxima is reached by at least
+// `need` elements of the warp's chunk.  Returns its 16-bit orderable code (rounded down).
+__device__ __forceinline__ unsigned first_tile_key_groups(float lane_max, int group_lanes) {
+    unsigned key = orderable(lane_max) >> 16;
+    for (int d = 1; d < group_lanes; d <<= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, d));
+    return __reduce_min_sync(0xffffffffu, key);
 }
 
 template <typename T, bool STATS, bool SMALL>
-__global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compress_filter_kernel(CompressArgs a, int tiles_per_row) {
+__global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS)
+compress_filter_kernel(CompressArgs a, FilterPlan plan, unsigned long long wait_limit_ns) {
     extern __shared__ __align__(1024) unsigned char dyn[];
     typedef CsGeom<T, SMALL> Geom;
     constexpr int STAGES = Geom::STAGES;
@@ -297,10 +419,12 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
     u64* cand = reinterpret_cast<u64*>(dyn + Geom::STAGE_BYTES);
     unsigned* hist = reinterpret_cast<unsigned*>(cand + CS_CAND_CAP);          // bins, then super-bins
     __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES];
-    __shared__ CsShared cs;
+    // Two copies of the per-piece state, used in turn: the copy of the piece that has just ended is
+    // reset by one thread while the other warps already start on the next piece.
+    __shared__ CsShared css[2];
+    __shared__ CsCta cta;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int rows = a.B * a.G;
     int k_eff = a.top_k > 0 ? a.top_k : a.k_max;
     if (k_eff > a.k_max) k_eff = a.k_max;
     if (k_eff > a.V) k_eff = a.V;
@@ -312,14 +436,11 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
             mbar_init(&empty[s], WARPS);
         }
         mbar_init_fence();
-        cs.thr_key = 0u;
-        cs.thr0_key = 0xffffffffu;
-        cs.top_key = 0u;
-        cs.overflow = 0;
-        cs.nan = 0;
-        cs.abort = 0;
-        cs.m = 0;
+        cs_reset(css[0]);
+        cs_reset(css[1]);
+        cta.abort = 0;
     }
+    if (tid < WARPS) cta.wcnt[tid] = 0;
     for (int i = tid; i < CS_HIST_WORDS; i += STREAM_THREADS) hist[i] = 0u;
     grid_dependency_sync();
     if (tid == 0 && blockIdx.x == 0) {
@@ -329,20 +450,22 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
     __syncthreads();
 
     if (warp == WARPS) {
-        // ---- producer: every tile of every row of this CTA, in order -------------------------
+        // ---- producer: every tile of every piece of this CTA, in order ---------------------------
         if (lane != 0) return;
         const uint64_t pol = l2_evict_first_policy();
         uint32_t i = 0;
-        for (int row = blockIdx.x; row < rows; row += gridDim.x) {
-            const long long srow = source_row(a, row);
-            const bool valid = temp_ok(a.temperature[row / a.G]) && srow >= 0;
+        FilterPiece pc;
+        for (int k = 0; plan_piece(plan, blockIdx.x, k, pc); ++k) {
+            const long long srow = source_row(a, pc.row);
+            const bool valid = temp_ok(a.temperature[pc.row / a.G]) && srow >= 0;
             const T* rowp = reinterpret_cast<const T*>(a.logits) + (srow < 0 ? 0 : srow) * a.row_stride;
-            for (int ti = 0; ti < tiles_per_row; ++ti, ++i) {
+            for (int ti = pc.tile0; ti < pc.tile1; ++ti, ++i) {
                 const int s = (int)(i % STAGES);
                 const uint32_t round = i / STAGES;
-                if (round > 0 && !mbar_wait(&empty[s], (round - 1) & 1)) {
-                    atomicOr(a.status, ST_INTERNAL);
-                    return;
+                if (round > 0) {
+                    const int wr = mbar_wait_twice(&empty[s], (round - 1) & 1, wait_limit_ns);
+                    if (wr != WAIT_OK) atomicOr(a.status, ST_INTERNAL);
+                    if (wr == WAIT_LOST) return;      // nothing more is issued
                 }
                 if (valid) {
                     const int v0 = ti * TILE_CHUNKS * CHUNK;
@@ -360,55 +483,69 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
 
     // ---- workers ------------------------------------------------------------------------------
     u64* region = cand + warp * CS_REGION;
-    const unsigned lt_mask = (1u << lane) - 1u;
     const int region_off = (int)(reinterpret_cast<unsigned char*>(region) - dyn);
     const int hist_off = (int)(reinterpret_cast<unsigned char*>(hist) - dyn);
-    // first-tile bound: groups of g elements, at least 4 k groups in the tile
+    // first-tile bound.  k <= 128 (every warp needs at most 16 elements): from the lane maxima, over
+    // groups of two or more lanes.  Larger k: the exact need-th largest maximum of groups of g elements,
+    // at least 4 k groups in the tile (cheaper bounds from lane maxima or lane pairs let 10 to 25 % of
+    // a tile pass: the extra candidates cost more than the search).
+    const int need = (k_eff + WARPS - 1) / WARPS;
+    int group_lanes = 1;
+    while (2 * group_lanes * need <= 32) group_lanes <<= 1;
     int g = VEC;
     while (g > 2 && (TILE_CHUNKS * CHUNK) / g < 4 * k_eff) g >>= 1;
-    const int need = (k_eff + WARPS - 1) / WARPS;
 
-    bool dead = false;      // this warp stopped waiting on copies; it still joins every barrier
+    bool dead = false;      // a wait ran out: this warp computes no more, but takes every tile and joins every barrier
+    bool lost = false;      // a wait did not complete at all: the warp stops waiting as well
     uint32_t i = 0;
-    for (int row = blockIdx.x; row < rows; row += gridDim.x) {
-        const int b = row / a.G;
-        const float Tb = a.temperature[b];
+    int parity = 0;         // which copy of the per-piece state this piece uses
+    FilterPiece pc;
+    for (int k = 0; plan_piece(plan, blockIdx.x, k, pc); ++k) {
+        if (pc.tile0 >= pc.tile1) continue;
+        CsShared& cs = css[parity];
+        parity ^= 1;
+        const int row = pc.row;
+        const float Tb = a.temperature[row / a.G];
         const bool in_range = source_row(a, row) >= 0;
         const bool valid = temp_ok(Tb) && in_range;
         const float c32 = temp_scale(Tb);
         float ref_off = 0.f, acc = 0.f;
-        int wcount = 0;             // candidates in this warp's region
+        int wcount = 0;             // candidates in this warp's region (cs.wcnt[warp] holds the same number)
         int g0 = 0;                 // bin coordinate of the first tile's bound: origin of the histogram
-        bool full_region = false;   // the region ran out of room (the row goes to the redo list)
+        bool full_region = false;   // the region ran out of room (the row goes to the direct kernel)
 
-        for (int ti = 0; ti < tiles_per_row; ++ti, ++i) {
+        for (int ti = pc.tile0; ti < pc.tile1; ++ti, ++i) {
             const int s = (int)(i % STAGES);
             const uint32_t round = i / STAGES;
-            if (!dead && !mbar_wait(&full[s], round & 1)) {
-                dead = true;
-                if (lane == 0) {
-                    cs.abort = 1;
-                    atomicOr(a.status, ST_INTERNAL);
+            if (!lost) {
+                const int wr = mbar_wait_twice(&full[s], round & 1, wait_limit_ns);
+                if (wr != WAIT_OK) {
+                    dead = true;
+                    lost = wr == WAIT_LOST;
+                    if (lane == 0) {
+                        cta.abort = 1;
+                        atomicOr(a.status, ST_INTERNAL);
+                    }
                 }
             }
             const int c = ti * TILE_CHUNKS + warp;
             const bool work = !dead && valid && !full_region && c < a.nch;
             const unsigned char* chunk = stage_mem + s * TILE_BYTES + warp * (CHUNK * (int)sizeof(T));
             ChunkRegs<T> regs;
-            if (work) {
-                load_staged(regs, chunk, c * CHUNK, a.V, lane);
-                if (!STATS) {
-                    // without the exp-sum (which turns NaN by itself) a NaN has to be looked for
-                    const float lm = regs.lane_max();
-                    if (lm != lm) cs.nan = 1;
-                }
-            }
-            if (ti == 0 && valid) {
-                // first tile (every warp holds a full chunk): each warp's own bound, then the minimum
+            if (work) load_staged(regs, chunk, c * CHUNK, a.V, lane);
+            if (ti == pc.tile0 && valid) {
+                // first tile of a piece (every warp holds a full chunk): each warp's own bound, then the minimum
                 if (work) {
-                    const unsigned k16 = first_tile_key(regs, g, need);
+                    unsigned k16;
                     float wm = 0.f;
-                    if (STATS) wm = warp_max_redux(regs.lane_max_plain());
+                    if (SMALL && group_lanes >= 2) {
+                        const float lm = regs.lane_max_plain();
+                        k16 = first_tile_key_groups(lm, group_lanes);
+                        if (STATS) wm = warp_max_redux(lm);
+                    } else {
+                        k16 = first_tile_key(regs, g, need);
+                        if (STATS) wm = warp_max_redux(regs.lane_max_plain());
+                    }
                     if (lane == 0) {
                         atomicMin(&cs.thr0_key, k16 << 16);
                         if (STATS && wm == wm) atomicMax(&cs.top_key, orderable(wm));
@@ -421,6 +558,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
                 if (STATS) ref_off = __fmul_rn(from_orderable(*(volatile unsigned*)&cs.top_key), c32);
                 __syncwarp();
             }
+            int added = 0;          // what this chunk appends to the region
             if (work) {
                 const unsigned thr_key = *(volatile unsigned*)&cs.thr_key;
                 unsigned mask = pass_mask(regs, thr_of_key(thr_key));
@@ -429,38 +567,46 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
                     full_region = true;
                     mask = 0u;
                 }
-                if (STATS) acc += lane_exp_sum2(regs, c32, ref_off);
-                const int total = __reduce_add_sync(0xffffffffu, __popc(mask));     // what this chunk adds
-                if (wcount + total > CS_REGION) {
-                    // no room: bring the bound up to date and drop what fell below it
-                    wcount = maintain_region(wcount, region_off, hist_off, &cs, k_eff);
-                    if (wcount + total > CS_REGION) {     // ties, a coarse bin too full, or a very loose bound
-                        full_region = true;
-                        mask = 0u;
-                    }
-                }
-                // one set bit per lane per step; lanes are ranked by ballot
-                const int before = wcount;
-                const int vchunk = c * CHUNK;
-                for (;;) {
-                    const unsigned m = __ballot_sync(0xffffffffu, mask != 0u);
-                    if (m == 0u) break;
-                    if (mask != 0u) {
-                        const int bit = __ffs(mask) - 1;
-                        mask &= mask - 1u;
-                        const int off = bit_offset(bit, lane, (const T*)nullptr);
-                        const int pos = wcount + __popc(m & lt_mask);
-                        {
-                            const uint32_t bits = __float_as_uint(staged_value(chunk, off, (const T*)nullptr) + 0.0f);   // -0 becomes +0
-                            const uint32_t okey = bits ^ ((uint32_t)((int32_t)bits >> 31) | 0x80000000u);
-                            region[pos] = ((u64)okey << 32) | (u64)(~(uint32_t)(vchunk + off));
+                const int n = __popc(mask);
+                added = __reduce_add_sync(0xffffffffu, n);
+                if (added) {
+                    if (wcount + added > CS_REGION) {
+                        // no room: bring the bound up to date and drop what fell below it
+                        wcount = maintain_region(wcount, region_off, hist_off, &cs, &cta.wcnt[warp], k_eff);
+                        if (wcount + added > CS_REGION) {     // ties, a coarse bin too full, or a very loose bound
+                            full_region = true;
+                            mask = 0u;
+                            added = 0;
                         }
                     }
-                    wcount += __popc(m);
+                    const int vchunk = c * CHUNK;
+                    // every lane appends its own passing values: its slots come from the warp's counter
+                    if (mask) {
+                        int pos = atomicAdd(&cta.wcnt[warp], n);
+                        do {
+                            const int bit = __ffs(mask) - 1;
+                            mask &= mask - 1u;
+                            const int off = bit_offset(bit, lane, (const T*)nullptr);
+                            const uint32_t bits = __float_as_uint(staged_value(chunk, off, (const T*)nullptr) + 0.0f);   // -0 becomes +0
+                            const uint32_t okey = bits ^ ((uint32_t)((int32_t)bits >> 31) | 0x80000000u);
+                            region[pos++] = ((u64)okey << 32) | (u64)(~(uint32_t)(vchunk + off));
+                        } while (mask);
+                    }
                 }
-                __syncwarp();
+            }
+            __syncwarp();
+            if (lane == 0 && !lost) mbar_arrive(&empty[s]);     // the staged chunk is not read again
+            if (work) {
+                if (STATS) {
+                    acc += lane_exp_sum2(regs, c32, ref_off);
+                } else {
+                    // without the exp-sum (which turns NaN by itself) a NaN has to be looked for
+                    const float lm = regs.lane_max();
+                    if (lm != lm) cs.nan = 1;
+                }
                 // count the new entries in the histogram
-                for (int x = before + lane; x < wcount; x += 32) hist_add(hist, hist_bin((unsigned)(region[x] >> 32), g0));
+                for (int x = wcount + lane; x < wcount + added; x += 32) hist_add(hist, hist_bin((unsigned)(region[x] >> 32), g0));
+                wcount += added;
                 // the bound is refreshed after every tile, each time by another warp (the others'
                 // latest values may not be counted yet, which only makes it a little lower)
                 if (warp == (ti & (WARPS - 1))) {
@@ -468,35 +614,35 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
                     refresh_bound(hist_off, &cs, k_eff);
                 }
             }
-            __syncwarp();
-            if (lane == 0 && !dead) mbar_arrive(&empty[s]);     // the stage is free again
         }
 
-        // ---- row end: survivors and row statistics to global scratch -----------------------------
+        // ---- end of the piece: survivors and statistics to the piece's scratch area ------------------
         if (lane == 0 && full_region) cs.overflow = 1;
         if (STATS) {
             const double sw = (double)warp_sum(acc);
             if (lane == 0) cs.wsum[warp] = sw;
         }
-        workers_sync();
-        const bool row_ok = valid && !*(volatile int*)&cs.overflow && !*(volatile int*)&cs.abort;
-        if (row_ok && warp == 0) refresh_threshold(hist, cs, k_eff, lane);
-        workers_sync();
-        if (row_ok) {
-            // every warp filters its own region and appends to the row's scratch area
-            u64* dst = a.surv_keys + (long long)row * surv_cap;
-            const int n = compact_region(region, wcount, *(volatile unsigned*)&cs.thr_key, lane);
+        workers_sync();     // every candidate is counted, every flag is set
+        const bool piece_ok = valid && !*(volatile int*)&cs.overflow && !*(volatile int*)&cta.abort;
+        unsigned thr_final = *(volatile unsigned*)&cs.thr_key;
+        if (piece_ok) {
+            // the final bound, by every warp for itself (all get the same): no second barrier for it
+            const int found = kth_bin(hist, k_eff, lane);
+            if (found >= 0) thr_final = max(thr_final, coord_code(g0 + found) << 16);
+            // every warp filters its own region and appends to the piece's scratch area
+            u64* dst = a.surv_keys + (long long)pc.area * surv_cap;
+            const int n = compact_region(region, wcount, thr_final, lane);
             int base = 0;
             if (lane == 0 && n) base = atomicAdd(&cs.m, n);
             base = __shfl_sync(0xffffffffu, base, 0);
             for (int x = lane; x < n; x += 32)
                 if (base + x < surv_cap) dst[base + x] = region[x];
         }
-        workers_sync();
+        workers_sync();     // the survivors are counted; nobody reads the histogram any more
         if (tid == 0) {
             int flags = 0;
             const int m = cs.m;
-            if (cs.abort) flags = CSF_ABORT;
+            if (cta.abort) flags = CSF_ABORT;
             else if (!in_range) flags = CSF_RANGE;
             else if (!valid) flags = CSF_TEMPERATURE;
             else if (cs.overflow || m > surv_cap) flags = CSF_REDO;      // too many candidates or ties at the bound
@@ -507,27 +653,19 @@ __global__ void __launch_bounds__(STREAM_THREADS, CsGeom<T, SMALL>::CTAS) compre
                 for (int w = 0; w < WARPS; ++w) zs += cs.wsum[w];
             // a reference that later logits overflowed, or NaN / +inf data: the direct kernel sorts it out
             if (STATS && flags == 0 && !(zs > 0.0 && zs < CUDART_INF)) flags = CSF_REDO;
-            if (flags & CSF_REDO) {
-                a.redo_rows[atomicAdd(a.redo_count, 1)] = row;
-                atomicAdd(a.redo_total, 1ull);
-            }
             CsRowMeta meta;
             meta.count = m;
             meta.flags = flags;
             meta.ref_off = ref_off;
-            meta.thr_key = cs.thr_key;
+            meta.thr_key = thr_final;
             meta.z_stream = zs;
-            a.surv_meta[row] = meta;
-            // reset the row state
-            cs.thr_key = 0u;
-            cs.thr0_key = 0xffffffffu;
-            cs.top_key = 0u;
-            cs.overflow = 0;
-            cs.nan = 0;
-            cs.m = 0;
+            a.surv_meta[pc.area] = meta;
+            cs_reset(cs);       // this copy is used again by the piece after the next one
         }
+        // Ready for the next piece, without a barrier of its own: the histogram is not written before
+        // the barrier of that piece's first tile, which every warp reaches after its share of this.
+        if (lane == 0) cta.wcnt[warp] = 0;
         for (int x = tid; x < CS_HIST_WORDS; x += THREADS) hist[x] = 0u;
-        workers_sync();
     }
 }
 
@@ -631,42 +769,77 @@ __device__ __noinline__ void sort_keys(const u64* in, int count, u64* out, unsig
 }
 
 constexpr int CS_TIE_CAP = 256;     // boundary-group size up to which the survivors are trimmed to k
+constexpr int CS_MAX_PIECES = 8;    // most pieces a row is dealt in
 
 struct CsFinishShared {
     unsigned hi16;      // largest 16-bit logit code among the survivors
     int kept, ties;     // slot counters: survivors above the bound's code / with it
+    int overflow;       // more survivors than the exchange buffers hold
+    int found;          // multi-piece rows: bin of the k-th largest code among all pieces' survivors
+    int piece_id[CS_MAX_PIECES];
+    int piece_count[CS_MAX_PIECES];
 };
 
-// One CTA per row: trim the survivors to the k best where that is cheap, sort, cut / renormalise /
-// emit.  The survivors are all elements at or above the filter's final bound, i.e. the k best plus
-// whatever shares the bound's 16-bit code with the k-th (ties of a 16-bit logit; values within
-// 2^-7 relative of it for 32-bit logits).  When they would need a larger sort network than k
-// keys do, the members of that boundary group are ranked among themselves (all pairs) and only
-// the best k - (number above the group) are kept.
+// One CTA per row: put the row's pieces together, trim the survivors to the k best where that is
+// cheap, sort, cut / renormalise / emit.  The survivors of a piece are all its elements at or above
+// its final bound, i.e. its k best plus whatever shares the bound's 16-bit code with the k-th (ties
+// of a 16-bit logit; values within 2^-7 relative of it for 32-bit logits).  The largest of the
+// pieces' bounds is a bound for the row.  A row in several pieces holds about k survivors per piece
+// above it: their 16-bit codes are counted in the filter kernel's two-level histogram first, which
+// gives the code of the row's k-th largest logit, and only survivors at or above that code go on.
+// When the survivors would need a larger sort network than k keys do, the members of the boundary
+// group (the lowest code) are ranked among themselves (all pairs) and only the best
+// k - (number above the group) are kept.
 template <typename T, bool STATS>
-__global__ void __launch_bounds__(THREADS, 6) compress_finish_kernel(CompressArgs a, int n2cap) {
+__global__ void __launch_bounds__(THREADS, 6) compress_finish_kernel(CompressArgs a, FilterPlan plan, int n2cap) {
     extern __shared__ u64 keys[];          // two exchange buffers of n2cap keys; the sorted keys end up in the first
     __shared__ CompressShared sh;
     __shared__ CsFinishShared fs;
-    const int tid = threadIdx.x, lane = tid & 31;
+    __shared__ __align__(16) unsigned fhist[CS_HIST_WORDS];    // (kth_bin reads four super-bins at a time)
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int row = blockIdx.x;
     int k_eff = a.top_k > 0 ? a.top_k : a.k_max;
     if (k_eff > a.k_max) k_eff = a.k_max;
     if (k_eff > a.V) k_eff = a.V;
+    const int surv_cap = cs_survivor_cap(a.k_max);
+    // the scratch areas that hold this row: its own, or those of its pieces if it was dealt in pieces
+    const int whole_rows = plan.q * plan.grid;
+    const bool split_row = row >= whole_rows;
+    const int area0 = split_row ? plan.rows + (row - whole_rows) * plan.split : row;
+    const int nareas = split_row ? plan.split : 1;
     grid_dependency_sync();
-    const u64* src = a.surv_keys + (long long)row * cs_survivor_cap(a.k_max);
-    // the first 512 scratch slots exist for every k_max: requested before the row's count is known
-    const u64 first0 = src[tid], first1 = src[tid + THREADS];
-    const CsRowMeta meta = a.surv_meta[row];
-    if (meta.flags & CSF_REDO) return;                 // the direct kernel writes this row
-    if (meta.flags) {
+    // the first piece's first 512 scratch slots exist for every k_max: requested before its count is known
+    const u64* src0 = a.surv_keys + (long long)area0 * surv_cap;
+    const u64 first0 = src0[tid], first1 = src0[tid + THREADS];
+    // ---- the pieces: flags, the row's bound ----------------------------------------------------------
+    int np = 0, flags = 0;
+    unsigned thr_key = 0u;
+    for (int j = 0; j < nareas; ++j) {
+        if (split_row && j > 0 && plan_piece_tile(plan, j + 1) <= plan_piece_tile(plan, j)) continue;   // an empty piece
+        const CsRowMeta meta = a.surv_meta[area0 + j];
+        flags |= meta.flags;
+        thr_key = max(thr_key, meta.thr_key);
+        if (np < CS_MAX_PIECES && tid == 0) {
+            fs.piece_id[np] = area0 + j;
+            fs.piece_count[np] = meta.count;
+        }
+        ++np;
+    }
+    if (np > CS_MAX_PIECES) flags |= CSF_REDO;
+    if (flags & (CSF_ABORT | CSF_TEMPERATURE | CSF_LOGIT | CSF_RANGE)) {
         emit_invalid_row(a, row);
-        if (tid == 0 && (meta.flags & (CSF_TEMPERATURE | CSF_LOGIT | CSF_RANGE)))
-            atomicOr(a.status, (meta.flags & CSF_TEMPERATURE) ? ST_TEMPERATURE : (meta.flags & CSF_RANGE) ? ST_RANGE : ST_LOGIT);
+        if (tid == 0 && !(flags & CSF_ABORT))
+            atomicOr(a.status, (flags & CSF_TEMPERATURE) ? ST_TEMPERATURE : (flags & CSF_RANGE) ? ST_RANGE : ST_LOGIT);
         return;
     }
-    const int m = meta.count;
-    const unsigned thr16 = meta.thr_key >> 16;
+    if (flags & CSF_REDO) {
+        // a piece's candidates did not fit: the direct kernel writes this row
+        if (tid == 0) {
+            a.redo_rows[atomicAdd(a.redo_count, 1)] = row;
+            atomicAdd(a.redo_total, 1ull);
+        }
+        return;
+    }
     const float Tb = a.temperature[row / a.G];
     u64* bufA = keys;
     u64* bufB = keys + n2cap;
@@ -674,36 +847,80 @@ __global__ void __launch_bounds__(THREADS, 6) compress_finish_kernel(CompressArg
         fs.hi16 = 0u;
         fs.kept = 0;
         fs.ties = 0;
+        fs.overflow = 0;
+        fs.found = -1;
     }
+    if (np > 1)
+        for (int x = tid; x < CS_HIST_WORDS; x += THREADS) fhist[x] = 0u;
     __syncthreads();
+    if (np > 1) {
+        // ---- several pieces: the code of the row's k-th largest logit among all their survivors ------
+        const int g0 = bin_coord(thr_key >> 16);
+        for (int p = 0; p < np; ++p) {
+            const u64* src = a.surv_keys + (long long)fs.piece_id[p] * surv_cap;
+            const int m = fs.piece_count[p];
+            for (int e = tid; e < m; e += THREADS) {
+                const unsigned okey = (unsigned)(src[e] >> 32);
+                if (okey >= thr_key) hist_add(fhist, hist_bin(okey, g0));
+            }
+        }
+        __syncthreads();
+        if (warp == 0) {
+            const int found = kth_bin(fhist, k_eff, lane);
+            if (lane == 0) fs.found = found;
+        }
+        __syncthreads();
+        if (fs.found >= 0) thr_key = max(thr_key, coord_code(g0 + fs.found) << 16);
+    }
+    const unsigned thr16 = thr_key >> 16;
     // ---- survivors to shared memory: those above the bound's code to buffer A, the boundary group
     // ---- to buffer B, both in arrival order (warp-aggregated slots)
     {
         const unsigned lt = (1u << lane) - 1u;
         unsigned hi = 0u;
-        for (int e0 = 0; e0 < m; e0 += THREADS) {
-            const int e = e0 + tid;
-            const u64 key = e0 == 0 ? first0 : e0 == THREADS ? first1 : (e < m ? src[e] : 0ull);
-            const unsigned code = (unsigned)(key >> 48);
-            const bool is_above = e < m && code > thr16;
-            const bool is_tie = e < m && !is_above;
-            if (e < m) hi = max(hi, code);
-            const unsigned ma = __ballot_sync(0xffffffffu, is_above), mt = __ballot_sync(0xffffffffu, is_tie);
-            int ba = 0, bt = 0;
-            if (lane == 0) {
-                if (ma) ba = atomicAdd(&fs.kept, __popc(ma));
-                if (mt) bt = atomicAdd(&fs.ties, __popc(mt));
+        for (int p = 0; p < np; ++p) {
+            const u64* src = a.surv_keys + (long long)fs.piece_id[p] * surv_cap;
+            const int m = fs.piece_count[p];
+            for (int e0 = 0; e0 < m; e0 += THREADS) {
+                const int e = e0 + tid;
+                const u64 key = (p == 0 && e0 == 0) ? first0 : (p == 0 && e0 == THREADS) ? first1 : (e < m ? src[e] : 0ull);
+                const unsigned code = (unsigned)(key >> 48);
+                const bool live = e < m && (unsigned)(key >> 32) >= thr_key;
+                const bool is_above = live && code > thr16;
+                const bool is_tie = live && !is_above;
+                if (live) hi = max(hi, code);
+                const unsigned ma = __ballot_sync(0xffffffffu, is_above), mt = __ballot_sync(0xffffffffu, is_tie);
+                int ba = 0, bt = 0;
+                if (lane == 0) {
+                    if (ma) ba = atomicAdd(&fs.kept, __popc(ma));
+                    if (mt) bt = atomicAdd(&fs.ties, __popc(mt));
+                }
+                ba = __shfl_sync(0xffffffffu, ba, 0);
+                bt = __shfl_sync(0xffffffffu, bt, 0);
+                const int sa = ba + __popc(ma & lt), st = bt + __popc(mt & lt);
+                if (is_above) {
+                    if (sa < n2cap) bufA[sa] = key;
+                    else fs.overflow = 1;
+                }
+                if (is_tie) {
+                    if (st < n2cap) bufB[st] = key;
+                    else fs.overflow = 1;
+                }
             }
-            ba = __shfl_sync(0xffffffffu, ba, 0);
-            bt = __shfl_sync(0xffffffffu, bt, 0);
-            if (is_above) bufA[ba + __popc(ma & lt)] = key;
-            if (is_tie) bufB[bt + __popc(mt & lt)] = key;
         }
         hi = __reduce_max_sync(0xffffffffu, hi);
         if (lane == 0) atomicMax(&fs.hi16, hi);
     }
     __syncthreads();
-    const int above = fs.kept, t = m - above;
+    const int above = fs.kept, t = fs.ties, m = above + t;
+    if (fs.overflow || m > n2cap || m < k_eff) {
+        // more survivors than the buffers hold (a histogram window too coarse for this row): direct kernel
+        if (tid == 0) {
+            a.redo_rows[atomicAdd(a.redo_count, 1)] = row;
+            atomicAdd(a.redo_total, 1ull);
+        }
+        return;
+    }
     const bool narrow = sizeof(T) == 2 && a.V <= (1 << 18) && fs.hi16 - thr16 < (1u << 14);
     int nk = 256;                       // network size for k keys
     while (nk < k_eff) nk <<= 1;
@@ -743,9 +960,12 @@ __global__ void __launch_bounds__(THREADS, 6) compress_finish_kernel(CompressArg
     const float top = key_logit(keys[0]);
     double Z = 0.0;
     if (STATS) {
-        // move the streamed sum from its reference onto the scale of the weights exp(l/T - top/T)
+        // move every piece's streamed sum from its reference onto the scale of the weights exp(l/T - top/T)
         const float c32 = temp_scale(Tb);
-        Z = meta.z_stream * exp2((double)meta.ref_off - (double)top * (double)c32);
+        for (int p = 0; p < np; ++p) {
+            const CsRowMeta meta = a.surv_meta[fs.piece_id[p]];
+            Z += meta.z_stream * exp2((double)meta.ref_off - (double)top * (double)c32);
+        }
     }
     const bool bad = !(top > -CUDART_INF_F) || !(top < CUDART_INF_F) || (STATS && !(Z > 0.0));
     if (bad) {

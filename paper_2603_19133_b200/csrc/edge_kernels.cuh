@@ -31,6 +31,7 @@ __global__ void __launch_bounds__(THREADS) edge_finish_kernel(VerifyArgs a) {
         unsigned st_bits = 0;
         if (!temp_ok(Tb)) st_bits |= ST_TEMPERATURE;
         if (j < 0 || j > a.G || n <= 0 || n > a.k_max) st_bits |= ST_RANGE;
+        if (*(volatile unsigned*)a.status & ST_INTERNAL) st_bits |= ST_INTERNAL;   // incomplete statistics
         __syncthreads();
         if (tid == 0) {
             sbad = 0;

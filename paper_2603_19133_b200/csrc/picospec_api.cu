@@ -17,11 +17,14 @@
 using namespace picospec;
 
 #define PROF_RING 128
+// most CTAs per SM any shape of the staged filter kernel runs at (sizes the per-piece scratch)
+#define FILTER_MAX_CTAS_PER_SM 4
 
 struct picospec_ctx {
     int device;
     int max_batch, max_gamma, max_vocab, max_k;
     int num_sms;
+    unsigned long long wait_limit_ns;   // first limit of the staged kernels' waits
     int last_cuda_error;
     unsigned long long compress_calls;
     // optional per-kernel timing (picospec_profile_*): rings of event pairs per kernel kind
@@ -165,11 +168,10 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
     if (staged) {
         cudaError_t ea = ensure_kernel_attrs(ctx->device);
         if (ea != cudaSuccess) return ea;
-        const int tiles_per_row = (a.nch + TILE_CHUNKS - 1) / TILE_CHUNKS;
         int k_eff = a.top_k > 0 ? a.top_k : a.k_max;
         if (k_eff > a.k_max) k_eff = a.k_max;
         const bool small = k_eff <= CS_K_SMALL;
-        void (*kern)(CompressArgs, int) =
+        void (*kern)(CompressArgs, FilterPlan, unsigned long long) =
             small ? (stats ? compress_filter_kernel<T, true, true> : compress_filter_kernel<T, false, true>)
                   : (stats ? compress_filter_kernel<T, true, false> : compress_filter_kernel<T, false, false>);
         const int smem = small ? CsGeom<T, true>::SMEM_BYTES : CsGeom<T, false>::SMEM_BYTES;
@@ -177,10 +179,13 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
         cudaError_t eo = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, STREAM_THREADS, smem);
         if (eo != cudaSuccess) return eo;
         if (per_sm < 1) per_sm = 1;
-        const int g = rows < ctx->num_sms * per_sm ? rows : ctx->num_sms * per_sm;
+        if (per_sm > FILTER_MAX_CTAS_PER_SM) per_sm = FILTER_MAX_CTAS_PER_SM;
+        // whole rows first, the remainder in pieces so that every CTA streams about the same number of tiles
+        const FilterPlan plan = make_filter_plan(rows, (a.nch + TILE_CHUNKS - 1) / TILE_CHUNKS,
+                                                 a.V % (TILE_CHUNKS * CHUNK) != 0, (long long)ctx->num_sms * per_sm);
         {
             ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_STREAM, 1, s);
-            launch_chained(kern, g, STREAM_THREADS, smem, s, a, tiles_per_row);
+            launch_chained(kern, plan.grid, STREAM_THREADS, smem, s, a, plan, ctx->wait_limit_ns);
         }
         cudaError_t e0 = cudaGetLastError();
         if (e0 != cudaSuccess) return e0;
@@ -189,8 +194,8 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
             while (n2 < cs_survivor_cap(a.k_max)) n2 <<= 1;
             ProfScope ps(ctx, PICOSPEC_PROF_COMPRESS_FINISH, 2, s);
             // two exchange buffers of the sort network (the sorted keys end up in the first)
-            if (stats) launch_chained(compress_finish_kernel<T, true>, rows, THREADS, (size_t)n2 * 16, s, a, n2);
-            else launch_chained(compress_finish_kernel<T, false>, rows, THREADS, (size_t)n2 * 16, s, a, n2);
+            if (stats) launch_chained(compress_finish_kernel<T, true>, rows, THREADS, (size_t)n2 * 16, s, a, plan, n2);
+            else launch_chained(compress_finish_kernel<T, false>, rows, THREADS, (size_t)n2 * 16, s, a, plan, n2);
         }
         e0 = cudaGetLastError();
         if (e0 != cudaSuccess) return e0;
@@ -235,7 +240,8 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
         const int gcap = ctx->num_sms * StreamCfg<T>::CTAS_PER_SM;
         const int g = (int)(tiles < gcap ? tiles : gcap);
         ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_STREAM, 1, s);
-        launch_chained(chunk_stats_bulk_kernel<T>, g, STREAM_THREADS, TileGeom<T>::SMEM_BYTES, s, a, tiles_per_row, tiles);
+        launch_chained(chunk_stats_bulk_kernel<T>, g, STREAM_THREADS, TileGeom<T>::SMEM_BYTES, s, a, tiles_per_row, tiles,
+                       ctx->wait_limit_ns);
     } else {
         ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_STREAM, 1, s);
         if (aligned) launch_chained(chunk_stats_kernel<T, true>, grid, THREADS, 0, s, a);
@@ -310,6 +316,7 @@ int picospec_create(picospec_ctx** out, int device, int max_batch, int max_gamma
     ctx->max_gamma = max_gamma;
     ctx->max_vocab = max_vocab;
     ctx->max_k = max_k;
+    ctx->wait_limit_ns = WAIT_LIMIT_NS;
     DeviceGuard g(device);
     cudaError_t e = g.ok ? cudaSuccess : cudaErrorInvalidDevice;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, device);
@@ -322,8 +329,11 @@ int picospec_create(picospec_ctx** out, int device, int max_batch, int max_gamma
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->need_rows, rows * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->counters, 8 * sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->redo_rows, rows * sizeof(int));
-    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_keys, rows * (size_t)cs_survivor_cap(max_k) * sizeof(unsigned long long));
-    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_meta, rows * sizeof(CsRowMeta));
+    // one scratch area per whole row and per piece of a row that is dealt in pieces (at most twice
+    // the CTAs of the filter kernel)
+    const size_t pieces = rows + 2 * (size_t)ctx->num_sms * FILTER_MAX_CTAS_PER_SM;
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_keys, pieces * (size_t)cs_survivor_cap(max_k) * sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_meta, pieces * sizeof(CsRowMeta));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->wire_off, (rows + 1) * sizeof(int));
     ctx->max_rows = (long long)rows;
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->status, sizeof(unsigned));
@@ -376,6 +386,12 @@ const char* picospec_strerror(int err) {
 }
 
 int picospec_last_cuda_error(const picospec_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+int picospec_wait_limit(picospec_ctx* ctx, unsigned long long limit_ns) {
+    if (!ctx) return PICOSPEC_EINVAL;
+    ctx->wait_limit_ns = limit_ns < WAIT_LIMIT_NS ? limit_ns : WAIT_LIMIT_NS;
+    return PICOSPEC_OK;
+}
 
 int picospec_profile_enable(picospec_ctx* ctx, int level) {
     if (!ctx || level < 0 || level > 2) return PICOSPEC_EINVAL;
@@ -762,6 +778,7 @@ extern "C" int picospec_verify_static(const void* target_logits, picospec_dtype 
     StaticWorkspace* ws = nullptr;
     picospec_ctx local = {};          // host-side launch parameters only; owns nothing
     local.device = device;
+    local.wait_limit_ns = WAIT_LIMIT_NS;
     if (static_workspace(device, &ws, &local.num_sms) != cudaSuccess) return PICOSPEC_ECUDA;
 
     cudaStream_t s = (cudaStream_t)cuda_stream;

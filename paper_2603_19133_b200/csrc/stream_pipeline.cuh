@@ -2,7 +2,8 @@
 // mbarriers: one producer lane keeps STAGES tiles in flight, consumer warps take a tile as soon
 // as its bytes have landed and hand the stage back once they have moved it to registers.
 // Every wait is bounded: a barrier that does not complete within the limit makes the waiting
-// warp record ST_INTERNAL in the status word and leave its loop.
+// warp record ST_INTERNAL in the status word and stop computing; it keeps consuming tiles (with the
+// long limit) so that every copy that was issued has landed before its CTA exits.
 #pragma once
 #include "common.cuh"
 
@@ -39,6 +40,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// non-blocking: has the phase completed?
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // the same with a suspend-time hint (ns): the thread may sleep in hardware instead of polling
 __device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parity, uint32_t ns) {
     uint32_t ok;
@@ -57,13 +70,27 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 // false: the time limit ran out
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned long long limit_ns) {
+    // a limit of zero: only a wait that is complete already succeeds (try_wait may itself suspend the
+    // thread for a while, so this case asks with the non-blocking test_wait)
+    if (limit_ns == 0ull) return mbar_test_wait(bar, parity);
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (uint32_t i = 1;; ++i) {
         if (mbar_try_wait_hint(bar, parity, PICOSPEC_WAIT_HINT_NS)) return true;
-        if ((i & 7u) == 0u && global_ns() - t0 > WAIT_LIMIT_NS) return false;
+        if ((i & 7u) == 0u && global_ns() - t0 > limit_ns) return false;
     }
+}
+// The wait of the staged kernels, in two steps: first with the caller's limit, then -- so that no CTA
+// leaves while a bulk copy into its shared memory is still in flight -- once more with the long limit.
+//   WAIT_OK    completed within `limit_ns`;
+//   WAIT_LATE  completed, but only after `limit_ns` had run out: the caller records ST_INTERNAL, stops
+//              computing and keeps consuming, so every issued copy still lands and is waited for;
+//   WAIT_LOST  not complete after the long limit either: the caller gives up for good.
+enum { WAIT_OK = 0, WAIT_LATE = 1, WAIT_LOST = 2 };
+__device__ __forceinline__ int mbar_wait_twice(uint64_t* bar, uint32_t parity, unsigned long long limit_ns) {
+    if (mbar_wait(bar, parity, limit_ns)) return WAIT_OK;
+    return mbar_wait(bar, parity, WAIT_LIMIT_NS) ? WAIT_LATE : WAIT_LOST;
 }
 
 __device__ __forceinline__ uint64_t l2_evict_first_policy() {

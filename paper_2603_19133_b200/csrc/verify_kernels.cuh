@@ -157,7 +157,8 @@ struct TileDesc {
 
 template <typename T>
 __global__ void __launch_bounds__(STREAM_THREADS, StreamCfg<T>::CTAS_PER_SM) chunk_stats_bulk_kernel(VerifyArgs a, int tiles_per_row,
-                                                                             long long total_tiles) {
+                                                                             long long total_tiles,
+                                                                             unsigned long long wait_limit_ns) {
     extern __shared__ __align__(1024) unsigned char stage_mem[];
     constexpr int STAGES = StreamCfg<T>::STAGES;
     constexpr int CPW = StreamCfg<T>::CPW;
@@ -188,9 +189,10 @@ __global__ void __launch_bounds__(STREAM_THREADS, StreamCfg<T>::CTAS_PER_SM) chu
         for (uint32_t i = 0; t < total_tiles; ++i, t += gridDim.x) {
             const int s = (int)(i % STAGES);
             const uint32_t round = i / STAGES;
-            if (round > 0 && !mbar_wait(&empty[s], (round - 1) & 1)) {
-                atomicOr(a.status, ST_INTERNAL);
-                break;
+            if (round > 0) {
+                const int wr = mbar_wait_twice(&empty[s], (round - 1) & 1, wait_limit_ns);
+                if (wr != WAIT_OK) atomicOr(a.status, ST_INTERNAL);
+                if (wr == WAIT_LOST) break;       // nothing more is issued
             }
             const int r = (int)(t / tiles_per_row);
             const int tc = (int)(t - (long long)r * tiles_per_row);
@@ -226,18 +228,21 @@ __global__ void __launch_bounds__(STREAM_THREADS, StreamCfg<T>::CTAS_PER_SM) chu
 
     // ---- consumers ------------------------------------------------------------------------
     long long t = blockIdx.x;
+    bool late = false;      // a wait ran out: this warp computes no more, but keeps taking tiles
     for (uint32_t i = 0; t < total_tiles; ++i, t += gridDim.x) {
         const int s = (int)(i % STAGES);
         const uint32_t round = i / STAGES;
-        if (!mbar_wait(&full[s], round & 1)) {
+        const int wr = mbar_wait_twice(&full[s], round & 1, wait_limit_ns);
+        if (wr != WAIT_OK) {
+            late = true;
             if (lane == 0) atomicOr(a.status, ST_INTERNAL);
-            break;
+            if (wr == WAIT_LOST) break;
         }
         const TileDesc d = desc[s];
 #pragma unroll
         for (int q = 0; q < CPW; ++q) {
             const int c = d.c0 + warp * CPW + q;
-            const bool work = d.valid && c < a.nch;
+            const bool work = d.valid && c < a.nch && !late;
             ChunkRegs<T> regs;
             if (work) load_staged(regs, stage_mem + s * TILE_BYTES + (warp * CPW + q) * (CHUNK * (int)sizeof(T)), c * CHUNK, a.V, lane);
             if (q == CPW - 1) {
@@ -345,6 +350,9 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
         const T* seq = reinterpret_cast<const T*>(a.logits) + (long long)b * G1 * a.row_stride;
         unsigned st_bits = 0;
         if (!temp_ok(Tb)) st_bits |= ST_TEMPERATURE;
+        // a wait of the streaming pass ran out (now or in a call since the status word was last
+        // cleared): its statistics are not complete, nothing of this call is valid
+        if (*(volatile unsigned*)a.status & ST_INTERNAL) st_bits |= ST_INTERNAL;
         // rows lo .. row_hi-1 are read, positions lo .. hi-1 are tested; g is the bonus row
         const int lo = a.sample_only ? 0 : a.r0;
         const int g = (!a.sample_only && a.gamma) ? a.gamma[b] : G;

@@ -537,6 +537,43 @@ def test_redo_list_does_not_leak_into_later_calls(ps):
         ctx.close()
 
 
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(ps):
+    # The staged kernels bound every wait for their asynchronous copies.  With the limit set to zero the
+    # first wait that is not complete already gives up: the status word gets PICOSPEC_ST_INTERNAL, the
+    # outputs are marked invalid, and the kernels still end by themselves (every copy they issued is
+    # waited for).  No copy is skipped and nothing is made to hang.  Afterwards, with the limit back and
+    # the status cleared, the same context gives the oracle's results again.
+    w = gen.scaled(gen.WORKLOADS["config2"], B=4, V=32768)
+    inputs = gen.make_inputs(w, seed=99, device="cuda")
+    ctx = ps.Context(w.B, w.G, w.V, w.k_max)
+    try:
+        dl, tl, T = inputs["draft_logits"], inputs["target_logits"], inputs["temperature"]
+        o_qi, o_qp, o_qc, o_tok = oracle.compress(_np(dl), _np(T), w.top_k, w.top_p, w.k_max, _np(inputs["u_draft"]))
+        o = oracle.verify(_np(tl), _np(T), o_tok, o_qi, o_qp, o_qc, _np(inputs["u_accept"]), _np(inputs["u_resample"]))
+        ctx.wait_limit(0)
+        qi, qp, qc, tok = ctx.compress(dl, T, w.top_k, w.top_p, w.k_max, inputs["u_draft"])
+        st, _ = ctx.status(clear=True)
+        assert st & 8
+        g_qc = _np(qc)
+        assert (g_qc == -1).any()                                  # the rows of a CTA that gave up
+        keep = g_qc >= 0                                           # rows of CTAs that never had to wait
+        assert np.array_equal(_np(qi)[keep], o_qi[keep]) and np.array_equal(g_qc[keep], o_qc[keep])
+        g = ctx.verify(tl, T, _cuda(o_tok), _cuda(o_qi), _cuda(o_qp), _cuda(o_qc), inputs["u_accept"],
+                       inputs["u_resample"])
+        st, _ = ctx.status(clear=True)
+        assert st & 8
+        assert np.all(_np(g["accept_len"]) == -1) and np.all(_np(g["token"]) == -1)
+        ctx.wait_limit(2_000_000_000)
+        qi, qp, qc, tok = ctx.compress(dl, T, w.top_k, w.top_p, w.k_max, inputs["u_draft"])
+        g = ctx.verify(tl, T, tok, qi, qp, qc, inputs["u_accept"], inputs["u_resample"])
+        st, _ = ctx.status(clear=True)
+        assert st == 0
+        assert np.array_equal(_np(qi), o_qi) and np.array_equal(_np(qc), o_qc) and np.array_equal(_np(tok), o_tok)
+        assert np.array_equal(_np(g["accept_len"]), o["accept_len"]) and np.array_equal(_np(g["token"]), o["token"])
+    finally:
+        ctx.close()
+
+
 def test_staged_bad_data_is_reported(ps):
     # NaN and +inf inside rows that take the staged kernels (with and without the exp-sum)
     V, B, G, K = 16384, 4, 1, 16

@@ -46,7 +46,7 @@ __global__ void __launch_bounds__(THREADS) precise_chunk_sums_kernel(PreciseArgs
             c = (int)(item % a.nch);
             const long long t = item / a.nch;
             const int ri = (int)(t % a.expand);
-            const int e = a.queue[(int)(t / a.expand)] & 0x3FFFFFFF;     // (the verify path keeps a flag above the index)
+            const int e = a.queue[(int)(t / a.expand)] & 0x1FFFFFFF;     // (the verify path keeps flags above the index)
             if (a.need_rows && !a.pos && ri < 64 && !((a.need_rows[e] >> ri) & 1ull)) work = false;
             if (!a.pos && (ri < a.r0 || ri >= a.r1 || (a.gamma && ri > a.gamma[e]))) work = false;
             src_row = a.pos ? e * a.seq_rows + a.pos[e] : e * a.expand + ri;

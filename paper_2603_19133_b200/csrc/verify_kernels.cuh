@@ -279,7 +279,7 @@ struct FinishShared {
 };
 
 // queue entries of the verify path: the sequence, plus a flag
-constexpr int QUEUE_SEQ_MASK = 0x3FFFFFFF, QUEUE_DRAW_ONLY = 0x40000000;
+constexpr int QUEUE_SEQ_MASK = 0x1FFFFFFF, QUEUE_DRAW_ONLY = 0x40000000, QUEUE_MASS_ONLY = 0x20000000;
 
 // bit i of a sequence's row mask (rows beyond 63 always count as set)
 __device__ __forceinline__ bool row_needed(unsigned long long need, int i) { return i >= 64 || ((need >> i) & 1ull); }
@@ -334,10 +334,12 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
     const int nloop = PRECISE ? *a.queue_count : a.B;
     for (int slot = blockIdx.x; slot < nloop; slot += gridDim.x) {
         // a queue entry is the sequence, with QUEUE_DRAW_ONLY set when only the draw was too close to
-        // call: then the accept decisions of the fast pass stand and only the sampled row is redone
+        // call: then the accept decisions of the fast pass stand and only the sampled row is redone;
+        // with QUEUE_MASS_ONLY every decision stands and only small residual masses are recomputed
         const int qe = PRECISE ? a.queue[slot] : slot;
         const int b = PRECISE ? (qe & QUEUE_SEQ_MASK) : slot;
         const bool draw_only = PRECISE && (qe & QUEUE_DRAW_ONLY) != 0;
+        const bool mass_only = PRECISE && (qe & QUEUE_MASS_ONLY) != 0;
         const int alen_fast = draw_only ? a.accept_len[b] : 0;
         const unsigned long long need = PRECISE ? a.need_rows[b] : 0ull;   // rows with exact chunk sums
         if (!a.sample_only && a.state_in && a.state_in[b] == 0) {
@@ -376,6 +378,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
             const int i_lo = a.sample_only ? jpos : lo, i_hi = a.sample_only ? jpos + 1 : row_hi;
             for (int i = i_lo + warp; i < i_hi; i += WARPS) {
                 if (draw_only && i != alen_fast) continue;
+                if (mass_only && !row_needed(need, i)) continue;
                 double Z, Zraw;
                 float mx;
                 bool bad;
@@ -394,6 +397,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
         // ---- 2. per draft position: p(x), q~(x), accept test, residual mass ----------------
         if (!st_bits && !sh.bad && !a.sample_only && !draw_only) {
             for (int i = lo + warp; i < hi; i += WARPS) {
+                if (mass_only && !row_needed(need, i)) continue;
                 const int ri = b * G + i;
                 const int* idx = a.q_idx + (long long)ri * a.k_max;
                 const float* prob = a.q_prob + (long long)ri * a.k_max;
@@ -491,6 +495,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
         }
         __syncthreads();
         st_bits |= (unsigned)sh.bad;
+        if (mass_only) continue;        // (bad data was reported by the fast pass already)
 
         // ---- 3. first-rejection scan -----------------------------------------------------
         // A rejection inside the range decides the sequence; so does accepting every position
@@ -728,7 +733,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                     // draw needs the sampled row only; a small residual mass its own row.
                     unsigned long long nd = 0ull;
                     int nrows = 0;
-                    bool draw_only_flag = false;
+                    bool draw_only_flag = false, mass_only_flag = false;
                     if (a.sample_only) {
                         nd = ~0ull;
                         nrows = 1;
@@ -740,6 +745,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                         bool any_small = false;
                         for (int i = lo; i < hi; ++i) any_small |= sh.small[i] != 0;
                         draw_only_flag = first_amb < 0 && !any_small;
+                        mass_only_flag = first_amb < 0 && any_small && !sh.flag;
                         for (int i = lo; i < row_hi; ++i) {
                             const bool nr = i >= 64 || (first_amb >= 0 && i >= first_amb) || (i < hi && sh.small[i]) ||
                                             (sh.flag && want_token && decided && i == alen);
@@ -751,7 +757,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                     }
                     a.need_rows[b] = nd;
                     const int q = atomicAdd(a.queue_count, 1);
-                    a.queue[q] = b | (draw_only_flag ? QUEUE_DRAW_ONLY : 0);
+                    a.queue[q] = b | (draw_only_flag ? QUEUE_DRAW_ONLY : 0) | (mass_only_flag ? QUEUE_MASS_ONLY : 0);
                     atomicAdd(a.slow_rows, (unsigned long long)nrows);
                 }
             }

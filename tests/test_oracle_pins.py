@@ -791,3 +791,40 @@ def test_throughput_model_closed_forms_and_limits():
     # S is never below 1 and grows with alpha
     s = [wire.speedup(a, 5, td, tr, tv) for a in np.linspace(0, 0.999, 50)]
     assert min(s) >= 1.0 and all(b >= a - 1e-12 for a, b in zip(s, s[1:]))
+
+
+# ---------------------------------------------------------------------------------------
+# vocabulary-parallel verification (Sec. 4.1: the verifier model spans several GPUs, so the target
+# logits arrive sharded along the vocabulary): slicing, exchanging chunk records and gathered
+# entries, and deciding from them gives what the plain oracle gives on the whole vocabulary
+# ---------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("cuts", [[0, 5120], [0, 2048, 5120], [0, 1024, 3072, 4096, 5120 + 77]])
+def test_sharded_verification_equals_the_plain_oracle(cuts):
+    from oracle import vocab_parallel as vp
+    rng = _rng(41)
+    B, G, K = 6, 3, 24
+    V = cuts[-1]
+    base = rng.normal(0, 2.5, size=(B, G + 1, V)).astype(np.float32)
+    dl = base[:, :G] + rng.normal(0, 0.7, size=(B, G, V)).astype(np.float32)
+    tl = base.copy()
+    tl[1, 1, 100:200] = -np.inf                       # a stretch of zero-weight entries
+    T = rng.uniform(0.6, 1.3, size=B).astype(np.float32)
+    ud, ua = rng.random((B, G), dtype=np.float32), rng.random((B, G), dtype=np.float32)
+    ur = rng.random((B, 2), dtype=np.float32)
+    qi, qp, qc, tok = oracle.compress(dl, T, top_k=0, top_p=0.9, k_max=K, u_draft=ud)
+    tok[2, 0] = (int(qi[2, 0, 0]) + 7) % V            # a drafted token outside the stored support
+    ref = oracle.verify(tl, T, tok, qi, qp, qc, ua, ur)
+    slices = [np.ascontiguousarray(tl[:, :, a:b]) for a, b in zip(cuts[:-1], cuts[1:])]
+    got = vp.verify_sharded(slices, cuts[:-1], T, tok, qi, qp, qc, ua, ur)
+    assert np.array_equal(got["accept_len"], ref["accept_len"])
+    assert np.array_equal(got["token"], ref["token"])
+    assert got["borderline_count"] == ref["borderline_count"]
+    np.testing.assert_allclose(got["p_draft"], ref["p_draft"], rtol=1e-12, atol=0)
+    np.testing.assert_allclose(got["resid_mass"], ref["resid_mass"], rtol=1e-9, atol=1e-14)
+    # the exchange really is needed: a rank that decided from its own slice alone would differ
+    if len(slices) > 1:
+        alone = vp.verify_sharded(slices[:1], cuts[:1], T, np.minimum(tok, cuts[1] - 1), np.minimum(qi, cuts[1] - 1),
+                                  qp, qc, ua, ur)
+        assert not np.array_equal(alone["token"], ref["token"])
+

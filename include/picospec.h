@@ -307,6 +307,58 @@ PICOSPEC_API int picospec_edge_resample(picospec_ctx* ctx, const void* draft_log
                            const int* p_idx, const float* p_prob, const int* p_count, int k, const float* u,
                            int* token, float* mass, void* cuda_stream);
 
+/* Vocabulary-parallel verification -- Sec. 4.1: the verifier model runs on two to four GPUs, so its
+ * output layer leaves the target logits sharded along the vocabulary.  Rank r of `ranks` holds the
+ * columns [v0, v0 + Vs) of every row of target_logits [B, G+1, V]: v0 = r * chunks_per_rank *
+ * PICOSPEC_CHUNK, every rank but the last holds chunks_per_rank chunks, the last one the rest.  One
+ * verification is the sequence below, the same on every rank; the two kinds of exchange between the
+ * steps are the caller's (an all-gather and an element-wise maximum over ranks, e.g. NCCL), the
+ * library never touches another rank's memory.  Results equal picospec_verify on the whole rows.
+ *
+ *   picospec_vp_local    own slice -> records_local [B*(G+1), chunks_per_rank, 2] fp32 (per chunk: largest
+ *                        logit, sum of 2^((l - max) log2(e)/T)) and entries_local [B*G, k_max+1] fp32 (the
+ *                        slice's logits at the stored entries, last slot: at the drafted token; -inf where
+ *                        the slice does not hold the index)
+ *   exchange             records_all [ranks, B*(G+1), chunks_per_rank, 2] = all-gather(records_local);
+ *                        entries_all = max over ranks(entries_local)
+ *   picospec_vp_decide   (sums_all = NULL) accept tests, p_draft, resid_mass, accept_len, borderline count
+ *                        as in picospec_verify, and pick [B,4] int32: sampled row, picked chunk, flags, rows
+ *   picospec_vp_draw     (sums_all = NULL) the owner of a picked chunk draws the token inside it from its
+ *                        slice -> tok_flag_local [2, B] int32: token or -1; 1 if too close to call
+ *   exchange             tok_flag_all = max over ranks(tok_flag_local)
+ *   picospec_vp_queue    token [B] <- tok_flag_all; the context's list of sequences for the
+ *                        double-precision pass (the same on every rank)
+ *   picospec_vp_exact    own slice -> sums_local [B*(G+1), chunks_per_rank] fp64: exact chunk sums of the
+ *                        listed sequences' rows (other entries are not written)
+ *   exchange             sums_all [ranks, B*(G+1), chunks_per_rank] = all-gather(sums_local)
+ *   picospec_vp_decide   (sums_all given) the listed sequences again, in double precision
+ *   picospec_vp_draw     (sums_all given) their draws -> tok_flag_local
+ *   exchange             tok_flag_all = max over ranks(tok_flag_local)
+ *   picospec_vp_merge    token [B] <- the redone tokens
+ * All calls of one verification use one context and one stream.  All arrays are device pointers;
+ * capacity and data errors are reported as for picospec_verify. */
+PICOSPEC_API int picospec_vp_local(picospec_ctx* ctx, const void* slice_logits, picospec_dtype dtype, int B, int G, int Vs,
+                                   int v0, long long row_stride_elems, int chunks_per_rank, const float* temperature,
+                                   const int* draft_tok, const int* q_idx, const int* q_count, int k_max,
+                                   float* records_local, float* entries_local, void* cuda_stream);
+PICOSPEC_API int picospec_vp_decide(picospec_ctx* ctx, int B, int G, int V, int ranks, int chunks_per_rank,
+                                    const float* records_all, const double* sums_all, const float* entries_all,
+                                    const float* temperature, const int* draft_tok, const int* q_idx,
+                                    const float* q_prob, const int* q_count, int k_max, const float* u_accept,
+                                    const float* u_resample, int* accept_len, float* p_draft, float* resid_mass,
+                                    int* borderline_count, int* pick, void* cuda_stream);
+PICOSPEC_API int picospec_vp_draw(picospec_ctx* ctx, const void* slice_logits, picospec_dtype dtype, int B, int G, int V,
+                                  int v0, long long row_stride_elems, int rank, int ranks, int chunks_per_rank,
+                                  const float* records_all, const double* sums_all, const float* temperature,
+                                  const int* q_idx, const float* q_prob, const int* q_count, int k_max,
+                                  const float* u_resample, const int* pick, int* tok_flag_local, void* cuda_stream);
+PICOSPEC_API int picospec_vp_queue(picospec_ctx* ctx, int B, const int* pick, const int* tok_flag_all, int* token,
+                                   void* cuda_stream);
+PICOSPEC_API int picospec_vp_exact(picospec_ctx* ctx, const void* slice_logits, picospec_dtype dtype, int B, int G, int Vs,
+                                   long long row_stride_elems, int chunks_per_rank, const float* temperature,
+                                   double* sums_local, void* cuda_stream);
+PICOSPEC_API int picospec_vp_merge(picospec_ctx* ctx, int B, const int* tok_flag_all, int* token, void* cuda_stream);
+
 /* Verification without any allocation -- the paper has no counterpart; this entry point exists
  * for callers that cannot obtain device memory at all.  Two kinds of caller are meant: a plugin
  * inside a serving engine that has already claimed the whole of the GPU's memory for its own

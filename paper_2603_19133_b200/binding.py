@@ -62,6 +62,19 @@ def lib() -> ctypes.CDLL:
         L.picospec_wire_unpack.restype = c_int
         L.picospec_profile_samples.argtypes = [vp, c_int, ctypes.POINTER(c_f), c_int, ctypes.POINTER(c_int), vp]
         L.picospec_profile_samples.restype = c_int
+        # vocabulary-parallel verification (driven by vocab_parallel.py)
+        L.picospec_vp_local.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_int, c_ll, c_int, vp, vp, vp, vp, c_int,
+                                        vp, vp, vp]
+        L.picospec_vp_decide.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, vp, vp, vp, vp, vp, vp, vp, vp, c_int,
+                                         vp, vp, vp, vp, vp, vp, vp, vp]
+        L.picospec_vp_draw.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_int, c_ll, c_int, c_int, c_int, vp, vp, vp,
+                                       vp, vp, vp, c_int, vp, vp, vp, vp]
+        L.picospec_vp_queue.argtypes = [vp, c_int, vp, vp, vp, vp]
+        L.picospec_vp_exact.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, c_int, vp, vp, vp]
+        L.picospec_vp_merge.argtypes = [vp, c_int, vp, vp, vp]
+        for f in ("picospec_vp_local", "picospec_vp_decide", "picospec_vp_draw", "picospec_vp_queue",
+                  "picospec_vp_exact", "picospec_vp_merge"):
+            getattr(L, f).restype = c_int
         L.picospec_wait_limit.argtypes = [vp, ctypes.c_ulonglong]
         L.picospec_wait_limit.restype = c_int
         L.picospec_counters.argtypes = [vp, ctypes.POINTER(c_ll), c_int, vp]

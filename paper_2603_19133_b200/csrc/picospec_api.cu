@@ -13,6 +13,7 @@
 #include "verify_kernels.cuh"
 #include "edge_kernels.cuh"
 #include "wire_kernels.cuh"
+#include "vocab_parallel_kernels.cuh"
 
 using namespace picospec;
 
@@ -44,6 +45,7 @@ struct picospec_ctx {
     unsigned long long* surv_keys;  // staged compress: survivors per row
     CsRowMeta* surv_meta;
     int* wire_off;                  // wire codec: first entry of each row, [rows + 1]
+    int* vp_listed;                 // vocabulary-parallel verify: per sequence, its kind in the double-precision pass
     long long max_rows;
     unsigned* status;
     unsigned long long* slow_rows;
@@ -224,8 +226,9 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
     return cudaGetLastError();
 }
 
+// the streaming statistics pass over the rows a call reads
 template <typename T>
-cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, cudaStream_t s, bool edge = false) {
+cudaError_t launch_verify_stream(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, cudaStream_t s) {
     const int stream_rows = a.sample_only ? a.B : a.B * (a.r1 - a.r0);
     const long long items = (long long)stream_rows * a.nch;
     long long want = (items + WARPS - 1) / WARPS;
@@ -246,6 +249,15 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
         ProfScope ps(ctx, PICOSPEC_PROF_VERIFY_STREAM, 1, s);
         if (aligned) launch_chained(chunk_stats_kernel<T, true>, grid, THREADS, 0, s, a);
         else launch_chained(chunk_stats_kernel<T, false>, grid, THREADS, 0, s, a);
+    }
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, cudaStream_t s, bool edge = false) {
+    {
+        cudaError_t e0 = launch_verify_stream<T>(ctx, a, aligned, s);
+        if (e0 != cudaSuccess) return e0;
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -335,6 +347,7 @@ int picospec_create(picospec_ctx** out, int device, int max_batch, int max_gamma
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_keys, pieces * (size_t)cs_survivor_cap(max_k) * sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_meta, pieces * sizeof(CsRowMeta));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->wire_off, (rows + 1) * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->vp_listed, (size_t)max_batch * sizeof(int));
     ctx->max_rows = (long long)rows;
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->status, sizeof(unsigned));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->slow_rows, 2 * sizeof(unsigned long long));   // [0] slow rows, [1] redo rows
@@ -368,6 +381,7 @@ int picospec_destroy(picospec_ctx* ctx) {
     cudaFree(ctx->surv_keys);
     cudaFree(ctx->surv_meta);
     cudaFree(ctx->wire_off);
+    cudaFree(ctx->vp_listed);
     cudaFree(ctx->status);
     cudaFree(ctx->slow_rows);
     free(ctx);
@@ -700,6 +714,187 @@ int picospec_edge_resample(picospec_ctx* ctx, const void* draft_logits, picospec
     a.accept_len = nullptr; a.p_draft = nullptr; a.resid_mass = nullptr; a.borderline = nullptr;
     a.token = token; a.mass = mass;
     return verify_common(ctx, a, dtype, cuda_stream, true);
+}
+
+// ---- vocabulary-parallel verification ---------------------------------------------------------
+
+static int vp_check(const picospec_ctx* ctx, int B, int G, int V, int k_max, int ranks, int chunks_per_rank) {
+    if (!ctx) return PICOSPEC_EINVAL;
+    if (B < 0 || G < 0 || V <= 0 || k_max <= 0 || ranks < 1 || chunks_per_rank < 1) return PICOSPEC_EINVAL;
+    const long long nch = ((long long)V + CHUNK - 1) / CHUNK;
+    if ((long long)(ranks - 1) * chunks_per_rank >= nch || (long long)ranks * chunks_per_rank < nch) return PICOSPEC_EINVAL;
+    if (B > ctx->max_batch || G > ctx->max_gamma || V > ctx->max_vocab || k_max > ctx->max_k) return PICOSPEC_ECAPACITY;
+    return PICOSPEC_OK;
+}
+
+// the fields every vocabulary-parallel launch shares
+static void vp_args(picospec_ctx* ctx, VerifyArgs& a, int B, int G, int V, int k_max, int chunks_per_rank) {
+    a.B = B; a.G = G; a.V = V; a.k_max = k_max; a.sample_only = 0;
+    a.nch = (V + CHUNK - 1) / CHUNK;
+    a.r0 = 0; a.r1 = G + 1;
+    a.chunks_per_rank = chunks_per_rank;
+    a.rank_stride = (long long)B * (G + 1) * chunks_per_rank;
+    a.row_max = ctx->row_max; a.queue = ctx->queue; a.need_rows = ctx->need_rows;
+    a.queue_count = ctx->counters; a.status = ctx->status; a.slow_rows = ctx->slow_rows;
+    a.pos = nullptr; a.mass = nullptr; a.token = nullptr;
+    a.draft_tok = nullptr; a.q_idx = nullptr; a.q_prob = nullptr; a.q_count = nullptr;
+    a.u_accept = nullptr; a.u_resample = nullptr; a.accept_len = nullptr; a.p_draft = nullptr;
+    a.resid_mass = nullptr; a.borderline = nullptr; a.temperature = nullptr;
+    a.logits = nullptr; a.row_stride = 0; a.stats = nullptr; a.dsum = nullptr;
+}
+
+int picospec_vp_local(picospec_ctx* ctx, const void* slice_logits, picospec_dtype dtype, int B, int G, int Vs, int v0,
+                      long long row_stride_elems, int chunks_per_rank, const float* temperature, const int* draft_tok,
+                      const int* q_idx, const int* q_count, int k_max, float* records_local, float* entries_local,
+                      void* cuda_stream) {
+    if (!ctx || !slice_logits || !temperature || !records_local) return PICOSPEC_EINVAL;
+    if (dtype != PICOSPEC_F32 && dtype != PICOSPEC_BF16) return PICOSPEC_EINVAL;
+    if (B < 0 || G < 0 || Vs <= 0 || v0 < 0 || v0 % CHUNK != 0 || k_max <= 0 || row_stride_elems < Vs) return PICOSPEC_EINVAL;
+    const int slice_chunks = (Vs + CHUNK - 1) / CHUNK;
+    if (chunks_per_rank < slice_chunks) return PICOSPEC_EINVAL;
+    if (G > 0 && (!draft_tok || !q_idx || !q_count || !entries_local)) return PICOSPEC_EINVAL;
+    if (B > ctx->max_batch || G > ctx->max_gamma || (long long)v0 + Vs > ctx->max_vocab || k_max > ctx->max_k)
+        return PICOSPEC_ECAPACITY;
+    if (B == 0) return PICOSPEC_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
+    VerifyArgs a;
+    vp_args(ctx, a, B, G, Vs, k_max, 0);
+    a.rank_stride = 0;
+    a.logits = slice_logits; a.row_stride = row_stride_elems; a.temperature = temperature;
+    a.draft_tok = draft_tok; a.q_idx = q_idx; a.q_count = q_count;
+    a.stats = reinterpret_cast<float2*>(records_local);
+    a.stats_pitch = chunks_per_rank;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e;
+    if (dtype == PICOSPEC_BF16) {
+        e = launch_verify_stream<__nv_bfloat16>(ctx, a, rows_aligned(slice_logits, row_stride_elems, 2), s);
+        if (e == cudaSuccess && G > 0)
+            launch_chained(vp_gather_kernel<__nv_bfloat16>, ctx->num_sms * 4, THREADS, 0, s, a, v0, Vs, entries_local);
+    } else {
+        e = launch_verify_stream<float>(ctx, a, rows_aligned(slice_logits, row_stride_elems, 4), s);
+        if (e == cudaSuccess && G > 0)
+            launch_chained(vp_gather_kernel<float>, ctx->num_sms * 4, THREADS, 0, s, a, v0, Vs, entries_local);
+    }
+    if (e == cudaSuccess) e = cudaGetLastError();
+    return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
+}
+
+int picospec_vp_decide(picospec_ctx* ctx, int B, int G, int V, int ranks, int chunks_per_rank, const float* records_all,
+                       const double* sums_all, const float* entries_all, const float* temperature, const int* draft_tok,
+                       const int* q_idx, const float* q_prob, const int* q_count, int k_max, const float* u_accept,
+                       const float* u_resample, int* accept_len, float* p_draft, float* resid_mass,
+                       int* borderline_count, int* pick, void* cuda_stream) {
+    int rc = vp_check(ctx, B, G, V, k_max, ranks, chunks_per_rank);
+    if (rc != PICOSPEC_OK) return rc;
+    if (!records_all || !temperature || !accept_len || !borderline_count || !pick || !u_resample) return PICOSPEC_EINVAL;
+    if (G > 0 && (!entries_all || !draft_tok || !q_idx || !q_prob || !q_count || !u_accept || !p_draft || !resid_mass))
+        return PICOSPEC_EINVAL;
+    if (B == 0) return PICOSPEC_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
+    VerifyArgs a;
+    vp_args(ctx, a, B, G, V, k_max, chunks_per_rank);
+    a.temperature = temperature; a.draft_tok = draft_tok; a.q_idx = q_idx; a.q_prob = q_prob; a.q_count = q_count;
+    a.u_accept = u_accept; a.u_resample = u_resample;
+    a.accept_len = accept_len; a.p_draft = p_draft; a.resid_mass = resid_mass; a.borderline = borderline_count;
+    a.stats = reinterpret_cast<float2*>(const_cast<float*>(records_all));
+    a.dsum = const_cast<double*>(sums_all);
+    a.entry_logits = entries_all; a.pick = pick;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const size_t dyn = (size_t)a.nch * sizeof(double);
+    cudaError_t e = cudaSuccess;
+    if (!sums_all) {
+        e = cudaMemsetAsync(borderline_count, 0, sizeof(int), s);
+        if (e == cudaSuccess) launch_chained(verify_finish_kernel<float, false>, B, THREADS, dyn, s, a);
+    } else {
+        const int g2 = B < ctx->num_sms ? B : ctx->num_sms;
+        launch_chained(verify_finish_kernel<float, true>, g2, THREADS, dyn, s, a);
+    }
+    if (e == cudaSuccess) e = cudaGetLastError();
+    return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
+}
+
+int picospec_vp_draw(picospec_ctx* ctx, const void* slice_logits, picospec_dtype dtype, int B, int G, int V, int v0,
+                     long long row_stride_elems, int rank, int ranks, int chunks_per_rank, const float* records_all,
+                     const double* sums_all, const float* temperature, const int* q_idx, const float* q_prob,
+                     const int* q_count, int k_max, const float* u_resample, const int* pick, int* tok_flag_local,
+                     void* cuda_stream) {
+    int rc = vp_check(ctx, B, G, V, k_max, ranks, chunks_per_rank);
+    if (rc != PICOSPEC_OK) return rc;
+    if (!slice_logits || !records_all || !temperature || !u_resample || !pick || !tok_flag_local) return PICOSPEC_EINVAL;
+    if (dtype != PICOSPEC_F32 && dtype != PICOSPEC_BF16) return PICOSPEC_EINVAL;
+    if (rank < 0 || rank >= ranks || v0 != rank * chunks_per_rank * CHUNK) return PICOSPEC_EINVAL;
+    if (G > 0 && (!q_idx || !q_prob || !q_count)) return PICOSPEC_EINVAL;
+    if (B == 0) return PICOSPEC_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
+    VerifyArgs a;
+    vp_args(ctx, a, B, G, V, k_max, chunks_per_rank);
+    a.logits = slice_logits; a.row_stride = row_stride_elems; a.temperature = temperature;
+    a.q_idx = q_idx; a.q_prob = q_prob; a.q_count = q_count; a.u_resample = u_resample;
+    a.stats = reinterpret_cast<float2*>(const_cast<float*>(records_all));
+    a.dsum = const_cast<double*>(sums_all);
+    a.pick = const_cast<int*>(pick);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (dtype == PICOSPEC_BF16) {
+        if (sums_all) launch_chained(vp_draw_kernel<__nv_bfloat16, true>, B, THREADS, 0, s, a, v0, rank, ctx->vp_listed, tok_flag_local);
+        else launch_chained(vp_draw_kernel<__nv_bfloat16, false>, B, THREADS, 0, s, a, v0, rank, ctx->vp_listed, tok_flag_local);
+    } else {
+        if (sums_all) launch_chained(vp_draw_kernel<float, true>, B, THREADS, 0, s, a, v0, rank, ctx->vp_listed, tok_flag_local);
+        else launch_chained(vp_draw_kernel<float, false>, B, THREADS, 0, s, a, v0, rank, ctx->vp_listed, tok_flag_local);
+    }
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
+}
+
+int picospec_vp_queue(picospec_ctx* ctx, int B, const int* pick, const int* tok_flag_all, int* token, void* cuda_stream) {
+    if (!ctx || B < 0 || !pick || !tok_flag_all || !token) return PICOSPEC_EINVAL;
+    if (B > ctx->max_batch) return PICOSPEC_ECAPACITY;
+    if (B == 0) return PICOSPEC_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
+    VerifyArgs a;
+    vp_args(ctx, a, B, 0, 1, 1, 1);
+    a.pick = const_cast<int*>(pick);
+    a.token = token;
+    launch_chained(vp_queue_kernel, 1, THREADS, 0, (cudaStream_t)cuda_stream, a, tok_flag_all, ctx->vp_listed);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
+}
+
+int picospec_vp_exact(picospec_ctx* ctx, const void* slice_logits, picospec_dtype dtype, int B, int G, int Vs,
+                      long long row_stride_elems, int chunks_per_rank, const float* temperature, double* sums_local,
+                      void* cuda_stream) {
+    if (!ctx || !slice_logits || !temperature || !sums_local) return PICOSPEC_EINVAL;
+    if (dtype != PICOSPEC_F32 && dtype != PICOSPEC_BF16) return PICOSPEC_EINVAL;
+    if (B < 0 || G < 0 || Vs <= 0 || row_stride_elems < Vs || chunks_per_rank < (Vs + CHUNK - 1) / CHUNK) return PICOSPEC_EINVAL;
+    if (B > ctx->max_batch || G > ctx->max_gamma) return PICOSPEC_ECAPACITY;
+    if (B == 0) return PICOSPEC_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
+    PreciseArgs p;
+    p.logits = slice_logits; p.row_stride = row_stride_elems; p.V = Vs; p.nch = (Vs + CHUNK - 1) / CHUNK;
+    p.seq_rows = G + 1; p.expand = G + 1; p.pos = nullptr; p.temperature = temperature;
+    p.queue = ctx->queue; p.queue_count = ctx->counters; p.need_rows = ctx->need_rows;
+    p.row_max = ctx->row_max; p.dsum = sums_local; p.pitch = chunks_per_rank;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (dtype == PICOSPEC_BF16) launch_chained(precise_chunk_sums_kernel<__nv_bfloat16>, ctx->num_sms * 6, THREADS, 0, s, p);
+    else launch_chained(precise_chunk_sums_kernel<float>, ctx->num_sms * 6, THREADS, 0, s, p);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
+}
+
+int picospec_vp_merge(picospec_ctx* ctx, int B, const int* tok_flag_all, int* token, void* cuda_stream) {
+    if (!ctx || B < 0 || !tok_flag_all || !token) return PICOSPEC_EINVAL;
+    if (B > ctx->max_batch) return PICOSPEC_ECAPACITY;
+    if (B == 0) return PICOSPEC_OK;
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
+    launch_chained(vp_merge_kernel, (B + THREADS - 1) / THREADS, THREADS, 0, (cudaStream_t)cuda_stream, B, ctx->vp_listed,
+                   tok_flag_all, token);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
 }
 
 }  // extern "C"

@@ -23,6 +23,7 @@ struct PreciseArgs {
     const int* gamma = nullptr;
     const float* row_max;      // [rows] exact row maxima from the fp32 pass
     double* dsum;              // [rows, nch]
+    int pitch = 0;             // chunk sums per row in dsum (0: nch)
 };
 
 template <typename T>
@@ -79,7 +80,7 @@ __global__ void __launch_bounds__(THREADS) precise_chunk_sums_kernel(PreciseArgs
         if (lane == 0) part[warp] = s;
         __syncthreads();
         if (work && quarter == 0 && lane == 0)
-            a.dsum[(long long)src_row * a.nch + c] = (part[warp] + part[warp + 1]) + (part[warp + 2] + part[warp + 3]);
+            a.dsum[(long long)src_row * (a.pitch > 0 ? a.pitch : a.nch) + c] = (part[warp] + part[warp + 1]) + (part[warp + 2] + part[warp + 3]);
         __syncthreads();
     }
 }

@@ -32,6 +32,18 @@ struct VerifyArgs {
     int* borderline;           // [1]
     int* token;                // [B] or null
     float* mass;               // [B] or null (sample_only)
+    // Vocabulary-parallel verification (the logits are sharded along the vocabulary over several
+    // ranks): the chunk records of all ranks lie rank after rank, [ranks, rows, chunks_per_rank], and
+    // chunk c of the vocabulary is record c % chunks_per_rank of rank c / chunks_per_rank; one rank,
+    // chunks_per_rank = nch is the plain layout.  entry_logits, if set, holds the target logits at the
+    // stored entries (slots 0 .. k_max - 1) and at the drafted token (slot k_max) of every draft
+    // position, gathered from the ranks that own them: the finish kernel then reads no logits itself
+    // and hands the draw inside the picked chunk to that chunk's owner through `pick`.
+    int chunks_per_rank = 0;        // 0: nch
+    long long rank_stride = 0;      // records between two ranks' blocks
+    int stats_pitch = 0;            // records per row written by the streaming pass (0: nch)
+    const float* entry_logits = nullptr;   // [B*G, k_max + 1]
+    int* pick = nullptr;            // [B, 4]: sampled row, picked chunk (-1: none), flags, unused
     // workspace
     float2* stats;             // [B*(G+1), nch]: (chunk max logit, sum of 2^(l*c32 - max*c32))
     float* row_max;            // [B*(G+1)]
@@ -69,6 +81,15 @@ __device__ __forceinline__ bool streamed_row(const VerifyArgs& a, int r, int& b,
     return true;
 }
 
+// index of the record of (row, chunk c of the vocabulary) in stats / dsum
+__device__ __forceinline__ long long record_index(const VerifyArgs& a, int row, int c) {
+    const int L = a.chunks_per_rank > 0 ? a.chunks_per_rank : a.nch;
+    const int r = c / L;
+    return (long long)r * a.rank_stride + (long long)row * L + (c - r * L);
+}
+// flags of VerifyArgs::pick
+constexpr int PICK_RESIDUAL = 1, PICK_FLAGGED = 2, PICK_DRAW_ONLY = 4, PICK_MASS_ONLY = 8;
+
 template <typename T> __device__ __forceinline__ ItemMeta<T> decode_item(const VerifyArgs& a, long long item) {
     ItemMeta<T> m;
     const int r = (int)(item / a.nch);
@@ -88,7 +109,7 @@ template <typename T> __device__ __forceinline__ ItemMeta<T> decode_item(const V
     m.c32 = temp_scale(Tb);
     m.row = reinterpret_cast<const T*>(a.logits) + (long long)src_row * a.row_stride;
     m.v0 = c * CHUNK;
-    m.slot = (long long)src_row * a.nch + c;
+    m.slot = (long long)src_row * (a.stats_pitch > 0 ? a.stats_pitch : a.nch) + c;
     return m;
 }
 
@@ -255,7 +276,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, StreamCfg<T>::CTAS_PER_SM) chu
                 const float cm = warp_max_redux(regs.lane_max_plain());
                 const float off = cm > -CUDART_INF_F ? __fmul_rn(cm, d.c32) : 0.f;
                 const float sum = warp_sum(lane_exp_sum2(regs, d.c32, off));
-                if (lane == 0) a.stats[(long long)d.src_row * a.nch + c] = make_float2(cm, sum);
+                if (lane == 0) a.stats[(long long)d.src_row * (a.stats_pitch > 0 ? a.stats_pitch : a.nch) + c] = make_float2(cm, sum);
             }
         }
     }
@@ -294,14 +315,14 @@ __device__ __forceinline__ void row_stats(const VerifyArgs& a, int src_row, floa
     if (exact) {
         mx = a.row_max[src_row];
         double s = 0.0;
-        for (int c = lane; c < a.nch; c += 32) s += a.dsum[(long long)src_row * a.nch + c];
+        for (int c = lane; c < a.nch; c += 32) s += a.dsum[record_index(a, src_row, c)];
         Z = warp_sum(s);
     } else {
-        const float2* st = a.stats + (long long)src_row * a.nch;
+        const float2* st = a.stats;
         float m = -CUDART_INF_F;
         bool nan = false;
         for (int c = lane; c < a.nch; c += 32) {
-            float2 v = st[c];
+            float2 v = st[record_index(a, src_row, c)];
             m = fmaxf(m, v.x);
             nan |= (v.y != v.y);
         }
@@ -313,7 +334,7 @@ __device__ __forceinline__ void row_stats(const VerifyArgs& a, int src_row, floa
         if (!bad) {
             const double off = (double)__fmul_rn(m, c32);
             for (int c = lane; c < a.nch; c += 32) {
-                float2 v = st[c];
+                float2 v = st[record_index(a, src_row, c)];
                 if (v.x > -CUDART_INF_F) s += (double)v.y * exp2((double)__fmul_rn(v.x, c32) - off);
             }
         }
@@ -321,6 +342,74 @@ __device__ __forceinline__ void row_stats(const VerifyArgs& a, int src_row, floa
         if (!(Zraw > 0.0)) bad = true;
         Z = bad ? 0.0 : Zraw * stream_sum_scale(m, c32);
     }
+}
+
+// Level 2 of the sampler, by the 256 threads of a CTA: the token inside chunk `cs` of a row whose
+// logits start at `row` with vocabulary index `vbase` (0 for a whole row; the first index of the
+// slice when the vocabulary is sharded).  Weights are max(0, p - q~) with the stored entries
+// (idx, prob)[0 .. n) if use_resid, else p.  Sets sh.flag when the fast pass cannot call the draw.
+template <typename T, bool PRECISE>
+__device__ __forceinline__ int level2_draw(const VerifyArgs& a, const T* row, int vbase, int cs, const int* idx,
+                                           const float* prob, int n, bool use_resid, const Weight<PRECISE>& wt,
+                                           double invZ, float u2, FinishShared& sh) {
+    const int tid = threadIdx.x;
+    // the 1024 entries of chunk cs, four consecutive entries per thread
+    const int v0 = cs * CHUNK;
+    for (int k = tid; k < CHUNK; k += THREADS) sh.qloc[k] = 0.f;
+    if (tid == 0) {
+        sh.tok = 0x7fffffff;
+        sh.last = -1;
+    }
+    __syncthreads();
+    if (use_resid)
+        for (int k = tid; k < n; k += THREADS) {
+            const int v = idx[k];
+            if (v >= v0 && v < v0 + CHUNK) sh.qloc[v - v0] = prob[k];
+        }
+    __syncthreads();
+    double r[4], cum[4], qsum = 0.0, loc = 0.0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int v = v0 + tid * 4 + e;
+        double w = 0.0;
+        if (v < a.V) w = wt(load_logit(row, v - vbase)) * invZ;
+        const double q = (double)sh.qloc[tid * 4 + e];
+        qsum += q;
+        double d = w - q;
+        r[e] = d > 0.0 ? d : 0.0;
+        loc += r[e];
+        cum[e] = loc;
+    }
+    double M;
+    const double incl = block_scan_incl(loc, sh.warp_tot, M);
+    const double base = incl - loc;
+    double Q;
+    block_scan_incl(qsum, sh.warp_tot, Q);
+    const double thr2 = (double)u2 * M;
+    int mine = 0x7fffffff, mylast = -1;
+#pragma unroll
+    for (int e = 3; e >= 0; --e) {
+        if (base + cum[e] > thr2) mine = v0 + tid * 4 + e;
+        if (r[e] > 0.0 && mylast < 0) mylast = v0 + tid * 4 + e;
+    }
+    if (mine != 0x7fffffff) atomicMin(&sh.tok, mine);
+    if (mylast >= 0) atomicMax(&sh.last, mylast);
+    __syncthreads();
+    const int token = sh.tok != 0x7fffffff ? sh.tok : sh.last;
+    if (!PRECISE && use_resid && Q > 0.0) {
+        // with q~ present the thresholds depend on the normaliser: error <= GUARD_Z * Q
+        const double E2 = 2.0 * GUARD_Z * Q;
+        if (sh.tok == 0x7fffffff) {
+            if (tid == 0) sh.flag = 1;
+        } else if (mine == sh.tok) {
+            const int e = mine - (v0 + tid * 4);
+            const double hi = base + cum[e] - thr2;
+            const double lo = thr2 - (base + cum[e] - r[e]);
+            if (hi < E2 || lo < E2) sh.flag = 1;
+        }
+    }
+    __syncthreads();
+    return token;
 }
 
 template <typename T, bool PRECISE>
@@ -424,7 +513,8 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 float qx = 0.f, qx_mine = 0.f;
                 int kx = 0x7fffffff;
                 // p(x) on every lane (the same instructions as on one lane, and no divergent tail)
-                const float lx = range_bad ? -CUDART_INF_F : load_logit(row, x);
+                const float* ent = a.entry_logits ? a.entry_logits + (long long)ri * (a.k_max + 1) : nullptr;
+                const float lx = range_bad ? -CUDART_INF_F : (ent ? ent[a.k_max] : load_logit(row, x));
                 if (!range_bad) {
                     for (int k0 = 0; k0 < n; k0 += 256) {
                         if (k0 > 0) {
@@ -440,7 +530,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                             if (k0 + u * 32 + lane >= n) vv[u] = -2;
                             const bool ok = vv[u] >= 0 && vv[u] < a.V;
                             if (vv[u] != -2 && !ok) range_bad = true;
-                            ll[u] = ok ? load_logit(row, vv[u]) : -CUDART_INF_F;
+                            ll[u] = ok ? (ent ? ent[k0 + u * 32 + lane] : load_logit(row, vv[u])) : -CUDART_INF_F;
                         }
 #pragma unroll
                         for (int u = 0; u < 8; ++u) {
@@ -521,8 +611,10 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
 
         // ---- 4. residual / bonus sample --------------------------------------------------
         int token = -1;
+        int pick_row = 0, pick_chunk = -1;      // vocabulary-parallel: what the picked chunk's owner needs
+        bool pick_resid = false;
         double Rtot = -1.0;
-        const bool want_token = a.token != nullptr;
+        const bool want_token = a.token != nullptr || a.pick != nullptr;
         if (!st_bits && want_token && decided) {
             const int j = a.sample_only ? jpos : alen;
             const int rj = b * G + j;
@@ -545,13 +637,12 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
             for (int pass = 0; pass < 2 && !st_bits; ++pass) {
                 // chunk masses (in units where the row sums to one)
                 if (PRECISE && row_needed(need, j)) {
-                    for (int c = tid; c < a.nch; c += THREADS) cm[c] = a.dsum[(long long)(b * G1 + j) * a.nch + c] * invZ;
+                    for (int c = tid; c < a.nch; c += THREADS) cm[c] = a.dsum[record_index(a, b * G1 + j, c)] * invZ;
                 } else {
-                    const float2* st = a.stats + (long long)(b * G1 + j) * a.nch;
                     const double off = (double)__fmul_rn(sh.mx[j], c32);
                     const double Zraw = sh.Zraw[j];
                     for (int c = tid; c < a.nch; c += THREADS) {
-                        float2 v = st[c];
+                        float2 v = a.stats[record_index(a, b * G1 + j, c)];
                         cm[c] = v.x > -CUDART_INF_F ? (double)v.y * exp2((double)__fmul_rn(v.x, c32) - off) / Zraw : 0.0;
                     }
                 }
@@ -568,11 +659,12 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                             vv[u] = k < n ? idx[k] : -2;
                             qq[u] = k < n ? prob[k] : 0.f;
                         }
+                        const float* ent = a.entry_logits ? a.entry_logits + (long long)rj * (a.k_max + 1) : nullptr;
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
                             const bool ok = vv[u] >= 0 && vv[u] < a.V;
                             if (vv[u] != -2 && !ok) rb = true;
-                            ll[u] = ok ? load_logit(row, vv[u]) : -CUDART_INF_F;
+                            ll[u] = ok ? (ent ? ent[tid + u * THREADS] : load_logit(row, vv[u])) : -CUDART_INF_F;
                         }
 #pragma unroll
                         for (int u = 0; u < 4; ++u)
@@ -643,63 +735,12 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
             }
             st_bits |= (unsigned)sh.bad;
             const int cs = st_bits ? -1 : sh.cstar;
-            if (!st_bits && cs >= 0) {
-                // level 2: the 1024 entries of chunk cs, four consecutive entries per thread
-                const int v0 = cs * CHUNK;
-                for (int k = tid; k < CHUNK; k += THREADS) sh.qloc[k] = 0.f;
-                if (tid == 0) {
-                    sh.tok = 0x7fffffff;
-                    sh.last = -1;
-                }
-                __syncthreads();
-                if (use_resid)
-                    for (int k = tid; k < n; k += THREADS) {
-                        const int v = idx[k];
-                        if (v >= v0 && v < v0 + CHUNK) sh.qloc[v - v0] = prob[k];
-                    }
-                __syncthreads();
-                double r[4], cum[4], qsum = 0.0, loc = 0.0;
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int v = v0 + tid * 4 + e;
-                    double w = 0.0;
-                    if (v < a.V) w = wt(load_logit(row, v)) * invZ;
-                    const double q = (double)sh.qloc[tid * 4 + e];
-                    qsum += q;
-                    double d = w - q;
-                    r[e] = d > 0.0 ? d : 0.0;
-                    loc += r[e];
-                    cum[e] = loc;
-                }
-                double M;
-                const double incl = block_scan_incl(loc, sh.warp_tot, M);
-                const double base = incl - loc;
-                double Q;
-                block_scan_incl(qsum, sh.warp_tot, Q);
-                const double thr2 = (double)a.u_resample[2 * b + 1] * M;
-                int mine = 0x7fffffff, mylast = -1;
-#pragma unroll
-                for (int e = 3; e >= 0; --e) {
-                    if (base + cum[e] > thr2) mine = v0 + tid * 4 + e;
-                    if (r[e] > 0.0 && mylast < 0) mylast = v0 + tid * 4 + e;
-                }
-                if (mine != 0x7fffffff) atomicMin(&sh.tok, mine);
-                if (mylast >= 0) atomicMax(&sh.last, mylast);
-                __syncthreads();
-                token = sh.tok != 0x7fffffff ? sh.tok : sh.last;
-                if (!PRECISE && use_resid && Q > 0.0) {
-                    // with q~ present the thresholds depend on the normaliser: error <= GUARD_Z * Q
-                    const double E2 = 2.0 * GUARD_Z * Q;
-                    if (sh.tok == 0x7fffffff) {
-                        if (tid == 0) sh.flag = 1;
-                    } else if (mine == sh.tok) {
-                        const int e = mine - (v0 + tid * 4);
-                        const double hi = base + cum[e] - thr2;
-                        const double lo = thr2 - (base + cum[e] - r[e]);
-                        if (hi < E2 || lo < E2) sh.flag = 1;
-                    }
-                }
-                __syncthreads();
+            pick_row = j;
+            pick_chunk = cs;
+            pick_resid = use_resid;
+            if (!st_bits && cs >= 0 && !a.pick) {
+                token = level2_draw<T, PRECISE>(a, row, 0, cs, idx, prob, n, use_resid, wt, invZ,
+                                                a.u_resample[2 * b + 1], sh);
             }
             flagged |= sh.flag != 0;
         }
@@ -716,18 +757,28 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                     }
                     if (a.state_out) a.state_out[b] = 0;
                 }
-                if (want_token) a.token[b] = -1;
+                if (a.token) a.token[b] = -1;
+                if (a.pick) {
+                    a.pick[4 * b + 0] = 0;
+                    a.pick[4 * b + 1] = -1;
+                    a.pick[4 * b + 2] = 0;
+                }
                 if (a.mass) a.mass[b] = -1.f;
             } else {
                 if (!a.sample_only) {
                     a.accept_len[b] = decided ? alen : -2;
                     if (a.state_out) a.state_out[b] = decided ? 0 : 1;
                 }
-                if (want_token) a.token[b] = decided ? token : -2;
+                if (a.token) a.token[b] = decided ? token : -2;
                 if (a.mass) a.mass[b] = (float)Rtot;
                 if (PRECISE) {
                     if (nborder && a.borderline) atomicAdd(a.borderline, nborder);
-                } else if (flagged) {
+                    if (a.pick) {
+                        a.pick[4 * b + 0] = pick_row;
+                        a.pick[4 * b + 1] = (decided && want_token) ? pick_chunk : -1;
+                        a.pick[4 * b + 2] = pick_resid ? PICK_RESIDUAL : 0;
+                    }
+                } else if (flagged || a.pick) {
                     // Which rows need exact sums: an ambiguous accept test can move the first
                     // rejection anywhere from its position on, so every row from there; an ambiguous
                     // draw needs the sampled row only; a small residual mass its own row.
@@ -747,8 +798,10 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                         draw_only_flag = first_amb < 0 && !any_small;
                         mass_only_flag = first_amb < 0 && any_small && !sh.flag;
                         for (int i = lo; i < row_hi; ++i) {
+                            // (vocabulary-parallel: whether the draw inside the chunk is too close to call is
+                            // only known to the chunk's owner later, so the sampled row is always listed)
                             const bool nr = i >= 64 || (first_amb >= 0 && i >= first_amb) || (i < hi && sh.small[i]) ||
-                                            (sh.flag && want_token && decided && i == alen);
+                                            ((sh.flag || a.pick) && want_token && decided && i == alen);
                             if (nr) {
                                 if (i < 64) nd |= 1ull << i;
                                 ++nrows;
@@ -756,9 +809,18 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                         }
                     }
                     a.need_rows[b] = nd;
-                    const int q = atomicAdd(a.queue_count, 1);
-                    a.queue[q] = b | (draw_only_flag ? QUEUE_DRAW_ONLY : 0) | (mass_only_flag ? QUEUE_MASS_ONLY : 0);
-                    atomicAdd(a.slow_rows, (unsigned long long)nrows);
+                    if (a.pick) {
+                        // the queue is built once the owners' flags have been exchanged
+                        a.pick[4 * b + 0] = pick_row;
+                        a.pick[4 * b + 1] = (decided && want_token) ? pick_chunk : -1;
+                        a.pick[4 * b + 2] = (pick_resid ? PICK_RESIDUAL : 0) | (flagged ? PICK_FLAGGED : 0) |
+                                            (draw_only_flag ? PICK_DRAW_ONLY : 0) | (mass_only_flag ? PICK_MASS_ONLY : 0);
+                        a.pick[4 * b + 3] = nrows;
+                    } else {
+                        const int q = atomicAdd(a.queue_count, 1);
+                        a.queue[q] = b | (draw_only_flag ? QUEUE_DRAW_ONLY : 0) | (mass_only_flag ? QUEUE_MASS_ONLY : 0);
+                        atomicAdd(a.slow_rows, (unsigned long long)nrows);
+                    }
                 }
             }
         }

@@ -141,6 +141,62 @@ def test_sequence_sharding_world_size_2_gloo(tmp_path):
     assert "SHARD_OK" in run.stdout
 
 
+_VP_WORKER = r'''
+import os, sys
+sys.path.insert(0, sys.argv[1])
+import numpy as np, torch, torch.distributed as dist
+import gen, oracle
+from oracle import vocab_parallel as ovp
+from paper_2603_19133_b200 import vocab_parallel as vp
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+w = gen.Workload("t", V=5120 + 300, B=5, G=3, dtype="f32", s=1.1, sigma_d=1.5, corr=0.8, sigma_t=1.0, T=None,
+                 top_k=0, top_p=0.9, k_max=24)
+inp = gen.make_inputs(w, 21)                       # every rank generates the same global batch ...
+f = lambda t: t.float().numpy() if t.is_floating_point() else t.numpy()
+T = f(inp["temperature"])
+qi, qp, qc, tok = oracle.compress(f(inp["draft_logits"]), T, w.top_k, w.top_p, w.k_max, f(inp["u_draft"]))
+v0, v1 = vp.slice_bounds(w.V, world, rank)         # ... and keeps its own slice of the target logits only
+sl = np.ascontiguousarray(f(inp["target_logits"])[:, :, v0:v1])
+cpr = vp.chunks_per_rank(w.V, world)
+exch = vp.DistExchange()
+# the CPU stand-in for the per-rank kernels, the product's exchanges between them
+m, s = ovp.slice_records(sl, T)
+pad = cpr - m.shape[-1]
+rec = np.stack([np.pad(m, ((0, 0), (0, 0), (0, pad)), constant_values=-np.inf), np.pad(s, ((0, 0), (0, 0), (0, pad)))], -1)
+(rec_all,) = exch.gather([torch.from_numpy(rec)])                       # [world, B, G+1, cpr, 2]
+(ent_all,) = exch.maximum([torch.from_numpy(ovp.slice_entries(sl, v0, tok, qi, qc))])
+nch = (w.V + 1023) // 1024
+ra = rec_all.numpy()
+m_all = np.concatenate([ra[r, ..., 0] for r in range(world)], -1)[..., :nch]
+s_all = np.concatenate([ra[r, ..., 1] for r in range(world)], -1)[..., :nch]
+owner = np.arange(nch) // cpr
+d = ovp.decide(m_all, s_all, ent_all.numpy(), T, tok, qi, qp, qc, f(inp["u_accept"]), f(inp["u_resample"]), owner)
+mine = ovp.draw_in_slice(sl, v0, rank, d, T, qi, qp, qc, f(inp["u_resample"]))
+(token,) = exch.maximum([torch.from_numpy(mine)])
+ref = oracle.verify(f(inp["target_logits"]), T, tok, qi, qp, qc, f(inp["u_accept"]), f(inp["u_resample"]))
+assert np.array_equal(d["accept_len"], ref["accept_len"]) and np.array_equal(token.numpy(), ref["token"])
+assert (mine >= 0).sum() < w.B or world == 1      # no rank owns every picked chunk
+np.testing.assert_allclose(d["p_draft"], ref["p_draft"], rtol=1e-12)
+if rank == 0:
+    print("VP_OK")
+dist.destroy_process_group()
+'''
+
+
+def test_vocabulary_parallel_exchange_world_size_2_gloo(tmp_path):
+    # the product's exchange code (all-gather of chunk records, element-wise maximum of gathered logits and
+    # of tokens) between two gloo ranks on CPU tensors, with the oracle's per-slice routines standing in for
+    # the kernels: the result equals plain verification of the whole vocabulary
+    script = tmp_path / "vp_worker.py"
+    script.write_text(_VP_WORKER)
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", "29573", str(script), ROOT]
+    run = subprocess.run(cmd, capture_output=True, text=True, timeout=300)
+    assert run.returncode == 0, run.stdout[-2000:] + run.stderr[-2000:]
+    assert "VP_OK" in run.stdout
+
+
 def test_bench_starts_its_own_ranks_for_more_than_one_gpu():
     # `bench.py --gpus 2` without a torchrun environment starts two ranks of itself; the reference arm
     # needs no GPU (rank 0 alone times the oracle, the other rank leaves without work), so the launcher

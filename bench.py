@@ -262,9 +262,9 @@ class Step:
                       "resid_mass": torch.empty((B, G), dtype=f32, device=dev),
                       "borderline_count": torch.empty((1,), dtype=i32, device=dev),
                       "token": torch.empty((B,), dtype=i32, device=dev)}
-        # kernels per step: compress = filter, finish, redo list (+ exact sums and cut with top-p);
+        # kernels per step: compress = filter, finish, redo list (+ the double-precision cut with top-p);
         # verify = statistics, finish, exact sums, double-precision finish
-        self.launches_per_step = (5 if w.top_p < 1.0 else 3) + 4
+        self.launches_per_step = (4 if w.top_p < 1.0 else 3) + 4
 
     def compress(self, inp=None):
         inp = inp or self.inp

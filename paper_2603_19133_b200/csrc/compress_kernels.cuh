@@ -32,6 +32,7 @@ struct CompressArgs {
     int* queue;
     int* queue_count;          // zero on entry (cleared by the previous call)
     int* queue_count_next;     // cleared by this call for the next one
+    int* tickets;              // per queue slot: chunk sums completed in the double-precision pass
     unsigned* status;
     unsigned long long* slow_rows;
     // rows the staged kernel hands to the direct kernel (candidate buffer overflow)
@@ -324,7 +325,9 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
         a.q_count[row] = n;
         if (flagged) {
             a.row_max[row] = mx;
-            a.queue[atomicAdd(a.queue_count, 1)] = row;
+            const int q = atomicAdd(a.queue_count, 1);
+            a.queue[q] = row;
+            a.tickets[q] = 0;
             atomicAdd(a.slow_rows, 1ull);
         }
     }
@@ -489,37 +492,68 @@ __global__ void __launch_bounds__(THREADS, 2) compress_kernel(CompressArgs a) {
     }
 }
 
-// Double-precision redo of the top-p cut for the rows in the queue: the sorted candidates are
-// read back from q_idx, the exact normaliser from dsum.
+// Double-precision redo of the top-p cut for the rows in the queue, in one kernel: the exact chunk
+// sums of the queued rows (four warps per chunk, two chunks per CTA at a time, the whole grid sharing
+// the work) and, by the CTA that completes a row's last chunk, the cut of that row -- the sorted
+// candidates are read back from q_idx, the exact normaliser is the sum of the row's chunk sums.
+// Nothing waits (fence, then ticket); with an empty queue every CTA returns at once.
 template <typename T>
-__global__ void __launch_bounds__(THREADS) compress_precise_kernel(CompressArgs a) {
+__global__ void __launch_bounds__(THREADS) compress_precise_kernel(CompressArgs a, PreciseArgs p) {
     grid_dependency_sync();
     extern __shared__ u64 smem64[];
     u64* keep = smem64;
     __shared__ CompressShared sh;
+    __shared__ double part[WARPS];
+    __shared__ int last_slot[2];
+    const int nq = *a.queue_count;
+    if (nq == 0) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = warp >> 2, quarter = warp & 3;
     int k_eff = a.top_k > 0 ? a.top_k : a.k_max;
     if (k_eff > a.k_max) k_eff = a.k_max;
     if (k_eff > a.V) k_eff = a.V;
-    const int nq = *a.queue_count;
-    for (int slot = blockIdx.x; slot < nq; slot += gridDim.x) {
-        const int row = a.queue[slot];
-        const int b = row / a.G;
-        const T* rowp = reinterpret_cast<const T*>(a.logits) + (long long)row * a.row_stride;
-        workers_sync();
-        for (int j = tid; j < k_eff; j += THREADS) {
-            const int v = a.q_idx[(long long)row * a.k_max + j];
-            keep[j] = make_key(load_logit(rowp, v), v);
+    const long long total = (long long)nq * a.nch;
+    const long long pairs = (total + 1) / 2;
+    for (long long pi = blockIdx.x; pi < pairs; pi += gridDim.x) {
+        const long long item = 2 * pi + sub;
+        int qslot = -1;
+        const double s = precise_item_sum<T>(p, item, total, quarter, lane, qslot);
+        if (lane == 0) part[warp] = s;
+        __syncthreads();
+        if (quarter == 0 && lane == 0) {
+            int mine = -1;
+            if (item < total) {
+                precise_item_store(p, item, (part[warp] + part[warp + 1]) + (part[warp + 2] + part[warp + 3]));
+                __threadfence();
+                if (atomicAdd(&a.tickets[qslot], 1) == a.nch - 1) mine = qslot;
+            }
+            last_slot[sub] = mine;
         }
-        double s = 0.0;
-        for (int c = tid; c < a.nch; c += THREADS) s += a.dsum[(long long)row * a.nch + c];
-        s = warp_sum(s);
-        if (lane == 0) sh.wS[warp] = s;
-        workers_sync();
-        double Z = 0.0;
-        for (int w = 0; w < WARPS; ++w) Z += sh.wS[w];
-        workers_sync();
-        finish_row<true>(a, row, keep, k_eff, a.temperature[b], Z, sh);
+        __syncthreads();
+        const int l0 = last_slot[0], l1 = last_slot[1];
+        for (int which = 0; which < 2; ++which) {
+            const int slot = which ? l1 : l0;
+            if (slot < 0) continue;
+            __threadfence();
+            const int row = a.queue[slot];
+            const int b = row / a.G;
+            const T* rowp = reinterpret_cast<const T*>(a.logits) + (long long)row * a.row_stride;
+            workers_sync();
+            for (int j = tid; j < k_eff; j += THREADS) {
+                const int v = a.q_idx[(long long)row * a.k_max + j];
+                keep[j] = make_key(load_logit(rowp, v), v);
+            }
+            double z = 0.0;
+            for (int c = tid; c < a.nch; c += THREADS) z += a.dsum[(long long)row * a.nch + c];
+            z = warp_sum(z);
+            if (lane == 0) sh.wS[warp] = z;
+            workers_sync();
+            double Z = 0.0;
+            for (int w = 0; w < WARPS; ++w) Z += sh.wS[w];
+            workers_sync();
+            finish_row<true>(a, row, keep, k_eff, a.temperature[b], Z, sh);
+        }
+        __syncthreads();
     }
 }
 

@@ -46,6 +46,7 @@ struct picospec_ctx {
     CsRowMeta* surv_meta;
     int* wire_off;                  // wire codec: first entry of each row, [rows + 1]
     int* vp_listed;                 // vocabulary-parallel verify: per sequence, its kind in the double-precision pass
+    int* tickets;                   // compress: per queue slot, chunk sums completed in the double-precision cut
     long long max_rows;
     unsigned* status;
     unsigned long long* slow_rows;
@@ -220,9 +221,8 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
     p.seq_rows = a.G; p.expand = 1; p.pos = nullptr; p.temperature = a.temperature;
     p.queue = a.queue; p.queue_count = a.queue_count; p.row_max = a.row_max; p.dsum = a.dsum;
     p.need_rows = nullptr;
-    launch_chained(precise_chunk_sums_kernel<T>, ctx->num_sms * 6, THREADS, 0, s, p);
-    const int g2 = rows < ctx->num_sms ? rows : ctx->num_sms;
-    launch_chained(compress_precise_kernel<T>, g2, THREADS, MAX_K * 8, s, a);
+    // exact sums and the cut of the queued rows in one kernel
+    launch_chained(compress_precise_kernel<T>, ctx->num_sms * 6, THREADS, MAX_K * 8, s, a, p);
     return cudaGetLastError();
 }
 
@@ -290,6 +290,7 @@ void fill_compress_workspace(picospec_ctx* ctx, CompressArgs& a) {
     const int cur = 1 + (int)(ctx->compress_calls & 1ull);
     a.queue_count = ctx->counters + cur;
     a.queue_count_next = ctx->counters + (3 - cur);
+    a.tickets = ctx->tickets;
     a.redo_rows = ctx->redo_rows;
     a.redo_count = ctx->counters + 2 + cur;           // [3] / [4]
     a.redo_count_next = ctx->counters + 2 + (3 - cur);
@@ -348,6 +349,7 @@ int picospec_create(picospec_ctx** out, int device, int max_batch, int max_gamma
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->surv_meta, pieces * sizeof(CsRowMeta));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->wire_off, (rows + 1) * sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->vp_listed, (size_t)max_batch * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->tickets, rows * sizeof(int));
     ctx->max_rows = (long long)rows;
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->status, sizeof(unsigned));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->slow_rows, 2 * sizeof(unsigned long long));   // [0] slow rows, [1] redo rows
@@ -382,6 +384,7 @@ int picospec_destroy(picospec_ctx* ctx) {
     cudaFree(ctx->surv_meta);
     cudaFree(ctx->wire_off);
     cudaFree(ctx->vp_listed);
+    cudaFree(ctx->tickets);
     cudaFree(ctx->status);
     cudaFree(ctx->slow_rows);
     free(ctx);
@@ -806,10 +809,10 @@ int picospec_vp_decide(picospec_ctx* ctx, int B, int G, int V, int ranks, int ch
     cudaError_t e = cudaSuccess;
     if (!sums_all) {
         e = cudaMemsetAsync(borderline_count, 0, sizeof(int), s);
-        if (e == cudaSuccess) launch_chained(verify_finish_kernel<float, false>, B, THREADS, dyn, s, a);
+        if (e == cudaSuccess) launch_chained(verify_finish_kernel<float, false, true>, B, THREADS, dyn, s, a);
     } else {
         const int g2 = B < ctx->num_sms ? B : ctx->num_sms;
-        launch_chained(verify_finish_kernel<float, true>, g2, THREADS, dyn, s, a);
+        launch_chained(verify_finish_kernel<float, true, true>, g2, THREADS, dyn, s, a);
     }
     if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);

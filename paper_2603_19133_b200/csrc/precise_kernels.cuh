@@ -26,6 +26,63 @@ struct PreciseArgs {
     int pitch = 0;             // chunk sums per row in dsum (0: nch)
 };
 
+// One quarter of one item of the double-precision pass, by one warp.  Item = (queue entry, row of
+// the entry, chunk); returns the partial sum (0 for a row that is not wanted) and the queue slot.
+template <typename T>
+__device__ __forceinline__ double precise_item_sum(const PreciseArgs& a, long long item, long long total, int quarter,
+                                                   int lane, int& qslot) {
+    bool work = item < total;
+    int c = 0, src_row = 0;
+    qslot = -1;
+    if (work) {
+        c = (int)(item % a.nch);
+        const long long t = item / a.nch;
+        const int ri = (int)(t % a.expand);
+        qslot = (int)(t / a.expand);
+        const int e = a.queue[qslot] & 0x1FFFFFFF;     // (the verify path keeps flags above the index)
+        if (a.need_rows && !a.pos && ri < 64 && !((a.need_rows[e] >> ri) & 1ull)) work = false;
+        if (!a.pos && (ri < a.r0 || ri >= a.r1 || (a.gamma && ri > a.gamma[e]))) work = false;
+        src_row = a.pos ? e * a.seq_rows + a.pos[e] : e * a.expand + ri;
+    }
+    double s = 0.0;
+    if (work) {
+        const int b = src_row / a.seq_rows;
+        const T* row = reinterpret_cast<const T*>(a.logits) + (long long)src_row * a.row_stride;
+        // x = l * (1/T) instead of l / T: one rounding of 2^-53 more per term, far below every
+        // threshold this pass decides; four independent sums keep the exp pipeline busy
+        const double rT = 1.0 / (double)a.temperature[b];
+        const double m = (double)a.row_max[src_row] * rT;
+        const int v0 = c * CHUNK + quarter * (CHUNK / 4);
+        double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+#pragma unroll
+        for (int k = lane; k < CHUNK / 4; k += 128) {
+            const int v = v0 + k;
+            float l0 = -CUDART_INF_F, l1 = -CUDART_INF_F, l2 = -CUDART_INF_F, l3 = -CUDART_INF_F;
+            if (v < a.V) l0 = load_logit(row, v);
+            if (v + 32 < a.V) l1 = load_logit(row, v + 32);
+            if (v + 64 < a.V) l2 = load_logit(row, v + 64);
+            if (v + 96 < a.V) l3 = load_logit(row, v + 96);
+            s0 += exp((double)l0 * rT - m);
+            s1 += exp((double)l1 * rT - m);
+            s2 += exp((double)l2 * rT - m);
+            s3 += exp((double)l3 * rT - m);
+        }
+        s = warp_sum((s0 + s1) + (s2 + s3));
+    }
+    return s;
+}
+// where the sum of an item goes (rows that are not wanted are not written)
+__device__ __forceinline__ void precise_item_store(const PreciseArgs& a, long long item, double sum) {
+    const int c = (int)(item % a.nch);
+    const long long t = item / a.nch;
+    const int ri = (int)(t % a.expand);
+    const int e = a.queue[(int)(t / a.expand)] & 0x1FFFFFFF;
+    if (a.need_rows && !a.pos && ri < 64 && !((a.need_rows[e] >> ri) & 1ull)) return;
+    if (!a.pos && (ri < a.r0 || ri >= a.r1 || (a.gamma && ri > a.gamma[e]))) return;
+    const int src_row = a.pos ? e * a.seq_rows + a.pos[e] : e * a.expand + ri;
+    a.dsum[(long long)src_row * (a.pitch > 0 ? a.pitch : a.nch) + c] = sum;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(THREADS) precise_chunk_sums_kernel(PreciseArgs a) {
     grid_dependency_sync();
@@ -41,46 +98,12 @@ __global__ void __launch_bounds__(THREADS) precise_chunk_sums_kernel(PreciseArgs
     const long long pairs = (total + 1) / 2;
     for (long long pi = blockIdx.x; pi < pairs; pi += gridDim.x) {
         const long long item = 2 * pi + sub;
-        bool work = item < total;
-        int c = 0, src_row = 0;
-        if (work) {
-            c = (int)(item % a.nch);
-            const long long t = item / a.nch;
-            const int ri = (int)(t % a.expand);
-            const int e = a.queue[(int)(t / a.expand)] & 0x1FFFFFFF;     // (the verify path keeps flags above the index)
-            if (a.need_rows && !a.pos && ri < 64 && !((a.need_rows[e] >> ri) & 1ull)) work = false;
-            if (!a.pos && (ri < a.r0 || ri >= a.r1 || (a.gamma && ri > a.gamma[e]))) work = false;
-            src_row = a.pos ? e * a.seq_rows + a.pos[e] : e * a.expand + ri;
-        }
-        double s = 0.0;
-        if (work) {
-            const int b = src_row / a.seq_rows;
-            const T* row = reinterpret_cast<const T*>(a.logits) + (long long)src_row * a.row_stride;
-            // x = l * (1/T) instead of l / T: one rounding of 2^-53 more per term, far below every
-            // threshold this pass decides; four independent sums keep the exp pipeline busy
-            const double rT = 1.0 / (double)a.temperature[b];
-            const double m = (double)a.row_max[src_row] * rT;
-            const int v0 = c * CHUNK + quarter * (CHUNK / 4);
-            double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-#pragma unroll
-            for (int k = lane; k < CHUNK / 4; k += 128) {
-                const int v = v0 + k;
-                float l0 = -CUDART_INF_F, l1 = -CUDART_INF_F, l2 = -CUDART_INF_F, l3 = -CUDART_INF_F;
-                if (v < a.V) l0 = load_logit(row, v);
-                if (v + 32 < a.V) l1 = load_logit(row, v + 32);
-                if (v + 64 < a.V) l2 = load_logit(row, v + 64);
-                if (v + 96 < a.V) l3 = load_logit(row, v + 96);
-                s0 += exp((double)l0 * rT - m);
-                s1 += exp((double)l1 * rT - m);
-                s2 += exp((double)l2 * rT - m);
-                s3 += exp((double)l3 * rT - m);
-            }
-            s = warp_sum((s0 + s1) + (s2 + s3));
-        }
+        int qslot;
+        const double s = precise_item_sum<T>(a, item, total, quarter, lane, qslot);
         if (lane == 0) part[warp] = s;
         __syncthreads();
-        if (work && quarter == 0 && lane == 0)
-            a.dsum[(long long)src_row * (a.pitch > 0 ? a.pitch : a.nch) + c] = (part[warp] + part[warp + 1]) + (part[warp + 2] + part[warp + 3]);
+        if (item < total && quarter == 0 && lane == 0)
+            precise_item_store(a, item, (part[warp] + part[warp + 1]) + (part[warp + 2] + part[warp + 3]));
         __syncthreads();
     }
 }

@@ -83,7 +83,8 @@ __device__ __forceinline__ bool streamed_row(const VerifyArgs& a, int r, int& b,
 
 // index of the record of (row, chunk c of the vocabulary) in stats / dsum
 __device__ __forceinline__ long long record_index(const VerifyArgs& a, int row, int c) {
-    const int L = a.chunks_per_rank > 0 ? a.chunks_per_rank : a.nch;
+    if (a.chunks_per_rank == 0) return (long long)row * a.nch + c;      // one rank: the plain layout
+    const int L = a.chunks_per_rank;
     const int r = c / L;
     return (long long)r * a.rank_stride + (long long)row * L + (c - r * L);
 }
@@ -412,16 +413,14 @@ __device__ __forceinline__ int level2_draw(const VerifyArgs& a, const T* row, in
     return token;
 }
 
-template <typename T, bool PRECISE>
-__global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
-    extern __shared__ double cm[];  // [nch] chunk masses of the sampled row
-    __shared__ FinishShared sh;
+// One sequence (fast pass: sequence `slot`; double-precision pass: entry `slot` of the queue), by the
+// 256 threads of a CTA.  cm: [nch] doubles of shared memory (chunk masses of the sampled row).
+// SHARDED: vocabulary-parallel verification (a.entry_logits and a.pick are set).
+template <typename T, bool PRECISE, bool SHARDED>
+__device__ __forceinline__ void verify_finish_slot(const VerifyArgs& a, int slot, FinishShared& sh, double* cm) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int G = a.G, G1 = a.G + 1;
-    grid_dependency_sync();
-
-    const int nloop = PRECISE ? *a.queue_count : a.B;
-    for (int slot = blockIdx.x; slot < nloop; slot += gridDim.x) {
+    {
         // a queue entry is the sequence, with QUEUE_DRAW_ONLY set when only the draw was too close to
         // call: then the accept decisions of the fast pass stand and only the sampled row is redone;
         // with QUEUE_MASS_ONLY every decision stands and only small residual masses are recomputed
@@ -434,16 +433,18 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
         if (!a.sample_only && a.state_in && a.state_in[b] == 0) {
             // decided by an earlier call: nothing of this sequence is read or written
             if (tid == 0 && a.state_out) a.state_out[b] = 0;
-            continue;
+            return;
         }
         const float Tb = a.temperature[b];
         const float c32 = temp_scale(Tb);
         const T* seq = reinterpret_cast<const T*>(a.logits) + (long long)b * G1 * a.row_stride;
         unsigned st_bits = 0;
         if (!temp_ok(Tb)) st_bits |= ST_TEMPERATURE;
-        // a wait of the streaming pass ran out (now or in a call since the status word was last
-        // cleared): its statistics are not complete, nothing of this call is valid
-        if (*(volatile unsigned*)a.status & ST_INTERNAL) st_bits |= ST_INTERNAL;
+        // (requested now, looked at when the outputs are written)
+        const unsigned status_word = *(volatile unsigned*)a.status;
+        // the two uniforms of the draw, requested long before the chunk masses are ready
+        const float u_chunk = a.u_resample ? a.u_resample[2 * b] : 0.f;
+        const float u_entry = a.u_resample ? a.u_resample[2 * b + 1] : 0.f;
         // rows lo .. row_hi-1 are read, positions lo .. hi-1 are tested; g is the bonus row
         const int lo = a.sample_only ? 0 : a.r0;
         const int g = (!a.sample_only && a.gamma) ? a.gamma[b] : G;
@@ -513,8 +514,8 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 float qx = 0.f, qx_mine = 0.f;
                 int kx = 0x7fffffff;
                 // p(x) on every lane (the same instructions as on one lane, and no divergent tail)
-                const float* ent = a.entry_logits ? a.entry_logits + (long long)ri * (a.k_max + 1) : nullptr;
-                const float lx = range_bad ? -CUDART_INF_F : (ent ? ent[a.k_max] : load_logit(row, x));
+                const float* ent = SHARDED ? a.entry_logits + (long long)ri * (a.k_max + 1) : nullptr;
+                const float lx = range_bad ? -CUDART_INF_F : (SHARDED ? ent[a.k_max] : load_logit(row, x));
                 if (!range_bad) {
                     for (int k0 = 0; k0 < n; k0 += 256) {
                         if (k0 > 0) {
@@ -530,7 +531,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                             if (k0 + u * 32 + lane >= n) vv[u] = -2;
                             const bool ok = vv[u] >= 0 && vv[u] < a.V;
                             if (vv[u] != -2 && !ok) range_bad = true;
-                            ll[u] = ok ? (ent ? ent[k0 + u * 32 + lane] : load_logit(row, vv[u])) : -CUDART_INF_F;
+                            ll[u] = ok ? (SHARDED ? ent[k0 + u * 32 + lane] : load_logit(row, vv[u])) : -CUDART_INF_F;
                         }
 #pragma unroll
                         for (int u = 0; u < 8; ++u) {
@@ -585,7 +586,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
         }
         __syncthreads();
         st_bits |= (unsigned)sh.bad;
-        if (mass_only) continue;        // (bad data was reported by the fast pass already)
+        if (mass_only) return;          // (bad data was reported by the fast pass already)
 
         // ---- 3. first-rejection scan -----------------------------------------------------
         // A rejection inside the range decides the sequence; so does accepting every position
@@ -614,7 +615,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
         int pick_row = 0, pick_chunk = -1;      // vocabulary-parallel: what the picked chunk's owner needs
         bool pick_resid = false;
         double Rtot = -1.0;
-        const bool want_token = a.token != nullptr || a.pick != nullptr;
+        const bool want_token = SHARDED || a.token != nullptr;
         if (!st_bits && want_token && decided) {
             const int j = a.sample_only ? jpos : alen;
             const int rj = b * G + j;
@@ -659,12 +660,12 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                             vv[u] = k < n ? idx[k] : -2;
                             qq[u] = k < n ? prob[k] : 0.f;
                         }
-                        const float* ent = a.entry_logits ? a.entry_logits + (long long)rj * (a.k_max + 1) : nullptr;
+                        const float* ent = SHARDED ? a.entry_logits + (long long)rj * (a.k_max + 1) : nullptr;
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
                             const bool ok = vv[u] >= 0 && vv[u] < a.V;
                             if (vv[u] != -2 && !ok) rb = true;
-                            ll[u] = ok ? (ent ? ent[tid + u * THREADS] : load_logit(row, vv[u])) : -CUDART_INF_F;
+                            ll[u] = ok ? (SHARDED ? ent[tid + u * THREADS] : load_logit(row, vv[u])) : -CUDART_INF_F;
                         }
 #pragma unroll
                         for (int u = 0; u < 4; ++u)
@@ -694,7 +695,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                         if (lane >= d) incl += y;
                     }
                     const double R = __shfl_sync(0xffffffffu, incl, 31);
-                    const double thr = (double)a.u_resample[2 * b] * R;
+                    const double thr = (double)u_chunk * R;
                     double run = incl - s;
                     int first = 0x7fffffff, lastpos = -1;
                     double mind = 1e300;
@@ -738,14 +739,17 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
             pick_row = j;
             pick_chunk = cs;
             pick_resid = use_resid;
-            if (!st_bits && cs >= 0 && !a.pick) {
+            if (!st_bits && cs >= 0 && !SHARDED) {
                 token = level2_draw<T, PRECISE>(a, row, 0, cs, idx, prob, n, use_resid, wt, invZ,
-                                                a.u_resample[2 * b + 1], sh);
+                                                u_entry, sh);
             }
             flagged |= sh.flag != 0;
         }
 
         // ---- 5. outputs --------------------------------------------------------------------
+        // a wait of the streaming pass ran out (now or in a call since the status word was last
+        // cleared): its statistics are not complete, nothing of this call is valid
+        if (status_word & ST_INTERNAL) st_bits |= ST_INTERNAL;
         if (tid == 0) {
             if (st_bits) {
                 atomicOr(a.status, st_bits);
@@ -758,7 +762,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                     if (a.state_out) a.state_out[b] = 0;
                 }
                 if (a.token) a.token[b] = -1;
-                if (a.pick) {
+                if (SHARDED) {
                     a.pick[4 * b + 0] = 0;
                     a.pick[4 * b + 1] = -1;
                     a.pick[4 * b + 2] = 0;
@@ -773,12 +777,12 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                 if (a.mass) a.mass[b] = (float)Rtot;
                 if (PRECISE) {
                     if (nborder && a.borderline) atomicAdd(a.borderline, nborder);
-                    if (a.pick) {
+                    if (SHARDED) {
                         a.pick[4 * b + 0] = pick_row;
                         a.pick[4 * b + 1] = (decided && want_token) ? pick_chunk : -1;
                         a.pick[4 * b + 2] = pick_resid ? PICK_RESIDUAL : 0;
                     }
-                } else if (flagged || a.pick) {
+                } else if (flagged || SHARDED) {
                     // Which rows need exact sums: an ambiguous accept test can move the first
                     // rejection anywhere from its position on, so every row from there; an ambiguous
                     // draw needs the sampled row only; a small residual mass its own row.
@@ -801,7 +805,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                             // (vocabulary-parallel: whether the draw inside the chunk is too close to call is
                             // only known to the chunk's owner later, so the sampled row is always listed)
                             const bool nr = i >= 64 || (first_amb >= 0 && i >= first_amb) || (i < hi && sh.small[i]) ||
-                                            ((sh.flag || a.pick) && want_token && decided && i == alen);
+                                            ((sh.flag || SHARDED) && want_token && decided && i == alen);
                             if (nr) {
                                 if (i < 64) nd |= 1ull << i;
                                 ++nrows;
@@ -809,7 +813,7 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
                         }
                     }
                     a.need_rows[b] = nd;
-                    if (a.pick) {
+                    if (SHARDED) {
                         // the queue is built once the owners' flags have been exchanged
                         a.pick[4 * b + 0] = pick_row;
                         a.pick[4 * b + 1] = (decided && want_token) ? pick_chunk : -1;
@@ -825,6 +829,15 @@ __global__ void __launch_bounds__(THREADS) verify_finish_kernel(VerifyArgs a) {
             }
         }
     }
+}
+
+template <typename T, bool PRECISE, bool SHARDED = false>
+__global__ void __launch_bounds__(THREADS, 2) verify_finish_kernel(VerifyArgs a) {
+    extern __shared__ double cm[];  // [nch] chunk masses of the sampled row
+    __shared__ FinishShared sh;
+    grid_dependency_sync();
+    const int nloop = PRECISE ? *a.queue_count : a.B;
+    for (int slot = blockIdx.x; slot < nloop; slot += gridDim.x) verify_finish_slot<T, PRECISE, SHARDED>(a, slot, sh, cm);
 }
 
 }  // namespace picospec

@@ -352,7 +352,7 @@ PICOSPEC_API int picospec_vp_draw(picospec_ctx* ctx, const void* slice_logits, p
                                   const float* records_all, const double* sums_all, const float* temperature,
                                   const int* q_idx, const float* q_prob, const int* q_count, int k_max,
                                   const float* u_resample, const int* pick, int* tok_flag_local, void* cuda_stream);
-PICOSPEC_API int picospec_vp_queue(picospec_ctx* ctx, int B, const int* pick, const int* tok_flag_all, int* token,
+PICOSPEC_API int picospec_vp_queue(picospec_ctx* ctx, int B, int G, const int* pick, const int* tok_flag_all, int* token,
                                    void* cuda_stream);
 PICOSPEC_API int picospec_vp_exact(picospec_ctx* ctx, const void* slice_logits, picospec_dtype dtype, int B, int G, int Vs,
                                    long long row_stride_elems, int chunks_per_rank, const float* temperature,

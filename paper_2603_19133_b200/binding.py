@@ -69,7 +69,7 @@ def lib() -> ctypes.CDLL:
                                          vp, vp, vp, vp, vp, vp, vp, vp]
         L.picospec_vp_draw.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_int, c_ll, c_int, c_int, c_int, vp, vp, vp,
                                        vp, vp, vp, c_int, vp, vp, vp, vp]
-        L.picospec_vp_queue.argtypes = [vp, c_int, vp, vp, vp, vp]
+        L.picospec_vp_queue.argtypes = [vp, c_int, c_int, vp, vp, vp, vp]
         L.picospec_vp_exact.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_ll, c_int, vp, vp, vp]
         L.picospec_vp_merge.argtypes = [vp, c_int, vp, vp, vp]
         for f in ("picospec_vp_local", "picospec_vp_decide", "picospec_vp_draw", "picospec_vp_queue",

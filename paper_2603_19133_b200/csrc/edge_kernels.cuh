@@ -150,6 +150,7 @@ __global__ void __launch_bounds__(THREADS) edge_finish_kernel(VerifyArgs a) {
                 if (!PRECISE && sflag) {
                     a.need_rows[b] = ~0ull;
                     a.queue[atomicAdd(a.queue_count, 1)] = b;
+                    a.rowq[atomicAdd(a.rowq_count, 1)] = b * G1 + j;
                     atomicAdd(a.slow_rows, 1ull);
                 }
             }

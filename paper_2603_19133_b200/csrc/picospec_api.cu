@@ -47,6 +47,7 @@ struct picospec_ctx {
     int* wire_off;                  // wire codec: first entry of each row, [rows + 1]
     int* vp_listed;                 // vocabulary-parallel verify: per sequence, its kind in the double-precision pass
     int* tickets;                   // compress: per queue slot, chunk sums completed in the double-precision cut
+    int* rowq;                      // verify: rows whose exact chunk sums are wanted (count: counters[5])
     long long max_rows;
     unsigned* status;
     unsigned long long* slow_rows;
@@ -218,9 +219,8 @@ cudaError_t launch_compress(picospec_ctx* ctx, const CompressArgs& a, bool align
     // rows whose top-p cut was too close to call: exact normaliser, then redo the cut
     PreciseArgs p;
     p.logits = a.logits; p.row_stride = a.row_stride; p.V = a.V; p.nch = a.nch;
-    p.seq_rows = a.G; p.expand = 1; p.pos = nullptr; p.temperature = a.temperature;
-    p.queue = a.queue; p.queue_count = a.queue_count; p.row_max = a.row_max; p.dsum = a.dsum;
-    p.need_rows = nullptr;
+    p.seq_rows = a.G; p.temperature = a.temperature;
+    p.rows = a.queue; p.row_count = a.queue_count; p.row_max = a.row_max; p.dsum = a.dsum;
     // exact sums and the cut of the queued rows in one kernel
     launch_chained(compress_precise_kernel<T>, ctx->num_sms * 6, THREADS, MAX_K * 8, s, a, p);
     return cudaGetLastError();
@@ -270,12 +270,8 @@ cudaError_t launch_verify(picospec_ctx* ctx, const VerifyArgs& a, bool aligned, 
     ProfScope ps3(ctx, PICOSPEC_PROF_VERIFY_PRECISE, 2, s);
     PreciseArgs p;
     p.logits = a.logits; p.row_stride = a.row_stride; p.V = a.V; p.nch = a.nch;
-    p.seq_rows = a.G + 1; p.expand = a.sample_only ? 1 : a.G + 1; p.pos = a.sample_only ? a.pos : nullptr;
-    p.temperature = a.temperature; p.queue = a.queue; p.queue_count = a.queue_count;
-    p.need_rows = a.need_rows;
-    if (!a.sample_only) {
-        p.r0 = a.r0; p.r1 = a.r1; p.gamma = a.gamma;
-    }
+    p.seq_rows = a.G + 1; p.temperature = a.temperature;
+    p.rows = a.rowq; p.row_count = a.rowq_count;
     p.row_max = a.row_max; p.dsum = a.dsum;
     launch_chained(precise_chunk_sums_kernel<T>, ctx->num_sms * 6, THREADS, 0, s, p);
     const int g2 = a.B < ctx->num_sms ? a.B : ctx->num_sms;
@@ -350,6 +346,7 @@ int picospec_create(picospec_ctx** out, int device, int max_batch, int max_gamma
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->wire_off, (rows + 1) * sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->vp_listed, (size_t)max_batch * sizeof(int));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->tickets, rows * sizeof(int));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->rowq, rows * sizeof(int));
     ctx->max_rows = (long long)rows;
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->status, sizeof(unsigned));
     if (e == cudaSuccess) e = cudaMalloc((void**)&ctx->slow_rows, 2 * sizeof(unsigned long long));   // [0] slow rows, [1] redo rows
@@ -385,6 +382,7 @@ int picospec_destroy(picospec_ctx* ctx) {
     cudaFree(ctx->wire_off);
     cudaFree(ctx->vp_listed);
     cudaFree(ctx->tickets);
+    cudaFree(ctx->rowq);
     cudaFree(ctx->status);
     cudaFree(ctx->slow_rows);
     free(ctx);
@@ -599,7 +597,7 @@ static int verify_common(picospec_ctx* ctx, VerifyArgs& a, picospec_dtype dtype,
     a.nch = (a.V + CHUNK - 1) / CHUNK;
     if (a.r1 < 0) a.r1 = a.G + 1;
     a.stats = ctx->stats; a.row_max = ctx->row_max; a.dsum = ctx->dsum; a.queue = ctx->queue;
-    a.need_rows = ctx->need_rows;
+    a.need_rows = ctx->need_rows; a.rowq = ctx->rowq; a.rowq_count = ctx->counters + 5;
     a.queue_count = ctx->counters; a.status = ctx->status; a.slow_rows = ctx->slow_rows;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     cudaError_t e;
@@ -738,6 +736,7 @@ static void vp_args(picospec_ctx* ctx, VerifyArgs& a, int B, int G, int V, int k
     a.chunks_per_rank = chunks_per_rank;
     a.rank_stride = (long long)B * (G + 1) * chunks_per_rank;
     a.row_max = ctx->row_max; a.queue = ctx->queue; a.need_rows = ctx->need_rows;
+    a.rowq = ctx->rowq; a.rowq_count = ctx->counters + 5;
     a.queue_count = ctx->counters; a.status = ctx->status; a.slow_rows = ctx->slow_rows;
     a.pos = nullptr; a.mass = nullptr; a.token = nullptr;
     a.draft_tok = nullptr; a.q_idx = nullptr; a.q_prob = nullptr; a.q_count = nullptr;
@@ -851,14 +850,15 @@ int picospec_vp_draw(picospec_ctx* ctx, const void* slice_logits, picospec_dtype
     return e == cudaSuccess ? PICOSPEC_OK : fail_cuda(ctx, e);
 }
 
-int picospec_vp_queue(picospec_ctx* ctx, int B, const int* pick, const int* tok_flag_all, int* token, void* cuda_stream) {
-    if (!ctx || B < 0 || !pick || !tok_flag_all || !token) return PICOSPEC_EINVAL;
-    if (B > ctx->max_batch) return PICOSPEC_ECAPACITY;
+int picospec_vp_queue(picospec_ctx* ctx, int B, int G, const int* pick, const int* tok_flag_all, int* token,
+                      void* cuda_stream) {
+    if (!ctx || B < 0 || G < 0 || !pick || !tok_flag_all || !token) return PICOSPEC_EINVAL;
+    if (B > ctx->max_batch || G > ctx->max_gamma) return PICOSPEC_ECAPACITY;
     if (B == 0) return PICOSPEC_OK;
     DeviceGuard g(ctx->device);
     if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
     VerifyArgs a;
-    vp_args(ctx, a, B, 0, 1, 1, 1);
+    vp_args(ctx, a, B, G, 1, 1, 1);
     a.pick = const_cast<int*>(pick);
     a.token = token;
     launch_chained(vp_queue_kernel, 1, THREADS, 0, (cudaStream_t)cuda_stream, a, tok_flag_all, ctx->vp_listed);
@@ -878,8 +878,8 @@ int picospec_vp_exact(picospec_ctx* ctx, const void* slice_logits, picospec_dtyp
     if (!g.ok) return fail_cuda(ctx, cudaErrorInvalidDevice);
     PreciseArgs p;
     p.logits = slice_logits; p.row_stride = row_stride_elems; p.V = Vs; p.nch = (Vs + CHUNK - 1) / CHUNK;
-    p.seq_rows = G + 1; p.expand = G + 1; p.pos = nullptr; p.temperature = temperature;
-    p.queue = ctx->queue; p.queue_count = ctx->counters; p.need_rows = ctx->need_rows;
+    p.seq_rows = G + 1; p.temperature = temperature;
+    p.rows = ctx->rowq; p.row_count = ctx->counters + 5;
     p.row_max = ctx->row_max; p.dsum = sums_local; p.pitch = chunks_per_rank;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     if (dtype == PICOSPEC_BF16) launch_chained(precise_chunk_sums_kernel<__nv_bfloat16>, ctx->num_sms * 6, THREADS, 0, s, p);
@@ -915,6 +915,7 @@ struct StaticWorkspace {
     double dsum[STATIC_ROWS * STATIC_NCH];
     float row_max[STATIC_ROWS];
     int queue[STATIC_ROWS];
+    int rowq[STATIC_ROWS];
     unsigned long long need_rows[STATIC_ROWS];
     // the words below must read zero when a call starts; one memset covers them
     int counters[4];
@@ -993,7 +994,7 @@ extern "C" int picospec_verify_static(const void* target_logits, picospec_dtype 
     a.accept_len = accept_len; a.p_draft = p_draft; a.resid_mass = resid_mass; a.borderline = borderline_count;
     a.token = token; a.mass = nullptr;
     a.stats = ws->stats; a.row_max = ws->row_max; a.dsum = ws->dsum; a.queue = ws->queue;
-    a.need_rows = ws->need_rows;
+    a.need_rows = ws->need_rows; a.rowq = ws->rowq; a.rowq_count = ws->counters + 1;
     a.queue_count = ws->counters; a.status = &ws->status; a.slow_rows = &ws->slow_rows;
     cudaError_t e;
     if (dtype == PICOSPEC_BF16)

@@ -1,5 +1,5 @@
 // Double-precision chunk sums for rows whose fp32 statistics were too close to a decision
-// threshold.  Four warps per (queued row, chunk): sum of exp(l/T - max/T) over the chunk, exactly
+// threshold.  Four warps per (listed row, chunk): sum of exp(l/T - max/T) over the chunk, exactly
 // the terms of the definition.  The whole grid shares the work, so a handful of flagged rows
 // costs microseconds; with an empty queue every CTA returns at once.
 #pragma once
@@ -12,40 +12,25 @@ struct PreciseArgs {
     long long row_stride;
     int V, nch;
     int seq_rows;              // rows per sequence in the logits tensor (G or G+1)
-    int expand;                // rows per queue entry: entry e covers rows e*expand .. +expand-1
-    const int* pos;            // optional: entry b covers the single row b*seq_rows + pos[b]
     const float* temperature;  // [B]
-    const int* queue;
-    const int* queue_count;
-    const unsigned long long* need_rows;   // optional [entries]: bit ri = row ri of the entry is wanted
-    // optional row window of an entry: rows outside [r0, r1), or beyond gamma[entry], are never read
-    int r0 = 0, r1 = 0x7fffffff;
-    const int* gamma = nullptr;
+    const int* rows;           // the rows whose exact chunk sums are wanted (indices into the logits tensor)
+    const int* row_count;      // how many
     const float* row_max;      // [rows] exact row maxima from the fp32 pass
-    double* dsum;              // [rows, nch]
+    double* dsum;              // [rows, pitch]
     int pitch = 0;             // chunk sums per row in dsum (0: nch)
 };
 
-// One quarter of one item of the double-precision pass, by one warp.  Item = (queue entry, row of
-// the entry, chunk); returns the partial sum (0 for a row that is not wanted) and the queue slot.
+// One quarter of one item of the double-precision pass, by one warp.  Item = (listed row, chunk);
+// returns the partial sum and the position of the row in the list.
 template <typename T>
 __device__ __forceinline__ double precise_item_sum(const PreciseArgs& a, long long item, long long total, int quarter,
                                                    int lane, int& qslot) {
-    bool work = item < total;
-    int c = 0, src_row = 0;
     qslot = -1;
-    if (work) {
-        c = (int)(item % a.nch);
-        const long long t = item / a.nch;
-        const int ri = (int)(t % a.expand);
-        qslot = (int)(t / a.expand);
-        const int e = a.queue[qslot] & 0x1FFFFFFF;     // (the verify path keeps flags above the index)
-        if (a.need_rows && !a.pos && ri < 64 && !((a.need_rows[e] >> ri) & 1ull)) work = false;
-        if (!a.pos && (ri < a.r0 || ri >= a.r1 || (a.gamma && ri > a.gamma[e]))) work = false;
-        src_row = a.pos ? e * a.seq_rows + a.pos[e] : e * a.expand + ri;
-    }
     double s = 0.0;
-    if (work) {
+    if (item < total) {
+        const int c = (int)(item % a.nch);
+        qslot = (int)(item / a.nch);
+        const int src_row = a.rows[qslot] & 0x1FFFFFFF;     // (a list may keep flags above the index)
         const int b = src_row / a.seq_rows;
         const T* row = reinterpret_cast<const T*>(a.logits) + (long long)src_row * a.row_stride;
         // x = l * (1/T) instead of l / T: one rounding of 2^-53 more per term, far below every
@@ -71,22 +56,17 @@ __device__ __forceinline__ double precise_item_sum(const PreciseArgs& a, long lo
     }
     return s;
 }
-// where the sum of an item goes (rows that are not wanted are not written)
+// where the sum of an item goes
 __device__ __forceinline__ void precise_item_store(const PreciseArgs& a, long long item, double sum) {
     const int c = (int)(item % a.nch);
-    const long long t = item / a.nch;
-    const int ri = (int)(t % a.expand);
-    const int e = a.queue[(int)(t / a.expand)] & 0x1FFFFFFF;
-    if (a.need_rows && !a.pos && ri < 64 && !((a.need_rows[e] >> ri) & 1ull)) return;
-    if (!a.pos && (ri < a.r0 || ri >= a.r1 || (a.gamma && ri > a.gamma[e]))) return;
-    const int src_row = a.pos ? e * a.seq_rows + a.pos[e] : e * a.expand + ri;
+    const int src_row = a.rows[(int)(item / a.nch)] & 0x1FFFFFFF;
     a.dsum[(long long)src_row * (a.pitch > 0 ? a.pitch : a.nch) + c] = sum;
 }
 
 template <typename T>
 __global__ void __launch_bounds__(THREADS) precise_chunk_sums_kernel(PreciseArgs a) {
     grid_dependency_sync();
-    const int nq = *a.queue_count;
+    const int nq = *a.row_count;
     if (nq == 0) return;
     // A CTA takes two chunks at a time, four warps per chunk (a quarter of the chunk each, so that a
     // handful of rows still spreads over the whole GPU); the four partial sums of a chunk are added in
@@ -94,7 +74,7 @@ __global__ void __launch_bounds__(THREADS) precise_chunk_sums_kernel(PreciseArgs
     __shared__ double part[WARPS];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int sub = warp >> 2, quarter = warp & 3;
-    const long long total = (long long)nq * a.expand * a.nch;
+    const long long total = (long long)nq * a.nch;
     const long long pairs = (total + 1) / 2;
     for (long long pi = blockIdx.x; pi < pairs; pi += gridDim.x) {
         const long long item = 2 * pi + sub;

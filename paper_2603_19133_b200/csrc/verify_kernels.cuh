@@ -51,6 +51,8 @@ struct VerifyArgs {
     int* queue;                // [B] flagged sequences
     unsigned long long* need_rows;  // [B] per flagged sequence: bit i = row i needs exact chunk sums
     int* queue_count;          // [1]
+    int* rowq;                 // [B*(G+1)] rows (of the logits tensor) whose exact chunk sums are wanted
+    int* rowq_count;           // [1]
     unsigned* status;          // sticky status word
     unsigned long long* slow_rows;  // cumulative rows re-evaluated in double precision
 };
@@ -135,6 +137,7 @@ __global__ void __launch_bounds__(THREADS, 4) chunk_stats_kernel(VerifyArgs a) {
     const long long nw = (long long)gridDim.x * WARPS;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         *a.queue_count = 0;
+        *a.rowq_count = 0;
         if (a.borderline) *a.borderline = 0;
     }
     const long long total = (long long)(a.sample_only ? a.B : a.B * (a.r1 - a.r0)) * a.nch;
@@ -199,6 +202,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, StreamCfg<T>::CTAS_PER_SM) chu
     grid_dependency_sync();
     if (tid == 0 && blockIdx.x == 0) {
         *a.queue_count = 0;
+        *a.rowq_count = 0;
         if (a.borderline) *a.borderline = 0;
     }
     __syncthreads();
@@ -792,6 +796,7 @@ __device__ __forceinline__ void verify_finish_slot(const VerifyArgs& a, int slot
                     if (a.sample_only) {
                         nd = ~0ull;
                         nrows = 1;
+                        a.rowq[atomicAdd(a.rowq_count, 1)] = b * G1 + jpos;
                     } else {
                         int first_amb = -1;
                         const int last = rejected ? alen : hi - 1;
@@ -809,6 +814,7 @@ __device__ __forceinline__ void verify_finish_slot(const VerifyArgs& a, int slot
                             if (nr) {
                                 if (i < 64) nd |= 1ull << i;
                                 ++nrows;
+                                if (!SHARDED) a.rowq[atomicAdd(a.rowq_count, 1)] = b * G1 + i;
                             }
                         }
                     }

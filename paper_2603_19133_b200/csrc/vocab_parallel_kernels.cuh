@@ -153,7 +153,20 @@ __global__ void __launch_bounds__(THREADS) vp_queue_kernel(VerifyArgs a, const i
         __syncthreads();
     }
     if (rows) atomicAdd(a.slow_rows, rows);
-    if (tid == 0) *a.queue_count = carry;
+    if (tid == 0) {
+        *a.queue_count = carry;
+        *a.rowq_count = 0;
+    }
+    __syncthreads();
+    // the rows of the listed sequences that need exact chunk sums (any order: every rank sums its
+    // own slice of each, and the results are exchanged as whole arrays)
+    const int G1 = a.G + 1;
+    for (int b = tid; b < a.B; b += THREADS) {
+        if (!listed[b]) continue;
+        const unsigned long long nd = a.need_rows[b];
+        for (int i = 0; i < G1; ++i)
+            if (i >= 64 || ((nd >> i) & 1ull)) a.rowq[atomicAdd(a.rowq_count, 1)] = b * G1 + i;
+    }
 }
 
 // After the exchange of the double-precision pass's tokens: they replace the fast ones.

@@ -155,7 +155,7 @@ def verify_sharded(states: Sequence[RankState], exch, temperature, draft_tok, q_
     tf_a = exch.maximum(tf_l)
     for i, s in enumerate(states):
         with torch.cuda.device(dev(i)):
-            _b._check(L.picospec_vp_queue(s.ctx._h, B, P(pick[i]), P(tf_a[i]), P(out[i]["token"]), stream()),
+            _b._check(L.picospec_vp_queue(s.ctx._h, B, G, P(pick[i]), P(tf_a[i]), P(out[i]["token"]), stream()),
                       "picospec_vp_queue")
 
     # 3. double-precision pass over the listed sequences (an empty list costs a few empty kernels)

@@ -530,6 +530,49 @@ def bench_pipelined(ps, w, device, n_streams, iters):
             "verify_stream_bytes_GBps": alg["verify_stream"] * nsteps / sec / 1e9, "device_status": status}
 
 
+def bench_vocab_parallel(ps, w, device, ranks, iters):
+    """Vocabulary-parallel verification (Sec. 4.1: the verifier spans several GPUs) with the slices of
+    all ranks in this one GPU's memory and the exchanges done as copies: every kernel of the path runs
+    as it would on `ranks` devices, one rank after the other, so the time of a call divided by `ranks`
+    approximates one rank's compute; the NCCL transport itself is not measured here."""
+    from paper_2603_19133_b200 import vocab_parallel as vp
+    inp = gen.make_inputs(w, seed=7300, device=device)
+    ctx0 = ps.Context(w.B, w.G, w.V, w.k_max)
+    qi, qp, qc, tok = ctx0.compress(inp["draft_logits"], inp["temperature"], w.top_k, w.top_p, w.k_max, inp["u_draft"])
+    ctx0.close()
+    ctxs = [ps.Context(w.B, w.G, w.V, w.k_max) for _ in range(ranks)]
+    states = []
+    for r in range(ranks):
+        v0, v1 = vp.slice_bounds(w.V, ranks, r)
+        states.append(vp.RankState(ctxs[r], r, ranks, w.V, inp["target_logits"][:, :, v0:v1].contiguous()))
+    rep = lambda t: [t] * ranks
+    exch = vp.LocalExchange(ranks)
+
+    def call():
+        return vp.verify_sharded(states, exch, rep(inp["temperature"]), rep(tok), rep(qi), rep(qp), rep(qc),
+                                 rep(inp["u_accept"]), rep(inp["u_resample"]))
+
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / iters
+    status = 0
+    for c in ctxs:
+        status |= c.status(clear=True)[0]
+        c.close()
+    slice_bytes = w.B * (w.G + 1) * (vp.slice_bounds(w.V, ranks, 0)[1]) * w.bytes_per_logit
+    return {"ranks": ranks, "us_per_call_all_ranks_on_one_gpu": us, "us_per_rank": us / ranks,
+            "slice_bytes_per_rank": slice_bytes, "kernels_per_rank_per_call": 12,
+            "exchanges_per_call": "2 all-gathers (chunk records, exact sums), 4 element-wise maxima",
+            "transport": "not measured: one GPU per run, the exchanges are copies", "device_status": status}
+
+
 def bench_paper_direction(ps, w, device, k, iters):
     """The paper's own data flow (Sec. 3.3) on the same shape, timed per call with CUDA events:
     picospec_target_topk (Top-K of the target row at one position per sequence, K = 10 as in the
@@ -642,11 +685,12 @@ def run_ours(args):
                                    roofline_launches=16)
                 others[ws.name] = summary_of(r, k_sweep)
 
-    paper_direction = wire_codec = None
+    paper_direction = wire_codec = vocab_parallel = None
     pipelined = {}
     if args.all_configs and world == 1:
         paper_direction = bench_paper_direction(ps, w, device, k=10, iters=min(args.steps, 200))
         wire_codec = bench_wire(ps, w, device, iters=min(args.steps, 200))
+        vocab_parallel = {f"ranks{r}": bench_vocab_parallel(ps, w, device, r, iters=min(args.steps, 20)) for r in (2, 4)}
         for name in ("config1", "config2"):
             try:
                 pipelined[name] = bench_pipelined(ps, gen.WORKLOADS[name], device, n_streams=4,
@@ -702,6 +746,7 @@ def run_ours(args):
             "pipelined": pipelined,
             "paper_direction": paper_direction,
             "wire_codec": wire_codec,
+            "vocab_parallel": vocab_parallel,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -420,6 +420,35 @@ def test_staged_shapes(ps, V, B, G, K, dtype, top_k, top_p):
     assert r["status"] == 0
 
 
+@pytest.mark.parametrize("rows,V,top_k,top_p", [
+    (445, 65536, 64, 1.0),      # one row more than the filter kernel has CTAs: that row is dealt in pieces
+    (445, 32768, 0, 0.9),       # the same with top-p (the pieces' exp-sums are put together) and two-tile pieces
+    (666, 32768, 200, 1.0),     # half a wave of remainder rows, each in two pieces; the exact first-tile search
+    (887, 40960, 16, 1.0),      # almost two whole rows per CTA: the remainder is not cut; ragged last tile
+    (300, 24576, 300, 1.0),     # fewer rows than CTAs, three tiles per row (too short to cut), large buffer shape
+    (97, 131072, 0, 0.95),      # few long rows: eight pieces each
+])
+def test_filter_plan_edge_cases(ps, rows, V, top_k, top_p):
+    # how the rows are dealt to the CTAs of the staged filter kernel (whole rows, then pieces of the
+    # remainder) must not show in the result: compress alone, every row against the oracle
+    K = max(top_k, 64)
+    g = torch.Generator(device="cuda").manual_seed(rows + V)
+    dl = (torch.randn((rows, 1, V), generator=g, device="cuda") * 2.5).to(torch.bfloat16)
+    T = 0.6 + 0.6 * torch.rand((rows,), generator=g, device="cuda")
+    u = torch.rand((rows, 1), generator=g, device="cuda")
+    ctx = ps.Context(rows, 1, V, K)
+    try:
+        qi, qp, qc, tok = ctx.compress(dl, T, top_k, top_p, K, u)
+        _, redo = ctx.counters(clear=True)
+        assert ctx.status(clear=True)[0] == 0
+        o_qi, o_qp, o_qc, o_tok = oracle.compress(_np(dl), _np(T), top_k, top_p, K, _np(u), nthreads=oracle.cores())
+        assert np.array_equal(_np(qc), o_qc) and np.array_equal(_np(qi), o_qi) and np.array_equal(_np(tok), o_tok)
+        np.testing.assert_allclose(_np(qp), o_qp, rtol=RTOL, atol=0)
+        assert redo == 0
+    finally:
+        ctx.close()
+
+
 @pytest.mark.parametrize("V,k,shift", [
     (32000, 8, 24.0),         # up to 256 survivors: one key per thread
     (128256, 64, 24.0),

@@ -603,6 +603,25 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(ps):
         ctx.close()
 
 
+def test_profile_brackets_return_every_launch(ps):
+    # picospec_profile_samples: one device time per bracketed launch, oldest first; a read resets
+    w = gen.scaled(gen.WORKLOADS["config2"], B=2)
+    inp = gen.make_inputs(w, seed=5, device="cuda")
+    ctx = ps.Context(w.B, w.G, w.V, w.k_max)
+    try:
+        ctx.profile_enable(2, every=1)
+        for _ in range(5):
+            qi, qp, qc, tok = ctx.compress(inp["draft_logits"], inp["temperature"], w.top_k, w.top_p, w.k_max, inp["u_draft"])
+            ctx.verify(inp["target_logits"], inp["temperature"], tok, qi, qp, qc, inp["u_accept"], inp["u_resample"])
+        for kind in range(7):
+            ms = ctx.profile_samples(kind)
+            assert len(ms) == 5 and all(0.0 < x < 50.0 for x in ms), (kind, ms)
+            assert ctx.profile_samples(kind) == []
+        ctx.profile_enable(0)
+    finally:
+        ctx.close()
+
+
 def test_staged_bad_data_is_reported(ps):
     # NaN and +inf inside rows that take the staged kernels (with and without the exp-sum)
     V, B, G, K = 16384, 4, 1, 16

@@ -216,8 +216,8 @@ __device__ __forceinline__ void emit_invalid_row(const CompressArgs& a, int row)
 // sit sorted in keys[0..k_eff).  Z is the row normaliser on the scale of Weight<PRECISE>
 // (ignored when top_p >= 1).  Returns (to thread 0, via sh.flag) whether the cut was too close
 // to call in the fast path.
-template <bool PRECISE>
-__device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int k_eff, float Tb, double Z,
+template <bool PRECISE, int E>
+__device__ void finish_row_ranks(const CompressArgs& a, int row, const u64* keys, int k_eff, float Tb, double Z,
                            CompressShared& sh) {
     const int tid = threadIdx.x;
     const float mx = key_logit(keys[0]);
@@ -229,11 +229,11 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
         sh.flag = 0;
         sh.n = k_eff;
     }
-    // four consecutive ranks per thread
-    double w[4], cum[4], loc = 0.0;
+    // E consecutive ranks per thread
+    double w[E], cum[E], loc = 0.0;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const int j = tid * 4 + e;
+    for (int e = 0; e < E; ++e) {
+        const int j = tid * E + e;
         w[e] = j < k_eff ? wt(key_logit(keys[j])) : 0.0;
         loc += w[e];
         cum[e] = loc;
@@ -244,15 +244,15 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
         const double thrZ = (double)a.top_p * Z;
         int mine = 0x7fffffff;
 #pragma unroll
-        for (int e = 3; e >= 0; --e)
-            if (tid * 4 + e < k_eff && base + cum[e] >= thrZ) mine = tid * 4 + e;
+        for (int e = E - 1; e >= 0; --e)
+            if (tid * E + e < k_eff && base + cum[e] >= thrZ) mine = tid * E + e;
         if (mine != 0x7fffffff) atomicMin(&sh.first, mine);
         workers_sync();
         const int jn = sh.first;   // rank of the entry that reaches top_p, if any
         if (jn != 0x7fffffff && jn == mine) {
             sh.n = jn + 1;
             if (!PRECISE) {
-                const int e = jn - tid * 4;
+                const int e = jn - tid * E;
                 const double E = GUARD_Z * thrZ;
                 const double hi = base + cum[e] - thrZ;
                 const double lo = thrZ - (base + cum[e] - w[e]);
@@ -267,17 +267,17 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
     }
     const int n = sh.n;
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
-        if (tid * 4 + e == n - 1) sh.Wn = base + cum[e];
+    for (int e = 0; e < E; ++e)
+        if (tid * E + e == n - 1) sh.Wn = base + cum[e];
     workers_sync();
     const double Wn = sh.Wn;
     // stored probabilities, and their running sum for the draft draw
-    float pf[4];
-    double ploc = 0.0, pcum[4];
+    float pf[E];
+    double ploc = 0.0, pcum[E];
     const double inv = 1.0 / (a.raw_probs ? Z : Wn);   // one division per row; 2^-53 relative per entry
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const int j = tid * 4 + e;
+    for (int e = 0; e < E; ++e) {
+        const int j = tid * E + e;
         pf[e] = j < n ? (float)(w[e] * inv) : 0.f;
         ploc += (double)pf[e];
         pcum[e] = ploc;
@@ -285,8 +285,8 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
     const bool flagged = !PRECISE && sh.flag;
     long long o = (long long)row * a.k_max;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const int j = tid * 4 + e;
+    for (int e = 0; e < E; ++e) {
+        const int j = tid * E + e;
         if (j < a.k_max) {
             // a flagged row keeps all k_eff sorted candidates so that the double-precision pass
             // can redo the cut without a second selection
@@ -295,7 +295,7 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
             a.q_prob[o + j] = pf[e];
         }
     }
-    for (int j = THREADS * 4 + tid; j < a.k_max; j += THREADS) {   // k_max <= 1024: never taken
+    for (int j = THREADS * E + tid; j < a.k_max; j += THREADS) {   // slots beyond the ranks the threads hold
         a.q_idx[o + j] = -1;
         a.q_prob[o + j] = 0.f;
     }
@@ -309,9 +309,9 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
         const double thr = (double)a.u_draft[row] * Ptot;
         int mine = 0x7fffffff, mylast = -1;
 #pragma unroll
-        for (int e = 3; e >= 0; --e) {
-            if (tid * 4 + e < n && pbase + pcum[e] > thr) mine = tid * 4 + e;
-            if (pf[e] > 0.f && mylast < 0) mylast = tid * 4 + e;
+        for (int e = E - 1; e >= 0; --e) {
+            if (tid * E + e < n && pbase + pcum[e] > thr) mine = tid * E + e;
+            if (pf[e] > 0.f && mylast < 0) mylast = tid * E + e;
         }
         if (mine != 0x7fffffff) atomicMin(&sh.first, mine);
         if (mylast >= 0) atomicMax(&sh.last, mylast);
@@ -332,6 +332,16 @@ __device__ void finish_row(const CompressArgs& a, int row, const u64* keys, int 
         }
     }
     workers_sync();
+}
+
+// (the ranks are spread over as many threads as there are: one per thread up to 256 candidates,
+// which shortens the serial part -- the exponentials and the running sums -- fourfold)
+template <bool PRECISE>
+__device__ __forceinline__ void finish_row(const CompressArgs& a, int row, const u64* keys, int k_eff, float Tb, double Z,
+                                           CompressShared& sh) {
+    if (k_eff <= THREADS) finish_row_ranks<PRECISE, 1>(a, row, keys, k_eff, Tb, Z, sh);
+    else if (k_eff <= 2 * THREADS) finish_row_ranks<PRECISE, 2>(a, row, keys, k_eff, Tb, Z, sh);
+    else finish_row_ranks<PRECISE, 4>(a, row, keys, k_eff, Tb, Z, sh);
 }
 
 template <typename T, bool ALIGNED, bool STATS>

@@ -777,7 +777,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config4", choices=sorted(gen.WORKLOADS))
-    ap.add_argument("--ref-sample", type=int, default=64, help="sequences per step of the CPU oracle legs")
+    ap.add_argument("--ref-sample", type=int, default=256,
+                    help="most sequences per step of the CPU oracle legs (256 of config 4: about 20 core-seconds)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override B of the workload (profiling on a small case)")
     ap.add_argument("--roofline-launches", type=int, default=64,

@@ -407,7 +407,10 @@ def test_near_threshold_uniforms_are_decided_exactly(ps):
     (8192, 3, 2, 64, "bf16", 64, 1.0),        # exactly one tile
     (8200, 3, 2, 64, "bf16", 0, 0.9),         # one entry-vector into the second tile
     (16392, 2, 3, 256, "bf16", 256, 1.0),     # last tile holds a single ragged chunk
-    (40960, 2, 2, 300, "bf16", 300, 1.0),     # k > 256: large candidate buffer
+    (40960, 2, 2, 300, "bf16", 300, 1.0),     # k in (256, 512]: still the small candidate buffer
+    (40960, 3, 2, 512, "bf16", 512, 1.0),     # the largest k of the small buffer (64 per warp in the first tile)
+    (49152, 2, 2, 600, "bf16", 600, 1.0),     # k > 512: large candidate buffer, two stages
+    (24576, 2, 2, 512, "f32", 512, 1.0),      # fp32, small buffer at its largest k
     (65536, 2, 1, 1024, "bf16", 0, 0.9999),   # widest rows, top-p that never cuts
     (12292, 2, 2, 32, "f32", 32, 1.0),        # fp32 tiles, ragged
     (20000, 2, 2, 700, "f32", 0, 0.95),       # fp32, large buffer, top-p

@@ -692,7 +692,7 @@ def test_draws_next_to_a_chunk_boundary_are_decided_exactly(ps):
 # seeded random shapes and value scales (staged and direct kernels, both dtypes, top-k / top-p)
 # ---------------------------------------------------------------------------------------------
 
-@pytest.mark.parametrize("seed", list(range(24)))
+@pytest.mark.parametrize("seed", list(range(48)))
 def test_random_shapes_and_scales(ps, seed):
     rng = np.random.default_rng(9000 + seed)
     dtype = "bf16" if rng.random() < 0.6 else "f32"
@@ -700,7 +700,7 @@ def test_random_shapes_and_scales(ps, seed):
     V = int(rng.choice([rng.integers(1500, 8192), rng.integers(8192, 20000), rng.integers(20000, 70000)]))
     if rng.random() < 0.7:
         V = V // align * align                      # rows the staged kernels take (when V >= 8192)
-    K = int(rng.choice([1, 3, 17, 64, 200, 256, 257, 600, 1024]))
+    K = int(rng.choice([1, 3, 17, 64, 200, 256, 257, 512, 513, 600, 1024]))
     K = min(K, V)
     B, G = int(rng.integers(1, 4)), int(rng.integers(1, 4))
     use_p = rng.random() < 0.5
